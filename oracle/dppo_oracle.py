@@ -1,0 +1,235 @@
+"""Float64 CPU oracle of the DPPO per-token loss path (numpy, one row at a time).
+
+TEST INFRASTRUCTURE ONLY: never imported by the product package; it shares no
+code with the CUDA library.  Everything is evaluated in float64 on the stored
+input values (fp32 / bf16 values are upcast exactly by the caller), with no
+blocking, fusion or reordering beyond what the definitions state.
+
+What each function restates (paper: "Rethinking the Trust Region in LLM
+Reinforcement Learning", DPPO):
+
+* ``log_softmax_row``           pi(.|s_t) is a distribution over the vocabulary (Sec. 3).
+* ``ratio``                     r_t = pi(a_t)/mu(a_t)                      (Eq. ppo-clip).
+* ``binary_tv`` / ``binary_kl`` Bernoulli collapse on the sampled token    (Eq. binary_tv, Eq. binary_kl).
+* ``topk_reduced``              A'_t = TopK(mu, K) u {a_t} plus "other"    (Sec. 4.4, Top-K Approximation).
+* ``topk_tv`` / ``topk_kl``     divergences of the reduced categoricals    (Eq. topk_tv, Eq. topk_kl).
+* ``full_tv`` / ``full_kl``     exact full-vocabulary divergences          (App. B definitions).
+* ``dppo_mask``                 asymmetric trust-region mask               (Eq. dppo_obj).
+* ``dppo_row`` / ``dppo_loss_fwd_bwd``  surrogate and its logits-gradient   (Eq. dppo_obj, Eq. unified_grad with C = inf).
+* ``dppo_fused_lmhead_fwd_bwd`` the same applied to logits = H W with the chain rule into H and W.
+
+Readings of points the paper leaves open (each is listed in the design notes):
+the library *minimises*, so loss = -s * sum_t M_t r_t A_t with a caller scale s
+(default 1/N_valid); M_t is a constant with respect to the logits; comparisons
+are strict as printed; r_t >< 1 is decided as log pi(a_t) >< log mu(a_t);
+x*log(x/y) = 0 when x = 0 and +inf when x > 0 = y; "other" masses are clamped
+to [0, 1]; the sampled token is never counted twice when it is in the top-K
+list, where the list's stored probability is used for it.
+
+Parity pins: every function above is pinned by tests/test_oracle_pins.py
+(printed worked example, closed forms, App. B invariants, library routines,
+finite differences, brute force); nothing here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL = 0, 1, 2, 3
+VARIANT_NAMES = {BINARY_TV: "binary_tv", BINARY_KL: "binary_kl", TOPK_TV: "topk_tv", TOPK_KL: "topk_kl"}
+
+
+def _f64(x):
+    return np.asarray(x, dtype=np.float64)
+
+
+def log_softmax_row(z):
+    """log pi_j = z_j - lse, lse = m + log sum_j exp(z_j - m), m = max_j z_j.
+
+    Returns (log_pi[V], lse).  Two plain sweeps over one logits row (Sec. 3:
+    the policy is a categorical distribution over the vocabulary).
+    """
+    z = _f64(z)
+    m = np.max(z)
+    S = np.sum(np.exp(z - m))
+    lse = m + np.log(S)
+    return z - lse, lse
+
+
+def ratio(log_pi_a, mu_logp):
+    """r_t = pi(a_t|s_t) / mu(a_t|s_t)  (Eq. ppo-clip), from the two log-probs."""
+    return float(np.exp(float(log_pi_a) - float(mu_logp)))
+
+
+def _xlogx_over_y(x, y):
+    """x * log(x / y) with 0*log(0/y) = 0 and x*log(x/0) = +inf for x > 0."""
+    x = float(x)
+    y = float(y)
+    if x == 0.0:
+        return 0.0
+    if y == 0.0:
+        return float("inf")
+    return x * (np.log(x) - np.log(y))
+
+
+def binary_tv(mu_a, pi_a):
+    """Eq. binary_tv: | mu(a_t) - pi(a_t) |."""
+    return abs(float(mu_a) - float(pi_a))
+
+
+def binary_kl(mu_a, pi_a):
+    """Eq. binary_kl: KL between the Bernoulli collapses (mu(a), 1-mu(a)) and (pi(a), 1-pi(a))."""
+    mu_a = float(mu_a)
+    pi_a = float(pi_a)
+    return _xlogx_over_y(mu_a, pi_a) + _xlogx_over_y(1.0 - mu_a, 1.0 - pi_a)
+
+
+def topk_reduced(pi, a, mu_a, topk_ids, topk_p):
+    """Reduced categoricals over A''_t = A'_t u {other} (Sec. 4.4, Top-K Approximation).
+
+    A'_t is the *set* of the stored top-K ids of mu joined with the sampled id a.
+    p_mu(a') is the stored top-K probability for list members (also for a when it
+    is a member) and mu_a for a otherwise; p_pi(a') = pi[a'].  "other" is one
+    minus the sum over A'_t, clamped to [0, 1]; when A'_t already is the whole
+    vocabulary the bucket is empty and both masses are exactly 0.
+    Returns (p_mu, p_pi): two float64 arrays of length |A'_t| + 1, "other" last.
+    """
+    pi = _f64(pi)
+    ids = [int(i) for i in np.asarray(topk_ids).reshape(-1)]
+    ps = [float(p) for p in _f64(topk_p).reshape(-1)]
+    members = {}
+    for i, p in zip(ids, ps):
+        if i not in members:          # a duplicated id is a caller error; first entry wins
+            members[i] = p
+    if int(a) not in members:
+        members[int(a)] = float(mu_a)
+    keys = list(members.keys())
+    p_mu = np.array([members[i] for i in keys], dtype=np.float64)
+    p_pi = np.array([pi[i] for i in keys], dtype=np.float64)
+    if len(keys) == pi.shape[0]:      # A'_t is the whole vocabulary: nothing is left to aggregate
+        other_mu = other_pi = 0.0
+    else:
+        other_mu = min(1.0, max(0.0, 1.0 - float(np.sum(p_mu))))
+        other_pi = min(1.0, max(0.0, 1.0 - float(np.sum(p_pi))))
+    return np.append(p_mu, other_mu), np.append(p_pi, other_pi)
+
+
+def topk_tv(p_mu, p_pi):
+    """Eq. topk_tv: one half of the L1 distance of the reduced distributions."""
+    return 0.5 * float(np.sum(np.abs(_f64(p_mu) - _f64(p_pi))))
+
+
+def topk_kl(p_mu, p_pi):
+    """Eq. topk_kl: sum_a p_mu(a) log(p_mu(a)/p_pi(a)) over the reduced vocabulary."""
+    return float(sum(_xlogx_over_y(x, y) for x, y in zip(_f64(p_mu), _f64(p_pi))))
+
+
+def full_tv(mu, pi):
+    """Exact TV over the whole vocabulary: 1/2 sum_a |mu(a) - pi(a)|  (App. B)."""
+    return 0.5 * float(np.sum(np.abs(_f64(mu) - _f64(pi))))
+
+
+def full_kl(mu, pi):
+    """Exact KL(mu || pi) over the whole vocabulary  (App. B)."""
+    return float(sum(_xlogx_over_y(x, y) for x, y in zip(_f64(mu), _f64(pi))))
+
+
+def dppo_mask(adv, log_pi_a, mu_logp, D, delta):
+    """Eq. dppo_obj: M = 0 iff (A>0 and r>1 and D>delta) or (A<0 and r<1 and D>delta); else 1.
+
+    r >< 1 is decided in the log domain (log pi(a) >< log mu(a)); all comparisons strict.
+    """
+    adv = float(adv)
+    up = float(log_pi_a) > float(mu_logp)
+    down = float(log_pi_a) < float(mu_logp)
+    away = (adv > 0.0 and up) or (adv < 0.0 and down)
+    return 0 if (away and float(D) > float(delta)) else 1
+
+
+def divergence(variant, pi, a, mu_logp, topk_ids=None, topk_p=None):
+    """D_t of one row for the chosen approximation, given pi[V] (float64 probabilities)."""
+    mu_a = float(np.exp(float(mu_logp)))
+    pi_a = float(pi[int(a)])
+    if variant == BINARY_TV:
+        return binary_tv(mu_a, pi_a)
+    if variant == BINARY_KL:
+        return binary_kl(mu_a, pi_a)
+    if variant in (TOPK_TV, TOPK_KL):
+        if topk_ids is None:
+            topk_ids, topk_p = [], []
+        p_mu, p_pi = topk_reduced(pi, a, mu_a, topk_ids, topk_p)
+        return topk_tv(p_mu, p_pi) if variant == TOPK_TV else topk_kl(p_mu, p_pi)
+    raise ValueError(f"unknown variant {variant}")
+
+
+def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=None, want_grad=True):
+    """All per-token quantities of one valid row.
+
+    Returns a dict: lse, log_pi_a, r, D, M, loss (= -s*M*r*A), g (= s*M*r*A) and,
+    if want_grad, dlogits[V] = g * (pi - onehot(a)): the derivative of the loss
+    term with M held constant (Eq. unified_grad with C = inf; d log pi(a)/dz_j =
+    1[j=a] - pi_j).
+    """
+    log_pi, lse = log_softmax_row(z)
+    pi = np.exp(log_pi)
+    a = int(a)
+    log_pi_a = float(log_pi[a])
+    r = ratio(log_pi_a, mu_logp)
+    D = divergence(variant, pi, a, mu_logp, topk_ids, topk_p)
+    M = dppo_mask(adv, log_pi_a, mu_logp, D, delta)
+    g = float(scale) * M * r * float(adv)
+    out = dict(lse=float(lse), log_pi_a=log_pi_a, r=r, D=D, M=M, loss=-g, g=g)
+    if want_grad:
+        d = g * pi
+        d[a] -= g
+        out["dlogits"] = d
+    return out
+
+
+def default_scale(T, token_mask):
+    """Token-mean normaliser s = 1 / N_valid (0 if no row is valid)."""
+    n = int(T) if token_mask is None else int(np.count_nonzero(np.asarray(token_mask)))
+    return (1.0 / n) if n > 0 else 0.0
+
+
+def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV,
+                      K=0, delta=0.2, loss_scale=None, mu_topk_ids=None, mu_topk_p=None, want_grad=True):
+    """The whole path over T rows (Eq. dppo_obj summed over tokens, as a loss to minimise).
+
+    logits [T,V]; sampled_ids, mu_logp, advantages [T]; token_mask [T] or None;
+    mu_topk_ids / mu_topk_p [T,K] for the Top-K variants.  loss_scale None means
+    1/N_valid.  Rows with token_mask == 0 contribute nothing: D = 0, M = 0, zero
+    gradient row.  Returns dict(loss, D[T], M[T], r[T], row_loss[T], dlogits[T,V] or None).
+    """
+    logits = np.asarray(logits)
+    T, V = logits.shape
+    s = default_scale(T, token_mask) if loss_scale is None else float(loss_scale)
+    D = np.zeros(T)
+    M = np.zeros(T, dtype=np.uint8)
+    r = np.zeros(T)
+    row_loss = np.zeros(T)
+    dl = np.zeros((T, V)) if want_grad else None
+    for t in range(T):
+        if token_mask is not None and not token_mask[t]:
+            continue
+        ids = ps = None
+        if variant in (TOPK_TV, TOPK_KL) and K > 0:
+            ids, ps = mu_topk_ids[t][:K], mu_topk_p[t][:K]
+        o = dppo_row(logits[t], sampled_ids[t], mu_logp[t], advantages[t], variant, delta, s, ids, ps, want_grad)
+        D[t], M[t], r[t], row_loss[t] = o["D"], o["M"], o["r"], o["loss"]
+        if want_grad:
+            dl[t] = o["dlogits"]
+    return dict(loss=float(np.sum(row_loss)), D=D, M=M, r=r, row_loss=row_loss, dlogits=dl, scale=s)
+
+
+def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None,
+                              variant=BINARY_TV, delta=0.2, loss_scale=None):
+    """LM-head variant: logits = hidden @ W in float64 (never rounded), then the path above,
+    then the chain rule: dHidden = dlogits @ W^T, dW = hidden^T @ dlogits.
+    """
+    H = _f64(hidden)
+    Wm = _f64(W)
+    z = H @ Wm
+    o = dppo_loss_fwd_bwd(z, sampled_ids, mu_logp, advantages, token_mask, variant, 0, delta, loss_scale)
+    o["dHidden"] = o["dlogits"] @ Wm.T
+    o["dW"] = H.T @ o["dlogits"]
+    return o
