@@ -1,0 +1,296 @@
+"""Benchmark of the DPPO per-token loss path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one forward+backward pass of the whole path (prelude, row kernel, loss reduction) over one
+batch of the Qwen3-vocabulary Binary-TV workload: T = 16384 token rows (16 responses x 1024), V = 151936,
+bf16 logits and bf16 gradient, delta = 0.2, synthetic seeded inputs.  With N > 1 (launched by torchrun,
+one process per GPU) every rank owns T rows of a global batch of N*T rows, with the global token-mean
+scale passed in, so no collective is on the data path (weak scaling).  Rank 0 prints one JSON line.
+
+`--impl reference` times the float64 CPU oracle instead (rank 0 only), a bounded sample of the same
+workload per step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+T_ROWS = 16384
+VOCAB = 151936
+DELTA = 0.2
+METRIC = "tokens/sec fwd+bwd DPPO loss at V=151936 bf16"
+BYTES_PER_TOKEN = 4 * VOCAB          # bf16 logits read (2V) + bf16 dlogits written (2V)
+WORKLOAD = "qwen3_vocab_binary_tv: T=16384 (16 responses x 1024), V=151936, bf16 logits, Binary-TV, delta=0.2"
+ORACLE_ROWS_PER_STEP = 192           # CPU oracle sample per step (about a second of numpy work)
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--variant", default="binary_tv", choices=["binary_tv", "binary_kl"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+# ----------------------------------------------------------------------------------------- peaks / clocks
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU from a thread (NVML) while the GPU works."""
+
+    def __init__(self, index):
+        self.samples = []
+        self.stop_flag = False
+        self.thread = None
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:  # noqa: BLE001
+            self.max_mhz = None
+
+    def _run(self):
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                    else int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                self.samples.append((time.perf_counter(), mhz, reasons))
+            except Exception:  # noqa: BLE001
+                pass
+            time.sleep(0.01)
+
+    def start(self):
+        if self.ok:
+            self.thread = threading.Thread(target=self._run, daemon=True)
+            self.thread.start()
+
+    def stop(self):
+        self.stop_flag = True
+        if self.thread:
+            self.thread.join(timeout=2)
+
+    def summary(self, t0, t1):
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+                 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting"}
+        sel = [s for s in self.samples if t0 <= s[0] <= t1] or self.samples
+        if not sel:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        mhz = sorted(s[1] for s in sel)
+        bits = 0
+        for s in sel:
+            bits |= s[2]
+        reasons = sorted(n for b, n in names.items() if bits & b)
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(sel)}
+
+
+# ----------------------------------------------------------------------------------------- oracle arm
+
+def oracle_tokens_per_s(rows, seed, variant_code):
+    """Times the float64 oracle, as it stands, on `rows` rows of the workload generated on the CPU."""
+    import numpy as np
+    import torch
+    from paper_2602_04879_b200 import workloads as wl
+    from oracle import dppo_oracle as O
+    b = wl.qwen_vocab_rows("cpu", seed=seed, rows=rows)
+    z = b.logits.float().numpy().astype(np.float64)
+    ids = b.sampled_ids.numpy()
+    mu = b.mu_logp.numpy().astype(np.float64)
+    adv = b.advantages.numpy().astype(np.float64)
+    t0 = time.perf_counter()
+    O.dppo_loss_fwd_bwd(z, ids, mu, adv, None, variant_code, 0, DELTA, 1.0 / T_ROWS)
+    dt = time.perf_counter() - t0
+    return rows / dt, dt, torch.get_num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import dppo_oracle as O
+    code = O.BINARY_TV if args.variant == "binary_tv" else O.BINARY_KL
+    steps = max(1, min(args.steps, 8))
+    warm = max(0, min(args.warmup, 1))
+    for _ in range(warm):
+        oracle_tokens_per_s(ORACLE_ROWS_PER_STEP, 1, code)
+    tot_rows, tot_t = 0, 0.0
+    for _ in range(steps):
+        tps, dt, _ = oracle_tokens_per_s(ORACLE_ROWS_PER_STEP, 1, code)
+        tot_rows += ORACLE_ROWS_PER_STEP
+        tot_t += dt
+    value = tot_rows / tot_t
+    sample = f"{ORACLE_ROWS_PER_STEP} rows of the workload per step (first rows of the seeded batch), {steps} steps timed"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": 1e3 * tot_t / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "variant": args.variant, "note": "float64 numpy oracle on host cores"},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ----------------------------------------------------------------------------------------- our arm
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2602_04879_b200 as dppo
+    from paper_2602_04879_b200 import workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (the library has no CPU path)")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    variant = dppo.BINARY_TV if args.variant == "binary_tv" else dppo.BINARY_KL
+
+    # each rank owns T rows of the global batch of world*T rows
+    b = wl.qwen_vocab_rows(dev, seed=1 + rank)
+    T = b.T
+    scale = 1.0 / (T * world)
+    dlogits = torch.empty_like(b.logits)
+    ws = torch.empty(dppo.dppo_workspace_bytes(T), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step():
+        return dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, variant, 0, DELTA,
+                                      loss_scale=scale, dlogits=dlogits, workspace=ws, status=status)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    for _ in range(max(3, args.warmup)):
+        out = step()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    t_host0 = time.perf_counter()
+    ev0.record()
+    for _ in range(args.steps):
+        out = step()
+    ev1.record()
+    barrier()
+    t_host1 = time.perf_counter()
+    sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        loss_t = out["loss"].clone()
+        dist.all_reduce(loss_t)                     # global loss = sum of the shards' losses
+        loss_val = float(loss_t.item())
+    else:
+        loss_val = float(out["loss"].item())
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    ms_per_step = ms / args.steps
+    tokens_per_s = world * T * args.steps / (ms * 1e-3)
+
+    # roofline of the row kernel: algorithmic bytes of one launch over the step's device time (the step is
+    # the row kernel plus two single-CTA kernels of a few microseconds, so this slightly under-reports it)
+    peak, peak_src = measured_peaks()
+    achieved = T * BYTES_PER_TOKEN / (ms_per_step * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_source": "of " + peak_src, "kernel": "dppo_row_ring_kernel<bf16,bf16>",
+                "algorithmic_bytes_per_launch": T * BYTES_PER_TOKEN}
+    tr = os.path.join(ROOT, "profiles", "ring_traffic.json")
+    if os.path.exists(tr):
+        with open(tr) as f:
+            roofline["traffic"] = json.load(f).get("dram_bytes_per_launch_full_size")
+    clocks = sampler.summary(t_host0, t_host1)
+
+    line = {
+        "metric": METRIC, "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "variant": args.variant, "rows_per_gpu": T, "l2": "inputs_larger_than_L2 (4.98 GB read + 4.98 GB written per step)",
+                   "parallelism": f"dp{world} row shards, no data-path collective", "logits_dtype": "bf16", "dlogits_dtype": "bf16"},
+        "roofline": roofline, "clocks": clocks, "gpu_launches": 3 * args.steps, "loss": loss_val,
+    }
+
+    # end to end through the host-buffer entry point: pinned host inputs -> device -> loss / D / M back on the host
+    if not args.no_e2e:
+        rows_per_chunk = 1024
+        pin = lambda x: x.cpu().pin_memory()
+        h = dict(logits=pin(b.logits), ids=pin(b.sampled_ids), mu=pin(b.mu_logp), adv=pin(b.advantages))
+        outbuf = dict(divergence=torch.empty(T, dtype=torch.float32).pin_memory(), mask=torch.empty(T, dtype=torch.uint8).pin_memory())
+        staging = torch.empty(dppo.dppo_host_staging_bytes(rows_per_chunk, VOCAB, 0, dppo.BF16), dtype=torch.uint8, device=dev)
+
+        def e2e_step():
+            return dppo.dppo_loss_fwd_bwd_host(h["logits"], h["ids"], h["mu"], h["adv"], None, variant, 0, DELTA,
+                                               loss_scale=scale, rows_per_chunk=rows_per_chunk, staging=staging, out=outbuf)
+        e2e_steps = max(1, min(args.steps, 5))
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            r = e2e_step()                         # synchronises: results are on the host when it returns
+        barrier()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        assert r["status"] == 0
+        line["e2e"] = {"value": world * T * e2e_steps / dt, "unit": "tokens/s",
+                       "h2d_bytes_per_step": T * VOCAB * 2 + T * 12, "d2h_bytes_per_step": T * 5 + 8,
+                       "steps": e2e_steps, "note": "dppo_loss_fwd_bwd_host: pinned host logits/ids/mu_logp/advantages in, loss + divergence + mask out; dlogits stay on the device"}
+        del h, staging
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import dppo_oracle as O
+        code = O.BINARY_TV if args.variant == "binary_tv" else O.BINARY_KL
+        rows = 1536
+        tps, dt, _ = oracle_tokens_per_s(rows, 1, code)
+        line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                                "sample": f"first {rows} rows of the workload regenerated on the CPU, {dt:.1f} s of float64 numpy"}
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,170 @@
+/*
+ * dppo.h - C ABI of the DPPO per-token loss path for NVIDIA B200 (sm_100a).
+ *
+ * DPPO (Divergence Proximal Policy Optimization, "Rethinking the Trust Region
+ * in LLM Reinforcement Learning") replaces PPO's ratio clipping by a mask that
+ * depends on an estimate D_t of the divergence between the rollout policy mu
+ * and the trainer policy pi at every response token.  For each token row this
+ * library streams the trainer's vocabulary logits once and produces
+ *
+ *   lse_t      = log sum_j exp(z_tj)                      (Sec. 3: pi is a categorical over the vocabulary)
+ *   r_t        = pi(a_t) / mu(a_t)                        (Eq. ppo-clip)
+ *   D_t        = Binary-TV / Binary-KL / TopK-TV / TopK-KL (Eq. binary_tv, binary_kl, topk_tv, topk_kl)
+ *   M_t        = 0 iff D_t > delta and the update moves r_t away from 1
+ *                in the direction the advantage pushes     (Eq. dppo_obj)
+ *   loss       = -s * sum_t M_t r_t A_t                   (Eq. dppo_obj, as a loss to minimise)
+ *   dlogits_tj = s M_t r_t A_t (pi_tj - 1[j = a_t])       (Eq. unified_grad with C = infinity)
+ *
+ * without ever materialising a probability tensor.
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ *  - Unless a parameter says "host", every pointer is a DEVICE pointer owned by
+ *    the caller.  The library allocates nothing, keeps no state between calls,
+ *    enqueues its kernels on `cuda_stream` (a cudaStream_t passed as void*,
+ *    NULL = the default stream) and never synchronises.
+ *  - Return value: DPPO_OK (0) when the kernels were enqueued; a negative
+ *    DPPO_ERR_* code for misuse the host can see, in which case nothing was
+ *    launched.  dppo_error_string() names a code.
+ *  - Anomalies only the device can see never trap: they OR bits into *status
+ *    (DPPO_STATUS_*), and the offending row is treated as invalid (D = 0, M = 0,
+ *    zero gradient row, no loss term).  The caller zeroes *status beforehand.
+ *  - Results are deterministic: the same inputs give bit-identical outputs.
+ *  - Rows whose token_mask byte is 0 are never read; their outputs are zero.
+ *  - The scale s is opts->loss_scale when that is > 0, otherwise 1 / N_valid
+ *    with N_valid the number of rows of THIS call whose token_mask is non-zero
+ *    (0 if there is none, so an empty or fully masked call returns loss = 0).
+ */
+#ifndef DPPO_H_
+#define DPPO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Divergence approximations (Sec. 4.4: Binary and Top-K approximation). */
+enum { DPPO_BINARY_TV = 0, DPPO_BINARY_KL = 1, DPPO_TOPK_TV = 2, DPPO_TOPK_KL = 3 };
+/* Element types of the logits / dlogits tensors. */
+enum { DPPO_F32 = 0, DPPO_BF16 = 1 };
+/* opts->dlogits_dtype */
+enum { DPPO_DLOGITS_SAME = 0, DPPO_DLOGITS_F32 = 1 };
+/* opts->kernel */
+enum { DPPO_KERNEL_AUTO = 0, DPPO_KERNEL_GENERIC = 1, DPPO_KERNEL_RING = 2 };
+
+/* Host-visible error codes. */
+enum {
+  DPPO_OK = 0,
+  DPPO_ERR_NULL = -1,        /* a required pointer is NULL                                  */
+  DPPO_ERR_SHAPE = -2,       /* T < 0, V < 1, K < 0, K > V, d < 1                            */
+  DPPO_ERR_DTYPE = -3,       /* unknown logits / dlogits dtype                               */
+  DPPO_ERR_VARIANT = -4,     /* unknown variant                                              */
+  DPPO_ERR_TOPK = -5,        /* Top-K variant with K > 0 but a NULL id / probability list    */
+  DPPO_ERR_STRIDE = -6,      /* a row stride smaller than V                                  */
+  DPPO_ERR_ALIGN = -7,       /* pointer / stride alignment the requested kernel cannot take  */
+  DPPO_ERR_WORKSPACE = -8,   /* workspace NULL, misaligned or smaller than dppo_workspace_bytes */
+  DPPO_ERR_ALIAS = -9,       /* dlogits aliases logits but the element sizes differ          */
+  DPPO_ERR_CUDA = -10,       /* a CUDA runtime call failed (launch, copy)                    */
+  DPPO_ERR_UNSUPPORTED = -11 /* combination not implemented                                  */
+};
+
+/* Bits OR-ed into *status by the device. */
+enum {
+  DPPO_STATUS_BAD_SAMPLED_ID = 1, /* sampled_ids[t] outside [0, V)          */
+  DPPO_STATUS_BAD_TOPK_ID = 2,    /* a mu_topk_ids entry outside [0, V)     */
+  DPPO_STATUS_NONFINITE_ROW = 4,  /* lse of a row is NaN or infinite         */
+  DPPO_STATUS_WAIT_LIMIT = 8      /* a bounded on-chip wait gave up          */
+};
+
+/* Options; all-zero means defaults. */
+typedef struct dppo_opts {
+  float loss_scale;    /* s > 0: use it (e.g. a global 1/N for micro-batched or sharded calls);
+                          <= 0: s = 1 / N_valid of this call (token mean)                       */
+  int dlogits_dtype;   /* DPPO_DLOGITS_SAME: dlogits has the logits dtype; DPPO_DLOGITS_F32      */
+  int kernel;          /* DPPO_KERNEL_AUTO picks the shared-memory ring kernel when the layout
+                          allows 16-byte bulk copies and the scalar kernel otherwise            */
+  int reserved;
+} dppo_opts;
+
+/* Bytes of device scratch dppo_loss_fwd_bwd needs for T rows (256-byte aligned
+ * pointer expected).  Contents need no initialisation and carry nothing between calls. */
+size_t dppo_workspace_bytes(int64_t T);
+
+/*
+ * Forward + backward of the DPPO loss over T token rows (Eq. dppo_obj; gradient:
+ * Eq. unified_grad with C = infinity, the mask not differentiated).
+ *
+ *  logits          [T, V] row-major with row stride `logits_row_stride` elements (>= V),
+ *                  dtype `logits_dtype` (DPPO_F32 or DPPO_BF16).
+ *  sampled_ids     [T] token a_t sampled by the rollout policy.
+ *  mu_logp         [T] log mu(a_t | s_t) stored by the rollout engine; always required (r_t needs it).
+ *  mu_topk_ids     [T, K] ids of the rollout policy's K most probable tokens (any order, no
+ *                  duplicates), and
+ *  mu_topk_p       [T, K] their probabilities under mu; both may be NULL when K == 0 or for the
+ *                  Binary variants.  The reduced distribution is over set(mu_topk_ids) u {a_t}
+ *                  plus one "other" bucket (Sec. 4.4); a_t uses the list's probability when it is
+ *                  a member and exp(mu_logp) otherwise.
+ *  advantages      [T] per-token advantage A_t.
+ *  token_mask      [T] bytes, non-zero = valid row; NULL = all rows valid.
+ *  variant, K, delta   divergence approximation, list width, threshold (mask test is D_t > delta).
+ *  opts            NULL = defaults.
+ *  loss            [1]  out: -s * sum_t M_t r_t A_t.
+ *  divergence      [T]  out: D_t (0 for invalid rows; +inf possible for KL when pi puts zero mass
+ *                  where mu does not).
+ *  mask            [T]  out: M_t as bytes (0 for invalid rows).
+ *  dlogits         [T, V] out, row stride `dlogits_row_stride` (>= V), dtype per opts; may be the
+ *                  same buffer as logits (in place) when the element sizes match and the strides
+ *                  are equal.
+ *  stats           [8] out or NULL: N_valid, N_blocked (valid rows with M = 0), sum D, max D,
+ *                  sum |pi(a)-mu(a)|, sum r, sum |loss term|, reserved.  Sums skip non-finite D.
+ *  status          [1] in/out device word, see DPPO_STATUS_*.
+ *  workspace       device scratch of at least dppo_workspace_bytes(T) bytes.
+ */
+int dppo_loss_fwd_bwd(const void* logits, int64_t T, int64_t V, int64_t logits_row_stride, int logits_dtype,
+                      const int32_t* sampled_ids, const float* mu_logp,
+                      const int32_t* mu_topk_ids, const float* mu_topk_p,
+                      const float* advantages, const uint8_t* token_mask,
+                      int variant, int K, float delta, const dppo_opts* opts,
+                      float* loss, float* divergence, uint8_t* mask,
+                      void* dlogits, int64_t dlogits_row_stride,
+                      float* stats, int32_t* status,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Bytes of device staging dppo_loss_fwd_bwd_host needs (inputs, outputs and workspace for
+ * `rows_per_chunk` rows at a time, two chunks in flight). */
+size_t dppo_host_staging_bytes(int64_t rows_per_chunk, int64_t V, int K, int logits_dtype, int dlogits_dtype);
+
+/*
+ * The same operation on HOST buffers (pinned memory recommended): rows are copied to the device
+ * in chunks of `rows_per_chunk`, processed, and the per-token outputs copied back, with the
+ * copies of one chunk overlapping the kernels of the other on two internal streams.  Pointer
+ * arguments with the same names as above have the same meaning but are HOST pointers
+ * (contiguous rows: stride V).  `dlogits_host` may be NULL, in which case the gradient rows are
+ * left in the staging area of the last chunks and not copied back.  `staging` is DEVICE memory
+ * of at least dppo_host_staging_bytes(...) bytes, 256-byte aligned, owned by the caller.
+ * `status_host` receives the OR of the device status words.  Because the token-mean scale needs
+ * N_valid of the whole batch before the first chunk, it is counted on the host from token_mask.
+ * The call synchronises with the device before returning (the results are on the host).
+ * Creates and destroys two CUDA streams and events per call; allocates no device memory.
+ */
+int dppo_loss_fwd_bwd_host(const void* logits, int64_t T, int64_t V, int logits_dtype,
+                           const int32_t* sampled_ids, const float* mu_logp,
+                           const int32_t* mu_topk_ids, const float* mu_topk_p,
+                           const float* advantages, const uint8_t* token_mask,
+                           int variant, int K, float delta, const dppo_opts* opts,
+                           float* loss_host, float* divergence_host, uint8_t* mask_host,
+                           void* dlogits_host, int32_t* status_host,
+                           void* staging, size_t staging_bytes, int64_t rows_per_chunk);
+
+/* Name of an error code (static string, never NULL). */
+const char* dppo_error_string(int code);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int dppo_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DPPO_H_ */

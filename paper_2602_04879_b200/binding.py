@@ -1,0 +1,170 @@
+"""ctypes binding of libdppo.so: argument marshalling only.
+
+Every function mirrors the C entry point of the same name in include/dppo.h and takes torch
+tensors for the pointer arguments (CUDA tensors for the device entry points, CPU tensors for the
+``_host`` one).  Nothing is computed here; if the library is missing or cannot be loaded the
+import of a symbol raises, there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_void_p
+
+import torch
+
+BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL = 0, 1, 2, 3
+F32, BF16 = 0, 1
+DLOGITS_SAME, DLOGITS_F32 = 0, 1
+KERNEL_AUTO, KERNEL_GENERIC, KERNEL_RING = 0, 1, 2
+STATUS_BAD_SAMPLED_ID, STATUS_BAD_TOPK_ID, STATUS_NONFINITE_ROW, STATUS_WAIT_LIMIT = 1, 2, 4, 8
+VARIANTS = {"binary_tv": BINARY_TV, "binary_kl": BINARY_KL, "topk_tv": TOPK_TV, "topk_kl": TOPK_KL}
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdppo.so")
+_lib = None
+
+
+class DppoOpts(ctypes.Structure):
+    _fields_ = [("loss_scale", c_float), ("dlogits_dtype", c_int), ("kernel", c_int), ("reserved", c_int)]
+
+
+class DppoError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {error_string(code)} ({code})")
+
+
+def lib():
+    """The loaded library (loads it on first use; raises if it is not built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2602_04879_b200.build` (there is no fallback path)")
+        L = ctypes.CDLL(_LIB_PATH)
+        L.dppo_version.restype = c_int
+        L.dppo_error_string.restype = c_char_p
+        L.dppo_error_string.argtypes = [c_int]
+        L.dppo_workspace_bytes.restype = c_size_t
+        L.dppo_workspace_bytes.argtypes = [c_int64]
+        L.dppo_loss_fwd_bwd.restype = c_int
+        L.dppo_loss_fwd_bwd.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p, c_void_p, c_void_p,
+                                        c_void_p, c_void_p, c_int, c_int, c_float, POINTER(DppoOpts),
+                                        c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p,
+                                        c_void_p, c_size_t, c_void_p]
+        L.dppo_host_staging_bytes.restype = c_size_t
+        L.dppo_host_staging_bytes.argtypes = [c_int64, c_int64, c_int, c_int, c_int]
+        L.dppo_loss_fwd_bwd_host.restype = c_int
+        L.dppo_loss_fwd_bwd_host.argtypes = [c_void_p, c_int64, c_int64, c_int, c_void_p, c_void_p, c_void_p, c_void_p,
+                                             c_void_p, c_void_p, c_int, c_int, c_float, POINTER(DppoOpts),
+                                             c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                             c_void_p, c_size_t, c_int64]
+        _lib = L
+    return _lib
+
+
+def version():
+    return int(lib().dppo_version())
+
+
+def error_string(code):
+    return lib().dppo_error_string(int(code)).decode()
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _dtype_code(t):
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"logits dtype {t.dtype} not supported (float32 or bfloat16)")
+
+
+def dppo_workspace_bytes(T):
+    return int(lib().dppo_workspace_bytes(int(T)))
+
+
+def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, K=0, delta=0.2,
+                      mu_topk_ids=None, mu_topk_p=None, loss_scale=0.0, dlogits_f32=False, kernel=KERNEL_AUTO,
+                      dlogits=None, want_stats=False, workspace=None, status=None, stream=None):
+    """Calls ``dppo_loss_fwd_bwd`` on CUDA tensors.  Output tensors are allocated with torch unless
+    given.  Returns dict(loss[1], divergence[T], mask[T], dlogits[T,V], stats[8] or None, status[1]);
+    nothing is synchronised."""
+    assert logits.is_cuda and logits.dim() == 2 and logits.stride(1) == 1
+    T, V = logits.shape
+    dev = logits.device
+    out_dtype = torch.float32 if dlogits_f32 else logits.dtype
+    if dlogits is None:
+        dlogits = torch.empty((T, V), dtype=out_dtype, device=dev)
+    assert dlogits.dtype == out_dtype and dlogits.stride(1) == 1
+    loss = torch.empty(1, dtype=torch.float32, device=dev)
+    D = torch.empty(T, dtype=torch.float32, device=dev)
+    M = torch.empty(T, dtype=torch.uint8, device=dev)
+    stats = torch.empty(8, dtype=torch.float32, device=dev) if want_stats else None
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    nbytes = dppo_workspace_bytes(T)
+    if workspace is None:
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    for name, t, dt in (("sampled_ids", sampled_ids, torch.int32), ("mu_logp", mu_logp, torch.float32),
+                        ("advantages", advantages, torch.float32), ("token_mask", token_mask, torch.uint8),
+                        ("mu_topk_ids", mu_topk_ids, torch.int32), ("mu_topk_p", mu_topk_p, torch.float32)):
+        if t is not None:
+            assert t.is_cuda and t.dtype == dt and t.is_contiguous(), name
+    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), 0)
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    with torch.cuda.device(dev):
+        rc = lib().dppo_loss_fwd_bwd(_ptr(logits), T, V, logits.stride(0) if T > 0 else V, _dtype_code(logits),
+                                     _ptr(sampled_ids), _ptr(mu_logp), _ptr(mu_topk_ids), _ptr(mu_topk_p),
+                                     _ptr(advantages), _ptr(token_mask), int(variant), int(K), float(delta),
+                                     ctypes.byref(opts), _ptr(loss), _ptr(D), _ptr(M), _ptr(dlogits),
+                                     dlogits.stride(0) if T > 0 else V, _ptr(stats), _ptr(status), _ptr(workspace),
+                                     workspace.numel(), c_void_p(st.cuda_stream))
+    if rc != 0:
+        raise DppoError(rc, "dppo_loss_fwd_bwd")
+    return dict(loss=loss, divergence=D, mask=M, dlogits=dlogits, stats=stats, status=status)
+
+
+def dppo_host_staging_bytes(rows_per_chunk, V, K, logits_dtype, dlogits_f32=False):
+    return int(lib().dppo_host_staging_bytes(int(rows_per_chunk), int(V), int(K), int(logits_dtype),
+                                             DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME))
+
+
+def dppo_loss_fwd_bwd_host(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, K=0, delta=0.2,
+                           mu_topk_ids=None, mu_topk_p=None, loss_scale=0.0, dlogits_f32=False, kernel=KERNEL_AUTO,
+                           rows_per_chunk=1024, staging=None, want_dlogits=False, device="cuda:0", out=None):
+    """Calls ``dppo_loss_fwd_bwd_host`` on CPU tensors (pinned recommended); ``staging`` is a CUDA
+    uint8 tensor of at least ``dppo_host_staging_bytes`` bytes (allocated here if None).  Returns
+    dict(loss(float), divergence, mask, dlogits or None, status(int)) with host tensors."""
+    assert not logits.is_cuda and logits.dim() == 2 and logits.is_contiguous()
+    T, V = logits.shape
+    dt = _dtype_code(logits)
+    need = dppo_host_staging_bytes(rows_per_chunk, V, K if variant in (TOPK_TV, TOPK_KL) else 0, dt, dlogits_f32)
+    if staging is None:
+        staging = torch.empty(need, dtype=torch.uint8, device=device)
+    out = out or {}
+    D = out.get("divergence")
+    if D is None:
+        D = torch.empty(T, dtype=torch.float32).pin_memory()
+    M = out.get("mask")
+    if M is None:
+        M = torch.empty(T, dtype=torch.uint8).pin_memory()
+    dl = None
+    if want_dlogits:
+        dl = out.get("dlogits")
+        if dl is None:
+            dl = torch.empty((T, V), dtype=torch.float32 if dlogits_f32 else logits.dtype).pin_memory()
+    loss = c_float(0.0)
+    status = c_int32(0)
+    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), 0)
+    with torch.cuda.device(staging.device):
+        rc = lib().dppo_loss_fwd_bwd_host(_ptr(logits), T, V, dt, _ptr(sampled_ids), _ptr(mu_logp), _ptr(mu_topk_ids),
+                                          _ptr(mu_topk_p), _ptr(advantages), _ptr(token_mask), int(variant), int(K),
+                                          float(delta), ctypes.byref(opts), ctypes.byref(loss), _ptr(D), _ptr(M),
+                                          _ptr(dl), ctypes.byref(status), _ptr(staging), staging.numel(),
+                                          int(rows_per_chunk))
+    if rc != 0:
+        raise DppoError(rc, "dppo_loss_fwd_bwd_host")
+    return dict(loss=float(loss.value), divergence=D, mask=M, dlogits=dl, status=int(status.value))

@@ -1,0 +1,183 @@
+// Shared device-side pieces of the DPPO loss kernels: parameter block, numeric helpers and the
+// per-row scalar stage (ratio, divergence, mask, gradient coefficient).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "../../include/dppo.h"
+
+namespace dppo {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr double kLn2 = 0.6931471805599453;
+
+// Header of the caller's workspace, written by the prelude kernel of each call.
+struct WsHeader {
+  double scale;        // s of this call
+  int n_valid;         // rows with a non-zero token_mask byte
+  int pad[13];
+};
+static_assert(sizeof(WsHeader) == 64, "WsHeader layout");
+
+struct RowParams {
+  const void* logits;
+  int64_t T, V, ld_in;
+  const int32_t* sampled_ids;
+  const float* mu_logp;
+  const int32_t* topk_ids;
+  const float* topk_p;
+  const float* adv;
+  const uint8_t* token_mask;
+  int variant, K;
+  float delta;
+  float loss_scale;          // > 0: caller's s
+  void* dlogits;
+  int64_t ld_out;
+  float* divergence;
+  uint8_t* mask;
+  float* loss;
+  float* stats;
+  int32_t* status;
+  WsHeader* hdr;             // workspace
+  float* row_loss;           // [T] -s M r A
+  float* row_r;              // [T] r_t
+  float* row_absdiff;        // [T] |pi(a) - mu(a)|
+};
+
+// What the scalar stage hands to the gradient sweep of one row.
+struct RowCoef {
+  float c2;       // exponent offset: dlogits_j = sgn * 2^(z_j*log2e + c2) for j != a
+  float sgn;      // +1 / -1 (sign of g); 0 when the whole row is zero
+  float fix;      // value of dlogits at j = a
+  int zero_row;   // 1: write zeros (invalid row, blocked row, zero advantage)
+};
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// Merge two online-softmax partials (m, s): s counts exp(z - m).  -inf maxima carry s = 0.
+__device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2) {
+  float mn = fmaxf(m, m2);
+  float ref = (mn == -INFINITY) ? 0.f : mn;
+  s = s * ex2_approx((m - ref) * kLog2e) + s2 * ex2_approx((m2 - ref) * kLog2e);
+  m = mn;
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ double xlogx_over_y(double x, double y) {
+  if (x <= 0.0) return 0.0;
+  if (y <= 0.0) return INFINITY;
+  return x * (log(x) - log(y));
+}
+
+// Per-row scalar stage, run by ONE full warp (all 32 lanes call it with the same arguments).
+//   lse        log-sum-exp of the row (double, from fp32 partial sums)
+//   z_at(id)   fp32 value of this row's logit `id` (global read)
+// Returns on every lane the same values.  `flags` receives DPPO_STATUS_* bits found here.
+template <typename ZAt>
+__device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, int a, double lse, double scale,
+                                                 ZAt z_at, float& D_out, int& M_out, double& g_out,
+                                                 float& r_out, float& absdiff_out, double& pi_a_out, int& flags) {
+  const int lane = threadIdx.x & 31;
+  const double mu_logp = (double)p.mu_logp[t];
+  const double adv = (double)p.adv[t];
+  const double lpa = (double)z_at(a) - lse;           // log pi(a_t)
+  const double pi_a = exp(lpa);
+  const double mu_a = exp(mu_logp);
+  const double r = exp(lpa - mu_logp);                // Eq. ppo-clip
+  double D;
+  if (p.variant == DPPO_BINARY_TV) {
+    D = fabs(mu_a - pi_a);                            // Eq. binary_tv
+  } else if (p.variant == DPPO_BINARY_KL) {           // Eq. binary_kl
+    double first = (mu_a > 0.0) ? mu_a * (mu_logp - lpa) : 0.0;
+    D = first + xlogx_over_y(-expm1(mu_logp), -expm1(lpa));
+  } else {
+    // Reduced categorical over set(top-K ids) u {a} u {other}  (Sec. 4.4, Eq. topk_tv / topk_kl)
+    double sum_mu = 0.0, sum_pi = 0.0, tv = 0.0, kl = 0.0;
+    int in_list = 0, bad = 0;
+    const int32_t* ids = p.topk_ids + t * (int64_t)p.K;
+    const float* ps = p.topk_p + t * (int64_t)p.K;
+    for (int k = lane; k < p.K; k += 32) {
+      int id = ids[k];
+      if (id < 0 || (int64_t)id >= p.V) { bad = 1; continue; }
+      double pm = (double)ps[k];
+      double lpk = (double)z_at(id) - lse;
+      double pk = exp(lpk);
+      sum_mu += pm;
+      sum_pi += pk;
+      tv += fabs(pm - pk);
+      if (pm > 0.0) kl += pm * (log(pm) - lpk);
+      in_list |= (id == a);
+    }
+    sum_mu = warp_sum(sum_mu);
+    sum_pi = warp_sum(sum_pi);
+    tv = warp_sum(tv);
+    kl = warp_sum(kl);
+    in_list = __any_sync(0xffffffffu, in_list);
+    bad = __any_sync(0xffffffffu, bad);
+    if (bad) flags |= DPPO_STATUS_BAD_TOPK_ID;
+    if (!in_list) {
+      sum_mu += mu_a;
+      sum_pi += pi_a;
+      tv += fabs(mu_a - pi_a);
+      if (mu_a > 0.0) kl += mu_a * (mu_logp - lpa);
+    }
+    double om = 0.0, op = 0.0;                         // "other" bucket; empty when the set is the vocabulary
+    if ((int64_t)p.K + (in_list ? 0 : 1) < p.V) {
+      om = fmin(1.0, fmax(0.0, 1.0 - sum_mu));
+      op = fmin(1.0, fmax(0.0, 1.0 - sum_pi));
+    }
+    D = (p.variant == DPPO_TOPK_TV) ? 0.5 * (tv + fabs(om - op)) : kl + xlogx_over_y(om, op);
+  }
+  // Eq. dppo_obj: blocked iff D > delta and the ratio already left 1 on the side the advantage pushes.
+  const bool away = (adv > 0.0 && lpa > mu_logp) || (adv < 0.0 && lpa < mu_logp);
+  const int M = (away && D > (double)p.delta) ? 0 : 1;
+  D_out = (float)D;
+  M_out = M;
+  g_out = scale * (double)M * r * adv;
+  r_out = (float)r;
+  absdiff_out = (float)fabs(mu_a - pi_a);
+  pi_a_out = pi_a;
+}
+
+// Turns g, lse into the coefficients of the gradient sweep.
+__device__ __forceinline__ RowCoef make_coef(double g, double lse, double pi_a) {
+  RowCoef c;
+  if (g == 0.0) {
+    c.c2 = 0.f; c.sgn = 0.f; c.fix = 0.f; c.zero_row = 1;
+    return c;
+  }
+  c.zero_row = 0;
+  c.sgn = (g > 0.0) ? 1.f : -1.f;
+  c.c2 = (float)((log(fabs(g)) - lse) / kLn2);
+  c.fix = (float)(g * (pi_a - 1.0));
+  return c;
+}
+
+// Launchers implemented in the kernel files.
+cudaError_t launch_prelude(const RowParams& p, cudaStream_t st);
+cudaError_t launch_finalize(const RowParams& p, cudaStream_t st);
+cudaError_t launch_generic(const RowParams& p, int in_dtype, int out_dtype, cudaStream_t st);
+cudaError_t launch_ring(const RowParams& p, int in_dtype, int out_dtype, cudaStream_t st);
+bool ring_layout_ok(const RowParams& p, int in_dtype, int out_dtype);
+
+}  // namespace dppo

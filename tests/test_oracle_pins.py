@@ -293,7 +293,7 @@ def check_gradient(O):
         lp = torch.log_softmax(zt, dim=1)[torch.arange(T), torch.tensor(c["a"])]
         loss = -(s * torch.tensor(o["M"].astype(np.float64)) * torch.exp(lp - torch.tensor(c["mu_logp"])) * torch.tensor(c["adv"])).sum()
         loss.backward()
-        assert abs(float(loss) - o["loss"]) < 1e-13
+        assert abs(float(loss.detach()) - o["loss"]) < 1e-13
         np.testing.assert_allclose(o["dlogits"], zt.grad.numpy(), atol=1e-13)
         # structure: rows sum to zero; masked and invalid rows are exactly zero
         np.testing.assert_allclose(o["dlogits"].sum(1), 0, atol=1e-13)

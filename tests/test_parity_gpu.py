@@ -1,0 +1,272 @@
+"""GPU-vs-oracle parity through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2602_04879_b200 as dppo
+from paper_2602_04879_b200 import workloads as wl
+from oracle import dppo_oracle as O
+
+import parity_util as P
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+KERNELS = {"ring": dppo.KERNEL_RING, "generic": dppo.KERNEL_GENERIC}
+
+
+def _run(batch, variant, K, delta, kernel, dlogits_f32=False, loss_scale=0.0, want_stats=True, dlogits=None):
+    out = dppo.dppo_loss_fwd_bwd(batch.logits, batch.sampled_ids, batch.mu_logp, batch.advantages, batch.token_mask,
+                                 variant, K, delta, batch.mu_topk_ids, batch.mu_topk_p, loss_scale=loss_scale,
+                                 dlogits_f32=dlogits_f32, kernel=kernel, want_stats=want_stats, dlogits=dlogits)
+    torch.cuda.synchronize()
+    return out
+
+
+def _full_check(batch, variant, K, delta, kernel, dlogits_f32=False, loss_scale=0.0, expect_blocked=None):
+    out = _run(batch, variant, K, delta, kernel, dlogits_f32, loss_scale)
+    assert int(out["status"].item()) == 0
+    h = P.host_inputs(batch)
+    ora = P.run_oracle(h, variant, K, delta, None if loss_scale == 0.0 else loss_scale)
+    n_exempt, d_err = P.check_scalars(out["divergence"].cpu().numpy(), out["mask"].cpu().numpy(), ora, h, delta)
+    bf16_in = batch.logits.dtype == torch.bfloat16
+    info = P.check_loss(float(out["loss"].item()), ora["loss"], bf16_in, ora["row_loss"])
+    dinfo = P.check_dlogits(out["dlogits"], ora["dlogits"], out_is_bf16=(bf16_in and not dlogits_f32))
+    valid = np.ones(batch.T, bool) if h["token_mask"] is None else h["token_mask"] != 0
+    blocked = int(((ora["M"] == 0) & valid).sum())
+    if expect_blocked is not None:
+        assert expect_blocked(blocked, int(valid.sum())), f"blocked {blocked} of {int(valid.sum())}"
+    st = out["stats"].cpu().numpy()
+    assert st[0] == valid.sum() and st[1] == blocked
+    assert abs(st[4] - np.sum(np.abs(np.exp(h["mu_logp"][valid]) - ora["r"][valid] * np.exp(h["mu_logp"][valid])))) <= 1e-3 * max(1.0, st[4])
+    return out, ora, dict(n_exempt=n_exempt, d_err=d_err, **info, **dinfo)
+
+
+# ------------------------------------------------------------------------------------- config 1
+
+@pytest.mark.parametrize("kernel", sorted(KERNELS))
+def test_tiny_binary_tv_fp32(kernel):
+    """T=256, V=4096, fp32 logits, Binary-TV, delta=0.2, all valid, seed 0."""
+    b = wl.tiny_binary_tv(DEV, seed=0)
+    _full_check(b, dppo.BINARY_TV, 0, 0.2, KERNELS[kernel])
+    # mask-stress: threshold at the median divergence so that a good share of rows is blocked
+    out = _run(b, dppo.BINARY_TV, 0, 0.2, KERNELS[kernel])
+    med = float(out["divergence"].median().item())
+    _full_check(b, dppo.BINARY_TV, 0, med, KERNELS[kernel], expect_blocked=lambda k, n: 0.1 * n < k < 0.5 * n)
+    _full_check(b, dppo.BINARY_KL, 0, 1e-4, KERNELS[kernel])
+
+
+# ------------------------------------------------------------------------------------- config 2
+
+@pytest.fixture(scope="module")
+def qwen_rows():
+    """333 rows of the Qwen3-vocabulary workload (bf16, V=151936) with top-64 lists; 333 rows on 148 SMs
+    give two full waves and a ragged third; a row is 38 chunks of 8 KB with a 768-byte tail."""
+    return wl.qwen_vocab_rows(DEV, seed=1, n_resp=9, resp_len=37, K=64, group=9)
+
+
+@pytest.mark.parametrize("variant,delta", [(dppo.BINARY_TV, 0.1), (dppo.BINARY_TV, 0.2), (dppo.BINARY_KL, 0.1), (dppo.BINARY_KL, 0.2)])
+def test_qwen_binary(qwen_rows, variant, delta):
+    out, ora, info = _full_check(qwen_rows, variant, 0, delta, dppo.KERNEL_RING)
+    assert info["frac_literal"] > 0.999999
+
+
+@pytest.mark.parametrize("variant", [dppo.BINARY_TV, dppo.BINARY_KL])
+def test_qwen_binary_mask_stress(qwen_rows, variant):
+    out = _run(qwen_rows, variant, 0, 1.0, dppo.KERNEL_RING)
+    med = float(out["divergence"].median().item())
+    _full_check(qwen_rows, variant, 0, med, dppo.KERNEL_RING, expect_blocked=lambda k, n: 0.1 * n < k < 0.5 * n)
+
+
+def test_qwen_fp32_gradient_and_generic_kernel(qwen_rows):
+    """fp32 gradient output meets the literal 2e-3*max bound; the scalar kernel agrees with the oracle too."""
+    _, _, info = _full_check(qwen_rows, dppo.BINARY_TV, 0, 0.02, dppo.KERNEL_RING, dlogits_f32=True)
+    assert info["max_err_over_max"] < 2e-5
+    _full_check(qwen_rows, dppo.BINARY_TV, 0, 0.02, dppo.KERNEL_GENERIC)
+    _full_check(qwen_rows, dppo.TOPK_KL, 64, 0.02, dppo.KERNEL_GENERIC, dlogits_f32=True)
+
+
+# ------------------------------------------------------------------------------------- config 3
+
+def test_qwen_topk_tv_k20(qwen_rows):
+    b = qwen_rows
+    b20 = wl.Batch(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None,
+                   b.mu_topk_ids[:, :20].contiguous(), b.mu_topk_p[:, :20].contiguous())
+    _full_check(b20, dppo.TOPK_TV, 20, 0.2, dppo.KERNEL_RING)
+    out = _run(b20, dppo.TOPK_TV, 20, 1.0, dppo.KERNEL_RING)
+    med = float(out["divergence"].median().item())
+    _full_check(b20, dppo.TOPK_TV, 20, med, dppo.KERNEL_RING, expect_blocked=lambda k, n: 0.1 * n < k < 0.5 * n)
+    # Top-K refines Binary: D_bin <= D_topk row by row (App. B)
+    bin_ = _run(b20, dppo.BINARY_TV, 0, 1.0, dppo.KERNEL_RING)
+    assert torch.all(bin_["divergence"] <= out["divergence"] + 1e-6)
+
+
+# ------------------------------------------------------------------------------------- config 4
+
+def test_ragged_topk_kl_k64():
+    """Ragged responses in padded blocks with a token mask, TopK-KL K=64, delta=0.05, rollout noise 0.3;
+    each padded block is one call with the global token-mean scale, as the full-size workload is run."""
+    lengths = [37, 128, 5, 90]
+    max_len = 128
+    n_valid = sum(lengths)
+    scale = 1.0 / n_valid
+    total_gpu, total_ora, blocked = 0.0, 0.0, 0
+    for i in range(len(lengths)):
+        b = wl.ragged_response(DEV, i, lengths, seed=3, max_len=max_len, K=64, group=4)
+        # poison the padding so that a kernel reading it would be caught
+        b.logits[lengths[i]:] = float("nan")
+        b.sampled_ids[lengths[i]:] = -7
+        out, ora, info = _full_check(b, dppo.TOPK_KL, 64, 0.05, dppo.KERNEL_RING, loss_scale=scale)
+        total_gpu += float(out["loss"].item())
+        total_ora += ora["loss"]
+        blocked += int((ora["M"][: lengths[i]] == 0).sum())
+        assert not out["dlogits"][lengths[i]:].any() and not out["divergence"][lengths[i]:].any()
+    assert blocked > 0
+    assert abs(total_gpu - total_ora) <= 1e-3 * abs(total_ora)
+
+
+# ------------------------------------------------------------------------------------- edge cases
+
+@pytest.mark.parametrize("kernel", sorted(KERNELS))
+@pytest.mark.parametrize("V,dtype", [(8, torch.bfloat16), (4104, torch.bfloat16), (4, torch.float32), (2052, torch.float32)])
+def test_small_vocab_topk_full(kernel, V, dtype):
+    """K = V (exact divergence, empty 'other' bucket) and K = 0 (Binary) on small vocabularies."""
+    T = 40
+    logits, a, mu_logp, ids, ps = wl.logits_rows(0, T, V, dtype, 11, DEV, sigma=2.0, zipf=1.1, sigma_mu=0.5, K=V)
+    adv = torch.where(torch.arange(T, device=DEV) % 3 == 0, -1.0, 0.7).to(torch.float32)
+    adv[5] = 0.0
+    tok = torch.ones(T, dtype=torch.uint8, device=DEV)
+    tok[7] = 0
+    b = wl.Batch(logits, a, mu_logp, adv, tok, ids, ps)
+    for variant in (dppo.TOPK_TV, dppo.TOPK_KL):
+        _full_check(b, variant, V, 0.05, KERNELS[kernel])
+        b0 = wl.Batch(logits, a, mu_logp, adv, tok, None, None)
+        o_top0, _, _ = _full_check(b0, variant, 0, 0.05, KERNELS[kernel])
+        o_bin, _, _ = _full_check(b0, variant - 2, 0, 0.05, KERNELS[kernel])
+        assert torch.allclose(o_top0["divergence"], o_bin["divergence"], atol=1e-6)
+
+
+def test_odd_vocab_falls_back_to_scalar_kernel():
+    T, V = 19, 1001
+    logits, a, mu_logp, ids, ps = wl.logits_rows(0, T, V, torch.bfloat16, 12, DEV, sigma=2.0, zipf=1.1, sigma_mu=0.5, K=7)
+    adv = torch.linspace(-1, 1, T, device=DEV)
+    b = wl.Batch(logits, a, mu_logp, adv, None, ids, ps)
+    _full_check(b, dppo.TOPK_KL, 7, 0.01, dppo.KERNEL_AUTO)
+    with pytest.raises(dppo.DppoError) as e:
+        _run(b, dppo.TOPK_KL, 7, 0.01, dppo.KERNEL_RING)
+    assert "alignment" in str(e.value)
+    # strided rows (a view into a wider buffer)
+    wide = torch.zeros((T, V + 23), dtype=torch.bfloat16, device=DEV)
+    wide[:, :V] = logits
+    b2 = wl.Batch(wide[:, :V], a, mu_logp, adv, None, ids, ps)
+    _full_check(b2, dppo.TOPK_TV, 7, 0.01, dppo.KERNEL_AUTO)
+
+
+def test_empty_and_fully_masked():
+    V = 4096
+    b = wl.tiny_binary_tv(DEV, seed=2, T=32, V=V)
+    empty = wl.Batch(b.logits[:0], b.sampled_ids[:0], b.mu_logp[:0], b.advantages[:0], None)
+    out = _run(empty, dppo.BINARY_TV, 0, 0.2, dppo.KERNEL_AUTO, want_stats=False)
+    assert float(out["loss"].item()) == 0.0 and out["dlogits"].shape == (0, V)
+    b.token_mask = torch.zeros(32, dtype=torch.uint8, device=DEV)
+    for k in KERNELS.values():
+        out = _run(b, dppo.BINARY_TV, 0, 0.2, k)
+        assert float(out["loss"].item()) == 0.0 and not out["dlogits"].any() and not out["mask"].any()
+        assert out["stats"][0].item() == 0
+
+
+@pytest.mark.parametrize("kernel", sorted(KERNELS))
+def test_in_place_and_determinism(kernel, qwen_rows):
+    b = qwen_rows
+    ref = _run(b, dppo.BINARY_KL, 0, 0.01, KERNELS[kernel])
+    again = _run(b, dppo.BINARY_KL, 0, 0.01, KERNELS[kernel])
+    assert torch.equal(ref["dlogits"], again["dlogits"]) and torch.equal(ref["loss"], again["loss"])
+    buf = b.logits.clone()
+    inpl = wl.Batch(buf, b.sampled_ids, b.mu_logp, b.advantages, None)
+    out = _run(inpl, dppo.BINARY_KL, 0, 0.01, KERNELS[kernel], dlogits=buf)
+    assert torch.equal(out["dlogits"], ref["dlogits"]) and torch.equal(out["divergence"], ref["divergence"])
+
+
+@pytest.mark.parametrize("kernel", sorted(KERNELS))
+def test_device_detected_anomalies_set_status(kernel):
+    """Bad ids and non-finite rows never trap: status bits are set and the row is treated as invalid."""
+    b = wl.tiny_binary_tv(DEV, seed=4, T=64, V=4096)
+    _, _, _, ids, ps = wl.logits_rows(0, 64, 4096, torch.float32, 4, DEV, sigma=2.0, zipf=0.0, peak=6.0, sigma_mu=0.05, K=5)
+    b.mu_topk_ids, b.mu_topk_p = ids.clone(), ps
+    b.sampled_ids[3] = 4096
+    b.sampled_ids[9] = -1
+    b.mu_topk_ids[11, 2] = 1 << 20
+    b.logits[17, 100] = float("nan")
+    b.logits[21, 5] = float("inf")
+    b.logits[30, :] = float("-inf")
+    out = _run(b, dppo.TOPK_KL, 5, 0.05, KERNELS[kernel])
+    assert int(out["status"].item()) == (dppo.binding.STATUS_BAD_SAMPLED_ID | dppo.binding.STATUS_BAD_TOPK_ID | dppo.binding.STATUS_NONFINITE_ROW)
+    bad = [3, 9, 11, 17, 21, 30]
+    for t in bad:
+        assert not out["dlogits"][t].any() and out["mask"][t].item() == 0 and out["divergence"][t].item() == 0
+    good = [t for t in range(64) if t not in bad]
+    h = P.host_inputs(b, good)
+    ora = P.run_oracle(h, O.TOPK_KL, 5, 0.05, 1.0 / 64)
+    P.check_scalars(out["divergence"][good].cpu().numpy(), out["mask"][good].cpu().numpy(), ora, h, 0.05)
+    P.check_dlogits(out["dlogits"][good], ora["dlogits"], out_is_bf16=False)
+    # -inf entries in an otherwise finite row are fine (zero probability)
+    b2 = wl.tiny_binary_tv(DEV, seed=5, T=16, V=4096)
+    b2.logits[:, 7::13] = float("-inf")
+    b2.sampled_ids[:] = 8
+    _full_check(b2, dppo.BINARY_TV, 0, 0.2, KERNELS[kernel])
+
+
+# ------------------------------------------------------------------------------------- host-buffer entry point
+
+def test_host_buffer_entry_matches_device_entry(qwen_rows):
+    b = qwen_rows
+    dev = _run(b, dppo.TOPK_TV, 64, 0.02, dppo.KERNEL_AUTO)
+    pin = lambda x: x.cpu().pin_memory()
+    out = dppo.dppo_loss_fwd_bwd_host(pin(b.logits), pin(b.sampled_ids), pin(b.mu_logp), pin(b.advantages), None,
+                                      dppo.TOPK_TV, 64, 0.02, pin(b.mu_topk_ids), pin(b.mu_topk_p),
+                                      rows_per_chunk=100, want_dlogits=True, device=DEV)
+    assert out["status"] == 0
+    assert torch.equal(out["divergence"], dev["divergence"].cpu()) and torch.equal(out["mask"], dev["mask"].cpu())
+    assert torch.equal(out["dlogits"], dev["dlogits"].cpu())
+    assert abs(out["loss"] - float(dev["loss"].item())) <= 1e-6 * abs(out["loss"]) + 1e-12
+
+
+# ------------------------------------------------------------------------------------- full size
+
+def test_full_size_binary_tv_sampled_rows():
+    """The benchmark's configuration (T=16384, V=151936, bf16, Binary-TV, delta=0.2): mask, divergence and
+    loss against the oracle on all rows (forward only), the gradient on sampled rows, and properties that
+    hold at any size."""
+    T = 16384
+    b = wl.qwen_vocab_rows(DEV, seed=1)
+    assert b.T == T
+    out = _run(b, dppo.BINARY_TV, 0, 0.2, dppo.KERNEL_AUTO)
+    assert int(out["status"].item()) == 0
+    rng = np.random.default_rng(0)
+    rows = np.sort(rng.choice(T, 48, replace=False))
+    h = P.host_inputs(b, rows)
+    ora = P.run_oracle(h, O.BINARY_TV, 0, 0.2, 1.0 / T)
+    P.check_scalars(out["divergence"].cpu().numpy()[rows], out["mask"].cpu().numpy()[rows], ora, h, 0.2)
+    mx = float(out["dlogits"].abs().max().item())
+    P.check_dlogits(out["dlogits"][torch.as_tensor(rows, device=DEV)], ora["dlogits"], out_is_bf16=True, max_abs=mx)
+    # the loss over a random eighth of the rows (token mask), same tensors, oracle forward only
+    tok = (torch.rand(T, generator=torch.Generator().manual_seed(5)) < 0.125).to(torch.uint8)
+    idx = np.nonzero(tok.numpy())[0]
+    bm = wl.Batch(b.logits, b.sampled_ids, b.mu_logp, b.advantages, tok.to(DEV))
+    outm = _run(bm, dppo.BINARY_TV, 0, 0.2, dppo.KERNEL_AUTO)
+    hb = P.host_inputs(bm, idx)
+    hb["token_mask"] = None
+    ob = P.run_oracle(hb, O.BINARY_TV, 0, 0.2, 1.0 / len(idx), want_grad=False)
+    P.check_scalars(outm["divergence"].cpu().numpy()[idx], outm["mask"].cpu().numpy()[idx], ob, hb, 0.2)
+    P.check_loss(float(outm["loss"].item()), ob["loss"], True, ob["row_loss"])
+    assert outm["stats"][0].item() == len(idx)
+    inv = torch.nonzero(tok == 0)[:, 0][:64].to(DEV)
+    assert not outm["dlogits"][inv].any()
+    # valid rows of the masked call equal the unmasked call's rows up to the scale factor T/len(idx)
+    t0 = int(idx[0])
+    ratio = (outm["dlogits"][t0].float() / out["dlogits"][t0].float().clamp_min(1e-30))[out["dlogits"][t0].float() > 1e-20]
+    assert torch.allclose(ratio, torch.full_like(ratio, T / len(idx)), rtol=2e-2)
+    # properties: gradient rows sum to ~0 (bf16 rounding noise), blocked rows are exactly zero
+    sums = out["dlogits"].to(torch.float32).sum(dim=1).abs().max().item()
+    assert sums <= 2e-3 * mx * 40
+    blocked = torch.nonzero(out["mask"] == 0)[:, 0]
+    assert not out["dlogits"][blocked].any()
