@@ -40,6 +40,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default="binary_tv", choices=["binary_tv", "binary_kl"])
+    ap.add_argument("--rows", type=int, default=T_ROWS, help="rows per GPU; anything but the default is a reduced case for profiling, not the benchmark workload")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -176,7 +177,7 @@ def run_ours(args):
     variant = dppo.BINARY_TV if args.variant == "binary_tv" else dppo.BINARY_KL
 
     # each rank owns T rows of the global batch of world*T rows
-    b = wl.qwen_vocab_rows(dev, seed=1 + rank)
+    b = wl.qwen_vocab_rows(dev, seed=1 + rank, rows=args.rows) if args.rows != T_ROWS else wl.qwen_vocab_rows(dev, seed=1 + rank)
     T = b.T
     scale = 1.0 / (T * world)
     dlogits = torch.empty_like(b.logits)
@@ -237,7 +238,8 @@ def run_ours(args):
         "metric": METRIC, "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "variant": args.variant, "rows_per_gpu": T, "l2": "inputs_larger_than_L2 (4.98 GB read + 4.98 GB written per step)",
+        "config": {"workload": WORKLOAD if T == T_ROWS else f"REDUCED to {T} rows (profiling case): " + WORKLOAD,
+                   "variant": args.variant, "rows_per_gpu": T, "l2": "inputs_larger_than_L2 (4.98 GB read + 4.98 GB written per step)",
                    "parallelism": f"dp{world} row shards, no data-path collective", "logits_dtype": "bf16", "dlogits_dtype": "bf16"},
         "roofline": roofline, "clocks": clocks, "gpu_launches": 3 * args.steps, "loss": loss_val,
     }
