@@ -1,31 +1,46 @@
 // Row kernel for 16-byte aligned layouts: one persistent CTA per SM streams token rows through a
-// ring of shared-memory slots filled by bulk asynchronous copies (TMA, cp.async.bulk) that a
-// producer warp issues and mbarriers track.
+// ring of shared-memory slots filled by bulk asynchronous copies (TMA, cp.async.bulk) and runs a
+// four-role pipeline connected only by mbarriers:
 //
-// Per row: sweep 1 consumes the chunks as they land (online max / sum of exponentials); the last
-// `nslots` chunks of the row stay resident in the ring, so sweep 2 (the gradient) reads them from
-// shared memory; only the head of a row that is longer than the ring is fetched a second time
-// (it was loaded with an L2 evict-last hint and normally still sits in L2).  A row that fits in
-// the ring is read from HBM exactly once.  The gradient goes out with 128-bit streaming stores.
-// While sweep 2 frees slots the producer is already loading the next row into them.
+//   producer warp   issues the bulk copies of the rows' chunks, slot by slot, as slots are released
+//   sum warps (8)   sweep 1: consume the chunks of row n+1 as they land, sum of exponentials against
+//                   a per-thread reference (moved up only if a vector would overflow), hand the
+//                   per-warp partials to the scalar warp
+//   scalar warp     log-sum-exp, ratio, divergence, mask, loss term of the row; posts the gradient
+//                   coefficients
+//   grad warps (8)  sweep 2 of row n: read the chunks that are still resident in the ring, write
+//                   the gradient with 128-bit streaming stores, release the slots
+//
+// The last `nslots` chunks of a row stay resident between the sweeps; only the head of a row that
+// is longer than the ring is fetched a second time (it was loaded with an L2 evict-last hint and
+// normally still sits in L2).  A row that fits in the ring is read from HBM exactly once.  Because
+// the sum warps work one row ahead of the grad warps, the scalar stage and the waits of one group
+// are covered by the arithmetic of the other.
+//
+// Every wait is bounded: a wait that runs out sets a shared abort flag and the status bit
+// DPPO_STATUS_WAIT_LIMIT; from then on every warp skips its remaining work and returns.
 #include "dppo_common.cuh"
 
 namespace dppo {
 
-constexpr int kChunkBytes = 8192;
-constexpr int kConsumers = 512;                 // 16 warps; one 16-byte vector per thread per chunk
-constexpr int kConsumerWarps = kConsumers / 32;
-constexpr int kRingThreads = kConsumers + 32;   // + producer warp
-constexpr int kMiscBytes = 1024;                // barriers + reduction scratch
-constexpr int kMaxSlots = 28;
-static_assert(kChunkBytes == kConsumers * 16, "one vector per consumer thread per chunk");
+constexpr int kChunkBytes = 16384;
+constexpr int kGroupThreads = 256;              // threads of the sum group and of the grad group
+constexpr int kGroupWarps = kGroupThreads / 32;
+constexpr int kVecPerThread = kChunkBytes / 16 / kGroupThreads;   // 16-byte vectors per thread per chunk
+constexpr int kRingThreads = 2 * kGroupThreads + 64;              // + scalar warp + producer warp
+constexpr int kMiscBytes = 1024;                // barriers + hand-off buffers
+constexpr int kMaxSlots = 14;
+static_assert(kVecPerThread * kGroupThreads * 16 == kChunkBytes, "chunk geometry");
 
 struct RingMisc {
-  unsigned long long full[kMaxSlots];
-  unsigned long long empty[kMaxSlots];
-  float s_m[kConsumerWarps];
-  float s_s[kConsumerWarps];
-  RowCoef coef;
+  unsigned long long full[kMaxSlots];    // chunk landed            (producer -> sum, grad)
+  unsigned long long empty[kMaxSlots];   // chunk no longer needed  (sum or grad -> producer)
+  unsigned long long part_full[2];       // partials of a row ready (sum -> scalar)
+  unsigned long long part_empty[2];
+  unsigned long long coef_full[2];       // coefficients of a row ready (scalar -> grad)
+  unsigned long long coef_empty[2];
+  float2 part[2][kGroupWarps];           // (reference, sum of exp) per sum warp
+  RowCoef coef[2];
   int abort_flag;
 };
 static_assert(sizeof(RingMisc) <= kMiscBytes, "misc area");
@@ -58,7 +73,7 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 // Bounded wait: gives up after ~2 s (or when another thread already gave up) and returns false.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  unsigned long long t0 = globaltimer_ns();
+  const unsigned long long t0 = globaltimer_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 0xff) == 0) {
@@ -67,13 +82,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+// All lanes of a warp wait; the warp proceeds only if every lane saw the phase complete.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  const bool ok = mbar_wait(bar, parity, abort_flag);
+  return __all_sync(0xffffffffu, ok);
+}
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
       ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
       : "memory");
 }
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
@@ -106,27 +125,30 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// Writes N gradient values starting at element j0 of an output row.
+// Writes N gradient values starting at element j0 of an output row; `sign2` (0 or 0x80008000)
+// flips the sign of every value.
 template <typename OutT, int N> struct Store;
 template <> struct Store<__nv_bfloat16, 8> {
-  static __device__ __forceinline__ void run(__nv_bfloat16* row, int64_t j0, const float* v) {
+  static __device__ __forceinline__ void run(__nv_bfloat16* row, uint32_t j0, const float* v, uint32_t sign2 = 0u) {
     uint4 o;
-    o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
-    o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);
+    o.x = pack_bf16x2(v[0], v[1]) ^ sign2; o.y = pack_bf16x2(v[2], v[3]) ^ sign2;
+    o.z = pack_bf16x2(v[4], v[5]) ^ sign2; o.w = pack_bf16x2(v[6], v[7]) ^ sign2;
     stg128_cs(row + j0, o);
   }
 };
 template <> struct Store<float, 8> {
-  static __device__ __forceinline__ void run(float* row, int64_t j0, const float* v) {
-    uint4 o0 = {__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])};
-    uint4 o1 = {__float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7])};
+  static __device__ __forceinline__ void run(float* row, uint32_t j0, const float* v, uint32_t sign2 = 0u) {
+    const uint32_t sg = sign2 & 0x80000000u;
+    uint4 o0 = {__float_as_uint(v[0]) ^ sg, __float_as_uint(v[1]) ^ sg, __float_as_uint(v[2]) ^ sg, __float_as_uint(v[3]) ^ sg};
+    uint4 o1 = {__float_as_uint(v[4]) ^ sg, __float_as_uint(v[5]) ^ sg, __float_as_uint(v[6]) ^ sg, __float_as_uint(v[7]) ^ sg};
     stg128_cs(row + j0, o0);
     stg128_cs(row + j0 + 4, o1);
   }
 };
 template <> struct Store<float, 4> {
-  static __device__ __forceinline__ void run(float* row, int64_t j0, const float* v) {
-    uint4 o0 = {__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])};
+  static __device__ __forceinline__ void run(float* row, uint32_t j0, const float* v, uint32_t sign2 = 0u) {
+    const uint32_t sg = sign2 & 0x80000000u;
+    uint4 o0 = {__float_as_uint(v[0]) ^ sg, __float_as_uint(v[1]) ^ sg, __float_as_uint(v[2]) ^ sg, __float_as_uint(v[3]) ^ sg};
     stg128_cs(row + j0, o0);
   }
 };
@@ -140,6 +162,15 @@ struct RingPos {             // position in the endless sequence of slot uses
   }
 };
 
+// Row bookkeeping every role evaluates identically: >= 0 sampled id of a valid row, -1 row masked
+// out (or past the end), -2 sampled id out of range (row treated as invalid, status bit).
+__device__ __forceinline__ int load_meta(const RowParams& p, int64_t t) {
+  if (t >= p.T) return -1;
+  if (p.token_mask && p.token_mask[t] == 0) return -1;
+  const int a = p.sampled_ids[t];
+  return (a < 0 || (int64_t)a >= p.V) ? -2 : a;
+}
+
 template <typename InT, typename OutT>
 __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParams p, int nslots) {
   extern __shared__ __align__(128) unsigned char smem[];
@@ -148,13 +179,21 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
   const uint32_t slots_base = smem_u32(smem);
   const uint32_t full_base = smem_u32(&misc->full[0]);
   const uint32_t empty_base = smem_u32(&misc->empty[0]);
+  const uint32_t part_full = smem_u32(&misc->part_full[0]), part_empty = smem_u32(&misc->part_empty[0]);
+  const uint32_t coef_full = smem_u32(&misc->coef_full[0]), coef_empty = smem_u32(&misc->coef_empty[0]);
   volatile int* abort_flag = &misc->abort_flag;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
     for (int i = 0; i < nslots; ++i) {
       mbar_init(full_base + 8u * i, 1);
-      mbar_init(empty_base + 8u * i, kConsumerWarps);
+      mbar_init(empty_base + 8u * i, kGroupWarps);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(part_full + 8u * i, kGroupWarps);
+      mbar_init(part_empty + 8u * i, 1);
+      mbar_init(coef_full + 8u * i, 1);
+      mbar_init(coef_empty + 8u * i, kGroupWarps);
     }
     misc->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -162,142 +201,250 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
   }
   __syncthreads();
 
-  const int64_t row_bytes = p.V * (int64_t)sizeof(InT);
-  const int C = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);   // chunks per row
-  const int L = C > nslots ? C - nslots : 0;                          // head chunks fetched twice
-  const char* logits = reinterpret_cast<const char*>(p.logits);
+  const uint32_t row_bytes = (uint32_t)(p.V * (int64_t)sizeof(InT));     // launcher guarantees < 2^31
+  const int C = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);      // chunks per row
+  const int L = C > nslots ? C - nslots : 0;                             // head chunks fetched twice
+  const int64_t t0 = blockIdx.x, G = gridDim.x;
 
-  if (tid >= kConsumers) {
+  if (warp == 2 * kGroupWarps + 1) {
     // ------------------------------------------------------------------ producer (one lane)
-    if (tid == kConsumers) {
+    if (lane == 0) {
       uint64_t pol_keep, pol_stream;
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+      const char* logits = reinterpret_cast<const char*>(p.logits);
       RingPos pos{0, 0};
-      bool first_lap = true;
-      bool ok = true;
-      for (int64_t t = blockIdx.x; t < p.T && ok; t += gridDim.x) {
-        if (p.token_mask && p.token_mask[t] == 0) continue;
-        int a = p.sampled_ids[t];
-        if (a < 0 || (int64_t)a >= p.V) continue;
-        const char* row = logits + t * p.ld_in * (int64_t)sizeof(InT);
-        for (int i = 0; i < C + L; ++i) {
-          const int c = (i < C) ? i : i - C;
-          if (!first_lap) {
-            if (!mbar_wait(empty_base + 8u * pos.slot, pos.phase ^ 1u, abort_flag)) { ok = false; break; }
+      bool first_lap = true, ok = true;
+      int meta = load_meta(p, t0);
+      for (int64_t t = t0; t < p.T && ok; t += G) {
+        const int meta_next = load_meta(p, t + G);
+        if (meta >= 0) {
+          const char* row = logits + t * p.ld_in * (int64_t)sizeof(InT);
+          for (int i = 0; i < C + L; ++i) {
+            const int c = (i < C) ? i : i - C;
+            // lap u >= 1 of a slot needs its (u-1)-th release: parity (u-1)&1 = phase^1
+            if (!first_lap && !mbar_wait(empty_base + 8u * pos.slot, pos.phase ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t off = (uint32_t)c * kChunkBytes;
+            const uint32_t bytes = (row_bytes - off) < (uint32_t)kChunkBytes ? (row_bytes - off) : (uint32_t)kChunkBytes;
+            const uint32_t bar = full_base + 8u * pos.slot;
+            mbar_arrive_expect_tx(bar, bytes);
+            bulk_load(slots_base + (uint32_t)pos.slot * kChunkBytes, row + off, bytes, bar, (i < L) ? pol_keep : pol_stream);
+            pos.slot += 1;
+            if (pos.slot == nslots) { pos.slot = 0; pos.phase ^= 1u; first_lap = false; }
           }
-          const int64_t off = (int64_t)c * kChunkBytes;
-          const uint32_t bytes = (uint32_t)((row_bytes - off) < kChunkBytes ? (row_bytes - off) : kChunkBytes);
-          const uint32_t bar = full_base + 8u * pos.slot;
-          mbar_arrive_expect_tx(bar, bytes);
-          bulk_load(slots_base + (uint32_t)pos.slot * kChunkBytes, row + off, bytes, bar,
-                    (i < L) ? pol_keep : pol_stream);
-          pos.slot += 1;
-          if (pos.slot == nslots) { pos.slot = 0; pos.phase ^= 1u; first_lap = false; }
         }
+        meta = meta_next;
       }
     }
-    return;
-  }
-
-  // -------------------------------------------------------------------- consumers (16 warps)
-  // A wait that runs out sets abort_flag.  From then on every consumer keeps walking the same
-  // control flow (so the named barriers still match) but neither waits nor touches memory, and
-  // all of them leave together at the end of the row.
-  const int lane = tid & 31, warp = tid >> 5;
-  const double scale = p.hdr->scale;
-  OutT* dlogits = reinterpret_cast<OutT*>(p.dlogits);
-  const uint32_t my_off = (uint32_t)tid * 16u;
-  RingPos pos{0, 0};
-  bool alive = true;
-
-  for (int64_t t = blockIdx.x; t < p.T; t += gridDim.x) {
-    OutT* drow = dlogits + t * p.ld_out;
-    bool valid = p.token_mask ? (p.token_mask[t] != 0) : true;
-    int a = 0, flags = 0;
-    if (valid) {
-      a = p.sampled_ids[t];
-      if (a < 0 || (int64_t)a >= p.V) { valid = false; flags = DPPO_STATUS_BAD_SAMPLED_ID; }
-    }
-    if (!valid) {
-      float zero[N] = {};
-      for (int64_t j0 = (int64_t)tid * N; j0 < p.V; j0 += (int64_t)kConsumers * N) Store<OutT, N>::run(drow, j0, zero);
-      if (tid == 0) {
-        p.divergence[t] = 0.f; p.mask[t] = 0; p.row_loss[t] = 0.f; p.row_r[t] = 0.f; p.row_absdiff[t] = 0.f;
-        if (flags) atomicOr(p.status, flags);
+  } else if (warp < kGroupWarps) {
+    // ------------------------------------------------------------------ sum warps: sweep 1
+    const uint32_t gtid = (uint32_t)tid;
+    RingPos pos{0, 0};
+    uint32_t vrow = 0;
+    int meta = load_meta(p, t0);
+    for (int64_t t = t0; t < p.T; t += G) {
+      const int meta_next = load_meta(p, t + G);
+      if (__shfl_sync(0xffffffffu, *abort_flag, 0)) break;
+      if (meta >= 0) {
+        // per-thread partial: s = sum exp(z - ref); ref is the maximum of the thread's first finite
+        // vector and moves up only when a vector's sum shows that an entry exceeds it by > 44
+        float ref = -INFINITY, nm = 0.f, s = 0.f;
+        RingPos p1 = pos;
+        for (int c = 0; c < C; ++c) {
+          const bool ok = mbar_wait_warp(full_base + 8u * p1.slot, p1.phase, abort_flag);
+          const uint32_t cbase = (uint32_t)c * kChunkBytes;
+          const uint32_t sbase = slots_base + (uint32_t)p1.slot * kChunkBytes;
+          if (ok) {
+#pragma unroll
+            for (int k = 0; k < kVecPerThread; ++k) {
+              const uint32_t off = ((uint32_t)k * kGroupThreads + gtid) * 16u;
+              if (cbase + off < row_bytes) {
+                const uint4 v = lds128(sbase + off);
+                float z[N];
+                Vec<InT>::unpack(v, z);
+                if (ref == -INFINITY) {
+                  float vm = z[0];
+#pragma unroll
+                  for (int i = 1; i < N; ++i) vm = fmaxf(vm, z[i]);
+                  if (vm != -INFINITY) { ref = vm; nm = -vm * kLog2e; }
+                }
+                float e[N];
+#pragma unroll
+                for (int i = 0; i < N; ++i) e[i] = ex2_approx(fmaf(z[i], kLog2e, nm));
+#pragma unroll
+                for (int w = 1; w < N; w <<= 1)
+#pragma unroll
+                  for (int i = 0; i + w < N; i += 2 * w) e[i] += e[i + w];
+                float vs = e[0];
+                if (!(vs <= 1.8446744e19f) && ref != -INFINITY) {   // > 2^64 (or NaN): move the reference up
+                  float vm = z[0];
+#pragma unroll
+                  for (int i = 1; i < N; ++i) vm = fmaxf(vm, z[i]);
+                  if (vm > ref) {
+                    s *= ex2_approx((ref - vm) * kLog2e);
+                    ref = vm;
+                    nm = -vm * kLog2e;
+                    vs = 0.f;
+#pragma unroll
+                    for (int i = 0; i < N; ++i) vs += ex2_approx(fmaf(z[i], kLog2e, nm));
+                  }
+                }
+                if (ref != -INFINITY) s += vs;
+              }
+            }
+          }
+          if (c < L) {                     // head of a long row: give the slot back, it is re-fetched for sweep 2
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_base + 8u * p1.slot);
+          }
+          p1.advance(nslots);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float m2 = __shfl_xor_sync(0xffffffffu, ref, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
+          merge_ms(ref, s, m2, s2);
+        }
+        if (lane == 0) {
+          const uint32_t b = vrow & 1u;
+          bool ok = true;
+          if (vrow >= 2) ok = mbar_wait(part_empty + 8u * b, ((vrow >> 1) & 1u) ^ 1u, abort_flag);
+          if (ok) {
+            misc->part[b][warp] = make_float2(ref, s);
+            mbar_arrive(part_full + 8u * b);
+          }
+        }
+        pos = p1;
+        pos.advance(nslots, L);            // the re-fetched head chunks belong to the grad warps
+        ++vrow;
       }
-      continue;
+      meta = meta_next;
     }
-
-    // ---- sweep 1: online (max, sum exp) over the chunks as they land
-    float m = -INFINITY, s = 0.f;
-    RingPos p1 = pos;
-    for (int c = 0; c < C; ++c) {
-      if (alive && !mbar_wait(full_base + 8u * p1.slot, p1.phase, abort_flag)) alive = false;
-      const int64_t boff = (int64_t)c * kChunkBytes + my_off;
-      if (alive && boff < row_bytes) {
-        uint4 v = lds128(slots_base + (uint32_t)p1.slot * kChunkBytes + my_off);
-        float z[N];
-        Vec<InT>::unpack(v, z);
-        float vm = z[0];
-#pragma unroll
-        for (int i = 1; i < N; ++i) vm = fmaxf(vm, z[i]);
-        if (vm > m) { s *= ex2_approx((m - vm) * kLog2e); m = vm; }
-        const float nm = (m == -INFINITY) ? 0.f : -m * kLog2e;
-        float e[N];
-#pragma unroll
-        for (int i = 0; i < N; ++i) e[i] = ex2_approx(fmaf(z[i], kLog2e, nm));
-#pragma unroll
-        for (int w = 1; w < N; w <<= 1)
-#pragma unroll
-          for (int i = 0; i + w < N; i += 2 * w) e[i] += e[i + w];
-        s += e[0];
-      }
-      if (c < L) {                       // head of a long row: give the slot back, it is re-fetched for sweep 2
+  } else if (warp < 2 * kGroupWarps) {
+    // ------------------------------------------------------------------ grad warps: sweep 2
+    const uint32_t gtid = (uint32_t)(tid - kGroupThreads);
+    OutT* dlogits = reinterpret_cast<OutT*>(p.dlogits);
+    RingPos pos{0, 0};
+    uint32_t vrow = 0;
+    int meta = load_meta(p, t0);
+    for (int64_t t = t0; t < p.T; t += G) {
+      const int meta_next = load_meta(p, t + G);
+      if (__shfl_sync(0xffffffffu, *abort_flag, 0)) break;
+      OutT* drow = dlogits + t * p.ld_out;
+      if (meta < 0) {
+        const float zero[N] = {};
+        for (uint32_t j0 = gtid * N; j0 < (uint32_t)p.V; j0 += kGroupThreads * N) Store<OutT, N>::run(drow, j0, zero);
+      } else {
+        const uint32_t b = vrow & 1u;
+        const bool have = mbar_wait_warp(coef_full + 8u * b, (vrow >> 1) & 1u, abort_flag);
+        RowCoef coef = misc->coef[b];
         __syncwarp();
-        if (lane == 0) mbar_arrive(empty_base + 8u * p1.slot);
-      }
-      p1.advance(nslots);
-    }
+        if (lane == 0 && have) mbar_arrive(coef_empty + 8u * b);
+        if (!have) coef.zero_row = 1;
+        const uint32_t sign2 = (coef.sgn < 0.f) ? 0x80008000u : 0u;
+        const uint32_t a = (uint32_t)meta;
+        auto grad_chunk = [&](int c, int slot, bool ok) {
+          const uint32_t cbase = (uint32_t)c * kChunkBytes;
+          const uint32_t sbase = slots_base + (uint32_t)slot * kChunkBytes;
+          if (ok) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
-      merge_ms(m, s, m2, s2);
+            for (int k = 0; k < kVecPerThread; ++k) {
+              const uint32_t off = ((uint32_t)k * kGroupThreads + gtid) * 16u;
+              if (cbase + off < row_bytes) {
+                const uint32_t j0 = (cbase + off) / (uint32_t)sizeof(InT);
+                float v[N];
+                if (coef.zero_row) {
+#pragma unroll
+                  for (int i = 0; i < N; ++i) v[i] = 0.f;
+                } else {
+                  const uint4 raw = lds128(sbase + off);
+                  float z[N];
+                  Vec<InT>::unpack(raw, z);
+#pragma unroll
+                  for (int i = 0; i < N; ++i) v[i] = ex2_approx(fmaf(z[i], kLog2e, coef.c2));
+                  if (a - j0 < (uint32_t)N) {             // the sampled token's entry is g * (pi(a) - 1)
+#pragma unroll
+                    for (int i = 0; i < N; ++i)
+                      if (j0 + i == a) v[i] = coef.fix * coef.sgn;   // the store flips it back
+                  }
+                }
+                Store<OutT, N>::run(drow, j0, v, sign2);
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty_base + 8u * slot);
+        };
+        RingPos p2 = pos;
+        p2.advance(nslots, L);
+        for (int c = L; c < C; ++c) {              // resident chunks: the phase is complete, the wait returns at once
+          const bool ok = mbar_wait_warp(full_base + 8u * p2.slot, p2.phase, abort_flag);
+          grad_chunk(c, p2.slot, ok);
+          p2.advance(nslots);
+        }
+        for (int c = 0; c < L; ++c) {              // re-fetched head of a long row
+          const bool ok = mbar_wait_warp(full_base + 8u * p2.slot, p2.phase, abort_flag);
+          grad_chunk(c, p2.slot, ok);
+          p2.advance(nslots);
+        }
+        pos = p2;                                  // = start + C + L
+        ++vrow;
+      }
+      meta = meta_next;
     }
-    if (lane == 0) { misc->s_m[warp] = m; misc->s_s[warp] = s; }
-    consumer_bar();
-    const bool dead = (*abort_flag != 0);          // same answer on every consumer here
-
-    // ---- scalar stage (warp 0): lse, ratio, divergence, mask, coefficients
-    if (warp == 0) {
-      RowCoef coef;
-      coef.c2 = 0.f; coef.sgn = 0.f; coef.fix = 0.f; coef.zero_row = 1;
+  } else {
+    // ------------------------------------------------------------------ scalar warp
+    const double scale = p.hdr->scale;
+    uint32_t vrow = 0;
+    int meta = load_meta(p, t0);
+    for (int64_t t = t0; t < p.T; t += G) {
+      const int meta_next = load_meta(p, t + G);
+      if (__shfl_sync(0xffffffffu, *abort_flag, 0)) break;
+      int flags = (meta == -2) ? DPPO_STATUS_BAD_SAMPLED_ID : 0;
       float D = 0.f, r = 0.f, absdiff = 0.f;
       int M = 0;
       double g = 0.0;
-      if (!dead) {
-        float mm = -INFINITY;
-        for (int w = 0; w < kConsumerWarps; ++w) mm = fmaxf(mm, misc->s_m[w]);
-        double S = 0.0;
-        for (int w = 0; w < kConsumerWarps; ++w) {
-          float sw = misc->s_s[w];
-          if (sw > 0.f || sw != sw) S += (double)sw * exp((double)misc->s_m[w] - (double)mm);
+      if (meta >= 0) {
+        const int a = meta;
+        const uint32_t b = vrow & 1u;
+        const InT* zrow = reinterpret_cast<const InT*>(p.logits) + t * p.ld_in;
+        const float z_a = to_f32<InT>(zrow[a]);                       // in flight while we wait for the partials
+        const bool have = mbar_wait_warp(part_full + 8u * b, (vrow >> 1) & 1u, abort_flag);
+        float2 pr = make_float2(-INFINITY, 0.f);
+        if (lane < kGroupWarps) pr = misc->part[b][lane];
+        __syncwarp();
+        if (lane == 0 && have) mbar_arrive(part_empty + 8u * b);
+        RowCoef coef;
+        coef.c2 = 0.f; coef.sgn = 0.f; coef.fix = 0.f; coef.zero_row = 1;
+        if (have) {
+          float mm = pr.x;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
+          double part = 0.0;
+          if (pr.y > 0.f || pr.y != pr.y) part = (double)pr.y * exp((double)pr.x - (double)mm);
+          const double S = warp_sum(part);
+          const double lse = (double)mm + log(S);
+          if (!isfinite(lse)) {
+            flags |= DPPO_STATUS_NONFINITE_ROW;
+          } else {
+            double pi_a;
+            int f2 = 0;
+            auto z_at = [&](int id) { return id == a ? z_a : to_f32<InT>(zrow[id]); };
+            row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
+            if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
+            else coef = make_coef(g, lse, pi_a);
+          }
         }
-        const double lse = (double)mm + log(S);
-        if (!isfinite(lse)) {
-          flags |= DPPO_STATUS_NONFINITE_ROW;
-        } else {
-          const InT* zrow = reinterpret_cast<const InT*>(p.logits) + t * p.ld_in;
-          double pi_a;
-          int f2 = 0;
-          auto z_at = [&](int id) { return to_f32<InT>(zrow[id]); };
-          row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
-          if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
-          else coef = make_coef(g, lse, pi_a);
+        if (lane == 0) {
+          bool ok = have;
+          if (ok && vrow >= 2) ok = mbar_wait(coef_empty + 8u * b, ((vrow >> 1) & 1u) ^ 1u, abort_flag);
+          if (ok) {
+            misc->coef[b] = coef;
+            mbar_arrive(coef_full + 8u * b);
+          }
         }
+        ++vrow;
       }
       if (lane == 0) {
-        misc->coef = coef;
         p.divergence[t] = D;
         p.mask[t] = (uint8_t)M;
         p.row_loss[t] = (float)(-g);
@@ -305,58 +452,16 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         p.row_absdiff[t] = absdiff;
         if (flags) atomicOr(p.status, flags);
       }
+      meta = meta_next;
     }
-    consumer_bar();
-    const RowCoef coef = misc->coef;
-    const uint32_t sign_bit = (coef.sgn < 0.f) ? 0x80000000u : 0u;
-
-    // ---- sweep 2: gradient; resident chunks L..C-1 from the ring, then the re-fetched head 0..L-1
-    auto grad_chunk = [&](int c, int slot) {
-      const int64_t boff = (int64_t)c * kChunkBytes + my_off;
-      if (alive && boff < row_bytes) {
-        const int64_t j0 = boff / (int64_t)sizeof(InT);
-        float v[N];
-        if (coef.zero_row) {
-#pragma unroll
-          for (int k = 0; k < N; ++k) v[k] = 0.f;
-        } else {
-          uint4 raw = lds128(slots_base + (uint32_t)slot * kChunkBytes + my_off);
-          float z[N];
-          Vec<InT>::unpack(raw, z);
-#pragma unroll
-          for (int k = 0; k < N; ++k)
-            v[k] = __uint_as_float(__float_as_uint(ex2_approx(fmaf(z[k], kLog2e, coef.c2))) | sign_bit);
-          if ((int64_t)a >= j0 && (int64_t)a < j0 + N) {
-#pragma unroll
-            for (int k = 0; k < N; ++k)
-              if (j0 + k == (int64_t)a) v[k] = coef.fix;
-          }
-        }
-        Store<OutT, N>::run(drow, j0, v);
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty_base + 8u * slot);
-    };
-    RingPos p2 = pos;
-    p2.advance(nslots, L);
-    for (int c = L; c < C; ++c) {
-      grad_chunk(c, p2.slot);
-      p2.advance(nslots);
-    }
-    for (int c = 0; c < L; ++c) {                  // p1 points at the first re-fetched chunk
-      if (alive && !mbar_wait(full_base + 8u * p1.slot, p1.phase, abort_flag)) alive = false;
-      grad_chunk(c, p1.slot);
-      p1.advance(nslots);
-    }
-    pos = p1;                                     // = start + C + L
-    consumer_bar();                               // scratch (s_m, coef) is reused by the next row
-    if (*abort_flag) break;                       // uniform: written before the barrier
   }
+
+  __syncwarp();
   if (*abort_flag) {
-    if (tid == 0) atomicOr(p.status, DPPO_STATUS_WAIT_LIMIT);
+    if (lane == 0) atomicOr(p.status, DPPO_STATUS_WAIT_LIMIT);
     // leave time for bulk copies that may still be in flight towards this CTA's shared memory
-    const unsigned long long t0 = globaltimer_ns();
-    while (globaltimer_ns() - t0 < 1000000ull) __nanosleep(1000);
+    const unsigned long long t_exit = globaltimer_ns();
+    while (globaltimer_ns() - t_exit < 1000000ull) __nanosleep(1000);
   }
 }
 
@@ -370,7 +475,7 @@ static int ring_slots(int dev) {
 bool ring_layout_ok(const RowParams& p, int in_dtype, int out_dtype) {
   const int64_t in_sz = (in_dtype == DPPO_BF16) ? 2 : 4, out_sz = (out_dtype == DPPO_BF16) ? 2 : 4;
   if (in_dtype == DPPO_F32 && out_dtype != DPPO_F32) return false;
-  if ((p.V * in_sz) % 16 != 0) return false;
+  if ((p.V * in_sz) % 16 != 0 || p.V * in_sz >= ((int64_t)1 << 31)) return false;
   if (((uintptr_t)p.logits) % 16 != 0 || (p.ld_in * in_sz) % 16 != 0) return false;
   if (((uintptr_t)p.dlogits) % 16 != 0 || (p.ld_out * out_sz) % 16 != 0) return false;
   return true;

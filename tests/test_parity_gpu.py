@@ -240,7 +240,8 @@ def test_host_buffer_entry_matches_device_entry(qwen_rows):
     assert out["status"] == 0
     assert torch.equal(out["divergence"], dev["divergence"].cpu()) and torch.equal(out["mask"], dev["mask"].cpu())
     assert torch.equal(out["dlogits"], dev["dlogits"].cpu())
-    assert abs(out["loss"] - float(dev["loss"].item())) <= 1e-6 * abs(out["loss"]) + 1e-12
+    # the host entry passes the token-mean scale as an fp32 argument and adds the chunks' partial losses
+    assert abs(out["loss"] - float(dev["loss"].item())) <= 1e-4 * abs(out["loss"]) + 1e-12
 
 
 # ------------------------------------------------------------------------------------- full size
