@@ -255,41 +255,66 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
           const uint32_t sbase = slots_base + (uint32_t)p1.slot * kChunkBytes;
           if (ok) {
+            const bool full_chunk = cbase + (uint32_t)kChunkBytes <= row_bytes;
+            bool done = false;
+            if (full_chunk) {
+              // straight-line path: all loads first, then 4 x N independent exponentials
+              uint4 v[kVecPerThread];
 #pragma unroll
-            for (int k = 0; k < kVecPerThread; ++k) {
-              const uint32_t off = ((uint32_t)k * kGroupThreads + gtid) * 16u;
-              if (cbase + off < row_bytes) {
-                const uint4 v = lds128(sbase + off);
-                float z[N];
-                Vec<InT>::unpack(v, z);
-                if (ref == -INFINITY) {
-                  float vm = z[0];
+              for (int k = 0; k < kVecPerThread; ++k) v[k] = lds128(sbase + ((uint32_t)k * kGroupThreads + gtid) * 16u);
+              float z[kVecPerThread][N];
 #pragma unroll
-                  for (int i = 1; i < N; ++i) vm = fmaxf(vm, z[i]);
-                  if (vm != -INFINITY) { ref = vm; nm = -vm * kLog2e; }
-                }
+              for (int k = 0; k < kVecPerThread; ++k) Vec<InT>::unpack(v[k], z[k]);
+              if (ref == -INFINITY) {            // first chunk of the row: reference = maximum of the first entries
+                float vm = z[0][0];
+#pragma unroll
+                for (int k = 0; k < kVecPerThread; ++k)
+#pragma unroll
+                  for (int i = 0; i < N; ++i) vm = fmaxf(vm, z[k][i]);
+                if (vm != -INFINITY) { ref = vm; nm = -vm * kLog2e; }
+              }
+              float acc[kVecPerThread];
+#pragma unroll
+              for (int k = 0; k < kVecPerThread; ++k) {
                 float e[N];
 #pragma unroll
-                for (int i = 0; i < N; ++i) e[i] = ex2_approx(fmaf(z[i], kLog2e, nm));
+                for (int i = 0; i < N; ++i) e[i] = ex2_approx(fmaf(z[k][i], kLog2e, nm));
 #pragma unroll
                 for (int w = 1; w < N; w <<= 1)
 #pragma unroll
                   for (int i = 0; i + w < N; i += 2 * w) e[i] += e[i + w];
-                float vs = e[0];
-                if (!(vs <= 1.8446744e19f) && ref != -INFINITY) {   // > 2^64 (or NaN): move the reference up
+                acc[k] = e[0];
+              }
+#pragma unroll
+              for (int w = 1; w < kVecPerThread; w <<= 1)
+#pragma unroll
+                for (int k = 0; k + w < kVecPerThread; k += 2 * w) acc[k] += acc[k + w];
+              if (acc[0] <= 7.3786976e19f && ref != -INFINITY) { s += acc[0]; done = true; }   // <= 2^66, not NaN
+            }
+            if (!done) {
+              // tail chunk, or an entry far above the reference (or NaN): vector by vector, moving the reference up
+#pragma unroll 1
+              for (int k = 0; k < kVecPerThread; ++k) {
+                const uint32_t off = ((uint32_t)k * kGroupThreads + gtid) * 16u;
+                if (cbase + off < row_bytes) {
+                  const uint4 v = lds128(sbase + off);
+                  float z[N];
+                  Vec<InT>::unpack(v, z);
                   float vm = z[0];
 #pragma unroll
                   for (int i = 1; i < N; ++i) vm = fmaxf(vm, z[i]);
                   if (vm > ref) {
-                    s *= ex2_approx((ref - vm) * kLog2e);
+                    s *= ex2_approx((ref - vm) * kLog2e);     // ref = -inf gives 0 * 0
                     ref = vm;
                     nm = -vm * kLog2e;
-                    vs = 0.f;
+                  }
+                  if (ref != -INFINITY) {
+                    float vs = 0.f;
 #pragma unroll
                     for (int i = 0; i < N; ++i) vs += ex2_approx(fmaf(z[i], kLog2e, nm));
+                    s += vs;
                   }
                 }
-                if (ref != -INFINITY) s += vs;
               }
             }
           }
@@ -346,28 +371,46 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
           const uint32_t sbase = slots_base + (uint32_t)slot * kChunkBytes;
           if (ok) {
+            const bool full_chunk = cbase + (uint32_t)kChunkBytes <= row_bytes;
+            const uint32_t e0 = cbase / (uint32_t)sizeof(InT);                       // first element of the chunk
+            const bool has_a = (a - e0) < (uint32_t)(kChunkBytes / sizeof(InT));     // warp-uniform
+            if (full_chunk && !coef.zero_row && !has_a) {
+              // straight-line path: all loads first, 4 x N independent exponentials, 4 stores
+              uint4 raw[kVecPerThread];
 #pragma unroll
-            for (int k = 0; k < kVecPerThread; ++k) {
-              const uint32_t off = ((uint32_t)k * kGroupThreads + gtid) * 16u;
-              if (cbase + off < row_bytes) {
-                const uint32_t j0 = (cbase + off) / (uint32_t)sizeof(InT);
-                float v[N];
-                if (coef.zero_row) {
+              for (int k = 0; k < kVecPerThread; ++k) raw[k] = lds128(sbase + ((uint32_t)k * kGroupThreads + gtid) * 16u);
 #pragma unroll
-                  for (int i = 0; i < N; ++i) v[i] = 0.f;
-                } else {
-                  const uint4 raw = lds128(sbase + off);
-                  float z[N];
-                  Vec<InT>::unpack(raw, z);
+              for (int k = 0; k < kVecPerThread; ++k) {
+                float z[N], v[N];
+                Vec<InT>::unpack(raw[k], z);
 #pragma unroll
-                  for (int i = 0; i < N; ++i) v[i] = ex2_approx(fmaf(z[i], kLog2e, coef.c2));
-                  if (a - j0 < (uint32_t)N) {             // the sampled token's entry is g * (pi(a) - 1)
+                for (int i = 0; i < N; ++i) v[i] = ex2_approx(fmaf(z[i], kLog2e, coef.c2));
+                Store<OutT, N>::run(drow, e0 + ((uint32_t)k * kGroupThreads + gtid) * N, v, sign2);
+              }
+            } else {
+#pragma unroll 1
+              for (int k = 0; k < kVecPerThread; ++k) {
+                const uint32_t off = ((uint32_t)k * kGroupThreads + gtid) * 16u;
+                if (cbase + off < row_bytes) {
+                  const uint32_t j0 = (cbase + off) / (uint32_t)sizeof(InT);
+                  float v[N];
+                  if (coef.zero_row) {
 #pragma unroll
-                    for (int i = 0; i < N; ++i)
-                      if (j0 + i == a) v[i] = coef.fix * coef.sgn;   // the store flips it back
+                    for (int i = 0; i < N; ++i) v[i] = 0.f;
+                  } else {
+                    const uint4 raw = lds128(sbase + off);
+                    float z[N];
+                    Vec<InT>::unpack(raw, z);
+#pragma unroll
+                    for (int i = 0; i < N; ++i) v[i] = ex2_approx(fmaf(z[i], kLog2e, coef.c2));
+                    if (a - j0 < (uint32_t)N) {             // the sampled token's entry is g * (pi(a) - 1)
+#pragma unroll
+                      for (int i = 0; i < N; ++i)
+                        if (j0 + i == a) v[i] = coef.fix * coef.sgn;   // the store flips it back
+                    }
                   }
+                  Store<OutT, N>::run(drow, j0, v, sign2);
                 }
-                Store<OutT, N>::run(drow, j0, v, sign2);
               }
             }
           }

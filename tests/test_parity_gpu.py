@@ -239,7 +239,10 @@ def test_host_buffer_entry_matches_device_entry(qwen_rows):
                                       rows_per_chunk=100, want_dlogits=True, device=DEV)
     assert out["status"] == 0
     assert torch.equal(out["divergence"], dev["divergence"].cpu()) and torch.equal(out["mask"], dev["mask"].cpu())
-    assert torch.equal(out["dlogits"], dev["dlogits"].cpu())
+    # same kernels on the same rows; only the scale differs in its last fp32 bit, which may move an
+    # occasional gradient entry to the neighbouring bf16 value
+    a_, b_ = out["dlogits"].float(), dev["dlogits"].cpu().float()
+    assert torch.all((a_ - b_).abs() <= 2.0 ** -7 * b_.abs()) and (a_ != b_).float().mean() < 1e-2
     # the host entry passes the token-mean scale as an fp32 argument and adds the chunks' partial losses
     assert abs(out["loss"] - float(dev["loss"].item())) <= 1e-4 * abs(out["loss"]) + 1e-12
 
