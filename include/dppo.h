@@ -67,7 +67,8 @@ enum {
   DPPO_ERR_WORKSPACE = -8,   /* workspace NULL, misaligned or smaller than dppo_workspace_bytes */
   DPPO_ERR_ALIAS = -9,       /* dlogits aliases logits but the element sizes differ          */
   DPPO_ERR_CUDA = -10,       /* a CUDA runtime call failed (launch, copy)                    */
-  DPPO_ERR_UNSUPPORTED = -11 /* combination not implemented                                  */
+  DPPO_ERR_UNSUPPORTED = -11, /* combination not implemented                                 */
+  DPPO_ERR_TOO_MANY_ROWS = -12 /* T above DPPO_STATIC_WS_MAX_ROWS (dppo_loss_fwd_bwd_static_ws)  */
 };
 
 /* Bits OR-ed into *status by the device. */
@@ -157,6 +158,39 @@ int dppo_loss_fwd_bwd_host(const void* logits, int64_t T, int64_t V, int logits_
                            float* loss_host, float* divergence_host, uint8_t* mask_host,
                            void* dlogits_host, int32_t* status_host,
                            void* staging, size_t staging_bytes, int64_t rows_per_chunk);
+
+/*
+ * dppo_loss_fwd_bwd for callers that cannot allocate device memory.  (The paper has no counterpart
+ * to this entry point; it exists for integration only.)
+ *
+ * Who needs it: code that runs where every byte of device memory already belongs to someone else,
+ * for instance a trainer whose framework allocator claimed the whole GPU at start-up, so that a
+ * cudaMalloc for the scratch may fail, or a step loop that must not call cudaMalloc / cudaFree
+ * because those calls stall the whole device.  Such a caller still owns its inputs and outputs, but
+ * has nowhere to get the `workspace` of dppo_loss_fwd_bwd from.
+ *
+ * Here the scratch is a fixed array inside the library image (256 + 12 * DPPO_STATIC_WS_MAX_ROWS
+ * bytes, about 0.75 MiB), present on every GPU that loads the library until the process exits.
+ * The call allocates nothing and frees nothing.  All other arguments, results, status bits and
+ * error codes are those of dppo_loss_fwd_bwd, with these differences:
+ *   - T may not exceed DPPO_STATIC_WS_MAX_ROWS; a larger T returns DPPO_ERR_TOO_MANY_ROWS and
+ *     launches nothing (split the batch and pass opts->loss_scale, as for micro-batches).
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array.  Nothing in it needs clearing: each call
+ *     rewrites what it reads, and what the previous call left behind is ignored.  Two calls
+ *     whose kernels can overlap on the GPU (different streams, no dependency) race on it and give
+ *     undefined results; keep such calls on one stream or order them with events.
+ */
+#define DPPO_STATIC_WS_MAX_ROWS 65536
+int dppo_loss_fwd_bwd_static_ws(const void* logits, int64_t T, int64_t V, int64_t logits_row_stride, int logits_dtype,
+                                const int32_t* sampled_ids, const float* mu_logp,
+                                const int32_t* mu_topk_ids, const float* mu_topk_p,
+                                const float* advantages, const uint8_t* token_mask,
+                                int variant, int K, float delta, const dppo_opts* opts,
+                                float* loss, float* divergence, uint8_t* mask,
+                                void* dlogits, int64_t dlogits_row_stride,
+                                float* stats, int32_t* status, void* cuda_stream);
 
 /* Name of an error code (static string, never NULL). */
 const char* dppo_error_string(int code);

@@ -58,6 +58,8 @@ def lib():
                                              c_void_p, c_void_p, c_int, c_int, c_float, POINTER(DppoOpts),
                                              c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                              c_void_p, c_size_t, c_int64]
+        L.dppo_loss_fwd_bwd_static_ws.restype = c_int
+        L.dppo_loss_fwd_bwd_static_ws.argtypes = L.dppo_loss_fwd_bwd.argtypes[:22] + [c_void_p]
         _lib = L
     return _lib
 
@@ -125,6 +127,42 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
     if rc != 0:
         raise DppoError(rc, "dppo_loss_fwd_bwd")
     return dict(loss=loss, divergence=D, mask=M, dlogits=dlogits, stats=stats, status=status)
+
+
+STATIC_WS_MAX_ROWS = 65536
+
+
+def dppo_loss_fwd_bwd_static_ws(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, K=0,
+                                delta=0.2, mu_topk_ids=None, mu_topk_p=None, loss_scale=0.0, dlogits_f32=False,
+                                kernel=KERNEL_AUTO, out=None, stream=None):
+    """Calls ``dppo_loss_fwd_bwd_static_ws``: the same operation with the scratch taken from the array
+    built into the library, for callers that cannot allocate device memory.  This wrapper does not
+    allocate either when ``out`` holds the output tensors (loss[1], divergence[T], mask[T],
+    dlogits[T,V], status[1], optionally stats[8]); without ``out`` it creates them with torch for
+    convenience.  At most ``STATIC_WS_MAX_ROWS`` rows per call; calls that may overlap on the GPU race on
+    the shared array."""
+    assert logits.is_cuda and logits.dim() == 2 and logits.stride(1) == 1
+    T, V = logits.shape
+    dev = logits.device
+    if out is None:
+        out = dict(loss=torch.empty(1, dtype=torch.float32, device=dev),
+                   divergence=torch.empty(T, dtype=torch.float32, device=dev),
+                   mask=torch.empty(T, dtype=torch.uint8, device=dev),
+                   dlogits=torch.empty((T, V), dtype=torch.float32 if dlogits_f32 else logits.dtype, device=dev),
+                   status=torch.zeros(1, dtype=torch.int32, device=dev), stats=None)
+    dl = out["dlogits"]
+    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), 0)
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    with torch.cuda.device(dev):
+        rc = lib().dppo_loss_fwd_bwd_static_ws(_ptr(logits), T, V, logits.stride(0) if T > 0 else V, _dtype_code(logits),
+                                               _ptr(sampled_ids), _ptr(mu_logp), _ptr(mu_topk_ids), _ptr(mu_topk_p),
+                                               _ptr(advantages), _ptr(token_mask), int(variant), int(K), float(delta),
+                                               ctypes.byref(opts), _ptr(out["loss"]), _ptr(out["divergence"]),
+                                               _ptr(out["mask"]), _ptr(dl), dl.stride(0) if T > 0 else V,
+                                               _ptr(out.get("stats")), _ptr(out["status"]), c_void_p(st.cuda_stream))
+    if rc != 0:
+        raise DppoError(rc, "dppo_loss_fwd_bwd_static_ws")
+    return out
 
 
 def dppo_host_staging_bytes(rows_per_chunk, V, K, logits_dtype, dlogits_f32=False):

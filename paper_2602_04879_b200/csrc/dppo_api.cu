@@ -30,6 +30,7 @@ const char* dppo_error_string(int code) {
     case DPPO_ERR_ALIAS: return "dlogits aliases logits with a different element size or stride";
     case DPPO_ERR_CUDA: return "CUDA runtime error";
     case DPPO_ERR_UNSUPPORTED: return "combination not implemented";
+    case DPPO_ERR_TOO_MANY_ROWS: return "T exceeds DPPO_STATIC_WS_MAX_ROWS of the built-in scratch array";
     default: return "unknown error code";
   }
 }

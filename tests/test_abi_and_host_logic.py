@@ -38,11 +38,11 @@ def test_every_declared_symbol_is_exported(binding):
 
 def test_error_strings(binding):
     seen = set()
-    for code in range(0, -12, -1):
+    for code in range(0, -13, -1):
         s = binding.error_string(code)
         assert s and s != "unknown error code"
         seen.add(s)
-    assert len(seen) == 12
+    assert len(seen) == 13
     assert binding.error_string(-99) == "unknown error code"
 
 
