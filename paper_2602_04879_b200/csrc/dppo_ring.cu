@@ -1,21 +1,21 @@
-// Row kernel for 16-byte aligned layouts: one persistent CTA per SM streams token rows through a
-// ring of shared-memory slots filled by bulk asynchronous copies (TMA, cp.async.bulk) and runs a
-// four-role pipeline connected only by mbarriers:
+// Row kernel for 16-byte aligned layouts: one persistent CTA per SM walks the token rows
+// blockIdx.x, blockIdx.x + gridDim.x, ... with two independent streams of bulk asynchronous copies
+// (TMA, cp.async.bulk) through two rings of shared-memory slots, connected only by mbarriers:
 //
-//   producer warp   issues the bulk copies of the rows' chunks, slot by slot, as slots are released
-//   sum warps (8)   sweep 1: consume the chunks of row n+1 as they land, sum of exponentials against
-//                   a per-thread reference (moved up only if a vector would overflow), hand the
-//                   per-warp partials to the scalar warp
-//   scalar warp     log-sum-exp, ratio, divergence, mask, loss term of the row; posts the gradient
-//                   coefficients
-//   grad warps (8)  sweep 2 of row n: read the chunks that are still resident in the ring, write
-//                   the gradient with 128-bit streaming stores, release the slots
+//   sum stream    producer warp S copies the chunks of row n+k from global memory (first touch: HBM,
+//                 L2 evict-last hint); 8 sum warps add up exp(z - ref) against a per-thread reference
+//                 (moved up only if a chunk would overflow) and hand per-warp partials to the scalar warp
+//   scalar warp   log-sum-exp, ratio, divergence, mask, loss term of the row; posts the gradient
+//                 coefficients
+//   grad stream   producer warp G copies the chunks of row n a second time (they were read a few
+//                 microseconds earlier by the sum stream and normally still sit in L2; evict-first
+//                 hint); 8 grad warps write the gradient with 128-bit streaming stores
 //
-// The last `nslots` chunks of a row stay resident between the sweeps; only the head of a row that
-// is longer than the ring is fetched a second time (it was loaded with an L2 evict-last hint and
-// normally still sits in L2).  A row that fits in the ring is read from HBM exactly once.  Because
-// the sum warps work one row ahead of the grad warps, the scalar stage and the waits of one group
-// are covered by the arithmetic of the other.
+// Neither stream has to keep a row resident in shared memory, so both run as plain pipelines with
+// several chunks in flight; the sum stream leads the grad stream by at most about two rows
+// (depth of the coefficient hand-off), which bounds the L2 footprint of rows waiting for their
+// second read to roughly 2 x 148 rows.  HBM traffic stays one read and one write of the tensor as
+// long as those rows survive in L2.
 //
 // Every wait is bounded: a wait that runs out sets a shared abort flag and the status bit
 // DPPO_STATUS_WAIT_LIMIT; from then on every warp skips its remaining work and returns.
@@ -27,14 +27,14 @@ constexpr int kChunkBytes = 16384;
 constexpr int kGroupThreads = 256;              // threads of the sum group and of the grad group
 constexpr int kGroupWarps = kGroupThreads / 32;
 constexpr int kVecPerThread = kChunkBytes / 16 / kGroupThreads;   // 16-byte vectors per thread per chunk
-constexpr int kRingThreads = 2 * kGroupThreads + 64;              // + scalar warp + producer warp
+constexpr int kRingThreads = 2 * kGroupThreads + 96;              // + scalar warp + two producer warps
 constexpr int kMiscBytes = 1024;                // barriers + hand-off buffers
-constexpr int kMaxSlots = 14;
+constexpr int kMaxSlots = 14;                   // both rings together
 static_assert(kVecPerThread * kGroupThreads * 16 == kChunkBytes, "chunk geometry");
 
 struct RingMisc {
-  unsigned long long full[kMaxSlots];    // chunk landed            (producer -> sum, grad)
-  unsigned long long empty[kMaxSlots];   // chunk no longer needed  (sum or grad -> producer)
+  unsigned long long full[kMaxSlots];    // chunk landed            (producer -> consumers of that ring)
+  unsigned long long empty[kMaxSlots];   // chunk consumed          (consumers -> producer)
   unsigned long long part_full[2];       // partials of a row ready (sum -> scalar)
   unsigned long long part_empty[2];
   unsigned long long coef_full[2];       // coefficients of a row ready (scalar -> grad)
@@ -42,6 +42,7 @@ struct RingMisc {
   float2 part[2][kGroupWarps];           // (reference, sum of exp) per sum warp
   RowCoef coef[2];
   int abort_flag;
+  unsigned int grad_chunks;              // chunks the grad warps have finished (written by one lane)
 };
 static_assert(sizeof(RingMisc) <= kMiscBytes, "misc area");
 
@@ -153,12 +154,11 @@ template <> struct Store<float, 4> {
   }
 };
 
-struct RingPos {             // position in the endless sequence of slot uses
+struct RingPos {             // position in the endless sequence of slot uses of one ring
   int slot;
   uint32_t phase;
-  __device__ __forceinline__ void advance(int nslots, int n = 1) {
-    slot += n;
-    while (slot >= nslots) { slot -= nslots; phase ^= 1u; }
+  __device__ __forceinline__ void advance(int nslots) {
+    if (++slot == nslots) { slot = 0; phase ^= 1u; }
   }
 };
 
@@ -169,6 +169,49 @@ __device__ __forceinline__ int load_meta(const RowParams& p, int64_t t) {
   if (p.token_mask && p.token_mask[t] == 0) return -1;
   const int a = p.sampled_ids[t];
   return (a < 0 || (int64_t)a >= p.V) ? -2 : a;
+}
+
+// One producer lane: copies every chunk of every valid row of this CTA into the ring
+// [first_slot, first_slot + nslots), in order, as slots are released.
+template <typename InT>
+__device__ __forceinline__ void produce_stream(const RowParams& p, uint32_t slots_base, uint32_t full_base, uint32_t empty_base,
+                                               int first_slot, int nslots, uint32_t row_bytes, int C, uint64_t policy,
+                                               volatile int* abort_flag, volatile unsigned int* follow, unsigned int lead) {
+  const char* logits = reinterpret_cast<const char*>(p.logits);
+  const int64_t t0 = blockIdx.x, G = gridDim.x;
+  RingPos pos{0, 0};
+  bool first_lap = true;
+  unsigned int issued = 0;
+  int meta = load_meta(p, t0);
+  for (int64_t t = t0; t < p.T; t += G) {
+    const int meta_next = load_meta(p, t + G);
+    if (meta >= 0) {
+      const char* row = logits + t * p.ld_in * (int64_t)sizeof(InT);
+      for (int c = 0; c < C; ++c) {
+        const int slot = first_slot + pos.slot;
+        if (follow) {                      // stay at most `lead` chunks ahead of the stream we feed L2 for
+          if (issued - *follow >= lead) {
+            const unsigned long long w0 = globaltimer_ns();
+            while (issued - *follow >= lead) {
+              if (*abort_flag) return;
+              if (globaltimer_ns() - w0 > 2000000000ull) { *abort_flag = 1; return; }
+              __nanosleep(64);
+            }
+          }
+          ++issued;
+        }
+        // lap u >= 1 of a slot needs its (u-1)-th release: parity (u-1)&1 = phase^1
+        if (!first_lap && !mbar_wait(empty_base + 8u * slot, pos.phase ^ 1u, abort_flag)) return;
+        const uint32_t off = (uint32_t)c * kChunkBytes;
+        const uint32_t bytes = (row_bytes - off) < (uint32_t)kChunkBytes ? (row_bytes - off) : (uint32_t)kChunkBytes;
+        const uint32_t bar = full_base + 8u * slot;
+        mbar_arrive_expect_tx(bar, bytes);
+        bulk_load(slots_base + (uint32_t)slot * kChunkBytes, row + off, bytes, bar, policy);
+        if (++pos.slot == nslots) { pos.slot = 0; pos.phase ^= 1u; first_lap = false; }
+      }
+    }
+    meta = meta_next;
+  }
 }
 
 template <typename InT, typename OutT>
@@ -183,6 +226,9 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
   const uint32_t coef_full = smem_u32(&misc->coef_full[0]), coef_empty = smem_u32(&misc->coef_empty[0]);
   volatile int* abort_flag = &misc->abort_flag;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // slots [0, ns_sum) feed the sum warps, [ns_sum, nslots) the grad warps; the second read comes from L2 with a
+  // shorter latency but is issued as early as possible, so the grad ring gets the larger share (4 + 10 of 14)
+  const int ns_sum = (2 * nslots + 3) / 7 < 2 ? 2 : (2 * nslots + 3) / 7, ns_grad = nslots - ns_sum;
 
   if (tid == 0) {
     for (int i = 0; i < nslots; ++i) {
@@ -196,6 +242,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
       mbar_init(coef_empty + 8u * i, kGroupWarps);
     }
     misc->abort_flag = 0;
+    misc->grad_chunks = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -203,37 +250,24 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
 
   const uint32_t row_bytes = (uint32_t)(p.V * (int64_t)sizeof(InT));     // launcher guarantees < 2^31
   const int C = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);      // chunks per row
-  const int L = C > nslots ? C - nslots : 0;                             // head chunks fetched twice
   const int64_t t0 = blockIdx.x, G = gridDim.x;
 
-  if (warp == 2 * kGroupWarps + 1) {
-    // ------------------------------------------------------------------ producer (one lane)
+  if (warp >= 2 * kGroupWarps + 1) {
+    // ------------------------------------------------------------------ producers (one lane each)
     if (lane == 0) {
-      uint64_t pol_keep, pol_stream;
-      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-      const char* logits = reinterpret_cast<const char*>(p.logits);
-      RingPos pos{0, 0};
-      bool first_lap = true, ok = true;
-      int meta = load_meta(p, t0);
-      for (int64_t t = t0; t < p.T && ok; t += G) {
-        const int meta_next = load_meta(p, t + G);
-        if (meta >= 0) {
-          const char* row = logits + t * p.ld_in * (int64_t)sizeof(InT);
-          for (int i = 0; i < C + L; ++i) {
-            const int c = (i < C) ? i : i - C;
-            // lap u >= 1 of a slot needs its (u-1)-th release: parity (u-1)&1 = phase^1
-            if (!first_lap && !mbar_wait(empty_base + 8u * pos.slot, pos.phase ^ 1u, abort_flag)) { ok = false; break; }
-            const uint32_t off = (uint32_t)c * kChunkBytes;
-            const uint32_t bytes = (row_bytes - off) < (uint32_t)kChunkBytes ? (row_bytes - off) : (uint32_t)kChunkBytes;
-            const uint32_t bar = full_base + 8u * pos.slot;
-            mbar_arrive_expect_tx(bar, bytes);
-            bulk_load(slots_base + (uint32_t)pos.slot * kChunkBytes, row + off, bytes, bar, (i < L) ? pol_keep : pol_stream);
-            pos.slot += 1;
-            if (pos.slot == nslots) { pos.slot = 0; pos.phase ^= 1u; first_lap = false; }
-          }
-        }
-        meta = meta_next;
+      uint64_t policy;
+      if (warp == 2 * kGroupWarps + 1) {
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+        // The sum stream runs at most one row and a few chunks ahead of the grad warps (at least one row, or
+        // the grad warps could never get their coefficients).  Rows between their first and second read then
+        // occupy about #SMs x lead chunks of L2 (61 MB at V = 151936 bf16); a longer lead makes the second
+        // read miss L2, a shorter one leaves the sum warps idle.  Measured optimum on B200: C + 7.
+        const int lead = (C + 7 <= 26 || C + 2 > 26) ? ((C + 7 <= 26) ? C + 7 : C + 2) : 26;
+        produce_stream<InT>(p, slots_base, full_base, empty_base, 0, ns_sum, row_bytes, C, policy, abort_flag,
+                            &misc->grad_chunks, (unsigned int)lead);
+      } else {
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+        produce_stream<InT>(p, slots_base, full_base, empty_base, ns_sum, ns_grad, row_bytes, C, policy, abort_flag, nullptr, 0u);
       }
     }
   } else if (warp < kGroupWarps) {
@@ -246,14 +280,13 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
       const int meta_next = load_meta(p, t + G);
       if (__shfl_sync(0xffffffffu, *abort_flag, 0)) break;
       if (meta >= 0) {
-        // per-thread partial: s = sum exp(z - ref); ref is the maximum of the thread's first finite
-        // vector and moves up only when a vector's sum shows that an entry exceeds it by > 44
+        // per-thread partial: s = sum exp(z - ref); ref is the maximum of the thread's first entries
+        // and moves up only when a chunk's sum shows that an entry exceeds it by > 44
         float ref = -INFINITY, nm = 0.f, s = 0.f;
-        RingPos p1 = pos;
         for (int c = 0; c < C; ++c) {
-          const bool ok = mbar_wait_warp(full_base + 8u * p1.slot, p1.phase, abort_flag);
+          const bool ok = mbar_wait_warp(full_base + 8u * pos.slot, pos.phase, abort_flag);
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
-          const uint32_t sbase = slots_base + (uint32_t)p1.slot * kChunkBytes;
+          const uint32_t sbase = slots_base + (uint32_t)pos.slot * kChunkBytes;
           if (ok) {
             const bool full_chunk = cbase + (uint32_t)kChunkBytes <= row_bytes;
             bool done = false;
@@ -318,11 +351,9 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
               }
             }
           }
-          if (c < L) {                     // head of a long row: give the slot back, it is re-fetched for sweep 2
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_base + 8u * p1.slot);
-          }
-          p1.advance(nslots);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty_base + 8u * pos.slot);
+          pos.advance(ns_sum);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -338,8 +369,6 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
             mbar_arrive(part_full + 8u * b);
           }
         }
-        pos = p1;
-        pos.advance(nslots, L);            // the re-fetched head chunks belong to the grad warps
         ++vrow;
       }
       meta = meta_next;
@@ -350,6 +379,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
     OutT* dlogits = reinterpret_cast<OutT*>(p.dlogits);
     RingPos pos{0, 0};
     uint32_t vrow = 0;
+    unsigned int chunks_done = 0;
     int meta = load_meta(p, t0);
     for (int64_t t = t0; t < p.T; t += G) {
       const int meta_next = load_meta(p, t + G);
@@ -367,7 +397,9 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         if (!have) coef.zero_row = 1;
         const uint32_t sign2 = (coef.sgn < 0.f) ? 0x80008000u : 0u;
         const uint32_t a = (uint32_t)meta;
-        auto grad_chunk = [&](int c, int slot, bool ok) {
+        for (int c = 0; c < C; ++c) {
+          const int slot = ns_sum + pos.slot;
+          const bool ok = mbar_wait_warp(full_base + 8u * slot, pos.phase, abort_flag);
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
           const uint32_t sbase = slots_base + (uint32_t)slot * kChunkBytes;
           if (ok) {
@@ -416,20 +448,10 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(empty_base + 8u * slot);
-        };
-        RingPos p2 = pos;
-        p2.advance(nslots, L);
-        for (int c = L; c < C; ++c) {              // resident chunks: the phase is complete, the wait returns at once
-          const bool ok = mbar_wait_warp(full_base + 8u * p2.slot, p2.phase, abort_flag);
-          grad_chunk(c, p2.slot, ok);
-          p2.advance(nslots);
+          ++chunks_done;
+          if (tid == kGroupThreads) *(volatile unsigned int*)&misc->grad_chunks = chunks_done;
+          pos.advance(ns_grad);
         }
-        for (int c = 0; c < L; ++c) {              // re-fetched head of a long row
-          const bool ok = mbar_wait_warp(full_base + 8u * p2.slot, p2.phase, abort_flag);
-          grad_chunk(c, p2.slot, ok);
-          p2.advance(nslots);
-        }
-        pos = p2;                                  // = start + C + L
         ++vrow;
       }
       meta = meta_next;
