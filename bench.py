@@ -56,6 +56,22 @@ def measured_peaks():
     return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one full-size launch of the row kernel, from the ncu
+# capture summarised in profiles/dppo_row_ring_kernel_bf16_V151936.md, and the hash of the kernel sources it was
+# taken with: once the kernel changes the figure no longer applies and None is reported.
+TRAFFIC_BYTES_PER_LAUNCH = 5514331733 + 4917249707
+TRAFFIC_KERNEL_SHA = "72311896fc13c8ed"
+
+
+def measured_traffic():
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("dppo_ring.cu", "dppo_common.cuh"):
+        with open(os.path.join(ROOT, "paper_2602_04879_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return TRAFFIC_BYTES_PER_LAUNCH if h.hexdigest()[:16] == TRAFFIC_KERNEL_SHA else None
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU from a thread (NVML) while the GPU works."""
 
@@ -228,10 +244,7 @@ def run_ours(args):
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None, "peak_source": "of " + peak_src, "kernel": "dppo_row_ring_kernel<bf16,bf16>",
                 "algorithmic_bytes_per_launch": T * BYTES_PER_TOKEN}
-    tr = os.path.join(ROOT, "profiles", "ring_traffic.json")
-    if os.path.exists(tr):
-        with open(tr) as f:
-            roofline["traffic"] = json.load(f).get("dram_bytes_per_launch_full_size")
+    roofline["traffic"] = measured_traffic()
     clocks = sampler.summary(t_host0, t_host1)
 
     line = {
