@@ -179,6 +179,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     import paper_2602_04879_b200 as dppo
+    from paper_2602_04879_b200 import parallel
     from paper_2602_04879_b200 import workloads as wl
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -195,7 +196,7 @@ def run_ours(args):
     # each rank owns T rows of the global batch of world*T rows
     b = wl.qwen_vocab_rows(dev, seed=1 + rank, rows=args.rows) if args.rows != T_ROWS else wl.qwen_vocab_rows(dev, seed=1 + rank)
     T = b.T
-    scale = 1.0 / (T * world)
+    scale = parallel.global_loss_scale(T, device=dev)        # one all-reduce of N_valid, before the timed region
     dlogits = torch.empty_like(b.logits)
     ws = torch.empty(dppo.dppo_workspace_bytes(T), dtype=torch.uint8, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -228,9 +229,7 @@ def run_ours(args):
         t = torch.tensor([ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
-        loss_t = out["loss"].clone()
-        dist.all_reduce(loss_t)                     # global loss = sum of the shards' losses
-        loss_val = float(loss_t.item())
+        loss_val = float(parallel.reduce_loss(out["loss"]).item())   # global loss = sum of the shards' losses
     else:
         loss_val = float(out["loss"].item())
     assert int(status.item()) == 0, f"device status {int(status.item())}"
