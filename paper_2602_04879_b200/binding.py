@@ -58,6 +58,15 @@ def lib():
                                              c_void_p, c_void_p, c_int, c_int, c_float, POINTER(DppoOpts),
                                              c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                              c_void_p, c_size_t, c_int64]
+        L.dppo_fused_workspace_bytes.restype = c_size_t
+        L.dppo_fused_workspace_bytes.argtypes = [c_int64, c_int64, c_int64]
+        L.dppo_fused_lmhead_fwd_bwd.restype = c_int
+        L.dppo_fused_lmhead_fwd_bwd.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
+                                                c_void_p, c_int, c_float, POINTER(DppoOpts), c_void_p, c_void_p, c_void_p,
+                                                c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.dppo_gemm_tn_bf16.restype = c_int
+        L.dppo_gemm_tn_bf16.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_int, c_int, c_int, c_void_p, c_int64,
+                                        c_void_p, c_void_p]
         L.dppo_loss_fwd_bwd_static_ws.restype = c_int
         L.dppo_loss_fwd_bwd_static_ws.argtypes = L.dppo_loss_fwd_bwd.argtypes[:22] + [c_void_p]
         _lib = L
@@ -127,6 +136,62 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
     if rc != 0:
         raise DppoError(rc, "dppo_loss_fwd_bwd")
     return dict(loss=loss, divergence=D, mask=M, dlogits=dlogits, stats=stats, status=status)
+
+
+def dppo_fused_workspace_bytes(T, d, V):
+    return int(lib().dppo_fused_workspace_bytes(int(T), int(d), int(V)))
+
+
+def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, delta=0.2,
+                              loss_scale=0.0, want_stats=False, workspace=None, dHidden=None, dW=None, status=None, stream=None):
+    """Calls ``dppo_fused_lmhead_fwd_bwd`` on CUDA tensors: hidden [T,d] bf16, W [d,V] bf16.  Returns
+    dict(loss[1], divergence[T], mask[T], dHidden[T,d] fp32, dW[d,V] fp32, stats, status); nothing is synchronised."""
+    assert hidden.is_cuda and W.is_cuda and hidden.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
+    assert hidden.is_contiguous() and W.is_contiguous() and hidden.shape[1] == W.shape[0]
+    T, d = hidden.shape
+    V = W.shape[1]
+    dev = hidden.device
+    loss = torch.empty(1, dtype=torch.float32, device=dev)
+    D = torch.empty(T, dtype=torch.float32, device=dev)
+    M = torch.empty(T, dtype=torch.uint8, device=dev)
+    if dHidden is None:
+        dHidden = torch.empty((T, d), dtype=torch.float32, device=dev)
+    if dW is None:
+        dW = torch.empty((d, V), dtype=torch.float32, device=dev)
+    stats = torch.empty(8, dtype=torch.float32, device=dev) if want_stats else None
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(dppo_fused_workspace_bytes(T, d, V), dtype=torch.uint8, device=dev)
+    opts = DppoOpts(float(loss_scale), 0, 0, 0)
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    with torch.cuda.device(dev):
+        rc = lib().dppo_fused_lmhead_fwd_bwd(_ptr(hidden), _ptr(W), T, d, V, _ptr(sampled_ids), _ptr(mu_logp), _ptr(advantages),
+                                             _ptr(token_mask), int(variant), float(delta), ctypes.byref(opts), _ptr(loss),
+                                             _ptr(D), _ptr(M), _ptr(dHidden), _ptr(dW), _ptr(stats), _ptr(status),
+                                             _ptr(workspace), workspace.numel(), c_void_p(st.cuda_stream))
+    if rc != 0:
+        raise DppoError(rc, "dppo_fused_lmhead_fwd_bwd")
+    return dict(loss=loss, divergence=D, mask=M, dHidden=dHidden, dW=dW, stats=stats, status=status)
+
+
+def dppo_gemm_tn_bf16(A, B, C=None, status=None, stream=None):
+    """C[M,N] fp32 = A[M,K] . B[N,K]^T for bf16 CUDA matrices (last dimension contiguous)."""
+    assert A.is_cuda and B.is_cuda and A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16
+    assert A.stride(1) == 1 and B.stride(1) == 1 and A.shape[1] == B.shape[1]
+    M, K = A.shape
+    N = B.shape[0]
+    if C is None:
+        C = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=A.device)
+    st = stream if stream is not None else torch.cuda.current_stream(A.device)
+    with torch.cuda.device(A.device):
+        rc = lib().dppo_gemm_tn_bf16(_ptr(A), A.stride(0), _ptr(B), B.stride(0), M, N, K, _ptr(C), C.stride(0), _ptr(status),
+                                     c_void_p(st.cuda_stream))
+    if rc != 0:
+        raise DppoError(rc, "dppo_gemm_tn_bf16")
+    return C, status
 
 
 STATIC_WS_MAX_ROWS = 65536

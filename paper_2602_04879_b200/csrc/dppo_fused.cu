@@ -1,0 +1,272 @@
+// Fused LM-head variant of the DPPO loss: logits = hidden x W are produced tile by tile on the tensor cores and
+// consumed in the accumulators' epilogue, so the [T, V] logits never exist in memory.
+//
+//   1. W^T, hidden^T  (bf16 transposes: every GEMM below then has both operands K-major)
+//   2. stats GEMM     z-tile = hidden . W^T-tile; epilogue: per-row (max, sum exp) of the tile, z at the sampled id
+//   3. scalar kernel  merge the tiles' partials -> lse; ratio, divergence, mask, loss term, gradient coefficients
+//   4. grad GEMM      the same tiles again; epilogue: P = dlogits = g (softmax - onehot) in bf16
+//   5. P^T            (bf16 transpose)
+//   6. dHidden = P . W     (A = P [T,V], B = W [d,V])          fp32
+//   7. dW = hidden^T . P   (A = hidden^T [d,T], B = P^T [V,T])  fp32
+//
+// dHidden and dW are d = thousands of columns wide, far more than the 512 accumulator columns of tensor memory, so they
+// cannot be accumulated on chip across the vocabulary; the bf16 gradient P (not the logits) is therefore staged in the
+// caller's workspace between steps 4 and 6/7.
+#include <mutex>
+
+#include "dppo_common.cuh"
+#include "dppo_gemm.cuh"
+
+namespace dppo {
+
+namespace {
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode() {
+  static EncodeFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeFn>(ptr);
+  });
+  return fn;
+}
+
+// Tensor map of a row-major bf16 matrix [rows, cols] (cols contiguous, leading dimension ld elements) with boxes of
+// 64 columns x box_rows rows and the 128-byte swizzle the MMA descriptors expect.  Out-of-range elements read as 0.
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+  EncodeFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)gemm::BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int EPI>
+cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
+  if (p.M <= 0 || p.N <= 0 || p.K <= 0) return cudaSuccess;
+  CUtensorMap ma, mb;
+  if (!make_map(&ma, A, p.M, p.K, lda, gemm::BM) || !make_map(&mb, B, p.N, p.K, ldb, gemm::BN)) return cudaErrorInvalidValue;
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaError_t e = cudaFuncSetAttribute(gemm::gemm_tn_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  const int64_t ntiles = (int64_t)((p.M + gemm::BM - 1) / gemm::BM) * ((p.N + gemm::BN - 1) / gemm::BN);
+  const int grid = (int)(ntiles < sms ? ntiles : sms);
+  gemm::gemm_tn_kernel<EPI><<<grid, gemm::THREADS, gemm::SMEM_BYTES, st>>>(ma, mb, p);
+  return cudaGetLastError();
+}
+
+// out[c, r] = in[r, c] for bf16 matrices; 64 x 64 tiles through shared memory.
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* in, int64_t rows, int64_t cols, int64_t ld_in,
+                                                             __nv_bfloat16* out, int64_t ld_out) {
+  __shared__ __nv_bfloat16 tile[64][66];
+  const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+  for (int i = ty; i < 64; i += 4) {
+    const int64_t r = r0 + i, c = c0 + tx;
+    tile[i][tx] = (r < rows && c < cols) ? in[r * ld_in + c] : __float2bfloat16(0.f);
+  }
+  __syncthreads();
+  for (int i = ty; i < 64; i += 4) {
+    const int64_t c = c0 + i, r = r0 + tx;
+    if (c < cols && r < rows) out[c * ld_out + r] = tile[tx][i];
+  }
+}
+
+cudaError_t transpose_bf16(const void* in, int64_t rows, int64_t cols, int64_t ld_in, void* out, int64_t ld_out, cudaStream_t st) {
+  if (rows <= 0 || cols <= 0) return cudaSuccess;
+  dim3 grid((unsigned)((cols + 63) / 64), (unsigned)((rows + 63) / 64));
+  transpose_bf16_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(in), rows, cols, ld_in,
+                                              reinterpret_cast<__nv_bfloat16*>(out), ld_out);
+  return cudaGetLastError();
+}
+
+// One warp per row: merge the stats GEMM's per-tile partials, then the same scalar stage as the streaming kernels.
+__global__ void __launch_bounds__(256) fused_scalar_kernel(RowParams p, const float2* part, int tiles_n, const float* z_a,
+                                                           float* c2, float* sgn, float* fix) {
+  const int lane = threadIdx.x & 31;
+  const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= p.T) return;
+  const double scale = p.hdr->scale;
+  bool valid = p.token_mask ? (p.token_mask[t] != 0) : true;
+  int flags = 0;
+  const int a = p.sampled_ids[t];
+  if (valid && (a < 0 || (int64_t)a >= p.V)) { valid = false; flags = DPPO_STATUS_BAD_SAMPLED_ID; }
+  float D = 0.f, r = 0.f, absdiff = 0.f;
+  int M = 0;
+  double g = 0.0;
+  RowCoef coef;
+  coef.c2 = 0.f; coef.sgn = 0.f; coef.fix = 0.f; coef.zero_row = 1;
+  if (valid) {
+    float mm = -INFINITY;
+    for (int i = lane; i < tiles_n; i += 32) mm = fmaxf(mm, part[t * tiles_n + i].x);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
+    double S = 0.0;
+    for (int i = lane; i < tiles_n; i += 32) {
+      const float2 pr = part[t * tiles_n + i];
+      if (pr.y > 0.f || pr.y != pr.y) S += (double)pr.y * exp((double)pr.x - (double)mm);
+    }
+    S = warp_sum(S);
+    const double lse = (double)mm + log(S);
+    if (!isfinite(lse)) {
+      flags |= DPPO_STATUS_NONFINITE_ROW;
+    } else {
+      double pi_a;
+      int f2 = 0;
+      const float za = z_a[t];
+      auto z_at = [&](int) { return za; };          // Binary variants only touch the sampled id
+      row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
+      coef = make_coef(g, lse, pi_a);
+    }
+  }
+  if (lane == 0) {
+    p.divergence[t] = D;
+    p.mask[t] = (uint8_t)M;
+    p.row_loss[t] = (float)(-g);
+    p.row_r[t] = r;
+    p.row_absdiff[t] = absdiff;
+    c2[t] = coef.c2;
+    sgn[t] = coef.zero_row ? 0.f : coef.sgn;
+    fix[t] = coef.fix;
+    if (flags) atomicOr(p.status, flags);
+  }
+}
+
+constexpr size_t kAlign = 256;
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct FusedLayout {
+  size_t wt, ht, P, Pt, part, z_a, c2, sgn, fix, loss_ws, total;
+  int64_t ldp, ldt;
+  int tiles_n;
+};
+FusedLayout fused_layout(int64_t T, int64_t d, int64_t V) {
+  FusedLayout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += round_up(bytes ? bytes : 1, kAlign); return o; };
+  L.ldp = (V + 7) / 8 * 8;
+  L.ldt = (T + 7) / 8 * 8;
+  L.tiles_n = (int)((V + gemm::BN - 1) / gemm::BN);
+  L.wt = take((size_t)V * d * 2);
+  L.ht = take((size_t)d * L.ldt * 2);
+  L.P = take((size_t)T * L.ldp * 2);
+  L.Pt = take((size_t)V * L.ldt * 2);
+  L.part = take((size_t)T * L.tiles_n * sizeof(float2));
+  L.z_a = take((size_t)T * 4);
+  L.c2 = take((size_t)T * 4);
+  L.sgn = take((size_t)T * 4);
+  L.fix = take((size_t)T * 4);
+  L.loss_ws = take(dppo_workspace_bytes(T));
+  L.total = off;
+  return L;
+}
+
+}  // namespace
+}  // namespace dppo
+
+extern "C" {
+
+size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V) {
+  if (T < 0 || d < 1 || V < 1) return 0;
+  return dppo::fused_layout(T, d, V).total;
+}
+
+int dppo_gemm_tn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,
+                      int32_t* status, void* cuda_stream) {
+  if (M < 0 || N < 0 || K < 0) return DPPO_ERR_SHAPE;
+  if (M == 0 || N == 0) return DPPO_OK;
+  if (!A || !B || !C) return DPPO_ERR_NULL;
+  if (lda < K || ldb < K || ldc < N) return DPPO_ERR_STRIDE;
+  if (((uintptr_t)A % 16) || ((uintptr_t)B % 16) || (lda % 8) || (ldb % 8) || ((uintptr_t)C % 4)) return DPPO_ERR_ALIGN;
+  dppo::gemm::Params p = {};
+  p.M = M; p.N = N; p.K = K; p.C = C; p.ldc = ldc; p.status = status;
+  return dppo::launch_gemm<dppo::gemm::EPI_STORE_F32>(A, lda, B, ldb, p, reinterpret_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? DPPO_OK : DPPO_ERR_CUDA;
+}
+
+int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int64_t d, int64_t V,
+                              const int32_t* sampled_ids, const float* mu_logp, const float* advantages,
+                              const uint8_t* token_mask, int variant, float delta, const dppo_opts* opts,
+                              float* loss, float* divergence, uint8_t* mask, float* dHidden, float* dW,
+                              float* stats, int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  using namespace dppo;
+  dppo_opts o = {};
+  if (opts) o = *opts;
+  if (T < 0 || d < 1 || V < 1 || T > (int64_t)1 << 30 || V > (int64_t)1 << 30 || d > (int64_t)1 << 30) return DPPO_ERR_SHAPE;
+  if (variant != DPPO_BINARY_TV && variant != DPPO_BINARY_KL) return DPPO_ERR_VARIANT;
+  if (!loss || !status || !W || !dW) return DPPO_ERR_NULL;
+  if (T > 0 && (!hidden || !sampled_ids || !mu_logp || !advantages || !divergence || !mask || !dHidden)) return DPPO_ERR_NULL;
+  if (((uintptr_t)hidden % 16) || ((uintptr_t)W % 16) || (d % 8) || (V % 8)) return DPPO_ERR_ALIGN;
+  if (((uintptr_t)dHidden % 16) || ((uintptr_t)dW % 16)) return DPPO_ERR_ALIGN;
+  const FusedLayout L = fused_layout(T, d, V);
+  if (!workspace || ((uintptr_t)workspace % kAlign) || workspace_bytes < L.total) return DPPO_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  char* ws = reinterpret_cast<char*>(workspace);
+
+  RowParams p = {};
+  p.T = T; p.V = V; p.sampled_ids = sampled_ids; p.mu_logp = mu_logp; p.adv = advantages; p.token_mask = token_mask;
+  p.variant = variant; p.K = 0; p.delta = delta; p.loss_scale = o.loss_scale;
+  p.divergence = divergence; p.mask = mask; p.loss = loss; p.stats = stats; p.status = status;
+  char* lws = ws + L.loss_ws;
+  const size_t per = round_up((size_t)T * sizeof(float), kAlign);
+  p.hdr = reinterpret_cast<WsHeader*>(lws);
+  p.row_loss = reinterpret_cast<float*>(lws + kAlign);
+  p.row_r = reinterpret_cast<float*>(lws + kAlign + per);
+  p.row_absdiff = reinterpret_cast<float*>(lws + kAlign + 2 * per);
+
+#define DPPO_TRY(call) do { if ((call) != cudaSuccess) return DPPO_ERR_CUDA; } while (0)
+  DPPO_TRY(launch_prelude(p, st));
+  // dW is written by a GEMM whose K dimension is T: with no rows it is all zero
+  if (T == 0) {
+    DPPO_TRY(cudaMemsetAsync(dW, 0, (size_t)d * V * sizeof(float), st));
+    DPPO_TRY(launch_finalize(p, st));
+    return DPPO_OK;
+  }
+  float2* part = reinterpret_cast<float2*>(ws + L.part);
+  float *z_a = reinterpret_cast<float*>(ws + L.z_a), *c2 = reinterpret_cast<float*>(ws + L.c2);
+  float *sgn = reinterpret_cast<float*>(ws + L.sgn), *fix = reinterpret_cast<float*>(ws + L.fix);
+  // 1. transposes of the operands
+  DPPO_TRY(transpose_bf16(W, d, V, V, ws + L.wt, d, st));
+  DPPO_TRY(transpose_bf16(hidden, T, d, d, ws + L.ht, L.ldt, st));
+  // 2. statistics of the logits
+  DPPO_TRY(cudaMemsetAsync(z_a, 0, (size_t)T * 4, st));
+  gemm::Params g1 = {};
+  g1.M = (int)T; g1.N = (int)V; g1.K = (int)d; g1.part = part; g1.z_a = z_a; g1.ids = sampled_ids; g1.status = status;
+  DPPO_TRY(launch_gemm<gemm::EPI_STATS>(hidden, d, ws + L.wt, d, g1, st));
+  // 3. per-row scalars, loss
+  fused_scalar_kernel<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(p, part, L.tiles_n, z_a, c2, sgn, fix);
+  DPPO_TRY(cudaGetLastError());
+  DPPO_TRY(launch_finalize(p, st));
+  // 4. gradient with respect to the logits, bf16, [T, ldp]
+  gemm::Params g2 = {};
+  g2.M = (int)T; g2.N = (int)V; g2.K = (int)d; g2.ids = sampled_ids; g2.c2 = c2; g2.sgn = sgn; g2.fix = fix;
+  g2.P = reinterpret_cast<__nv_bfloat16*>(ws + L.P); g2.ldp = L.ldp; g2.status = status;
+  DPPO_TRY(launch_gemm<gemm::EPI_GRAD>(hidden, d, ws + L.wt, d, g2, st));
+  // 5. P^T
+  DPPO_TRY(transpose_bf16(ws + L.P, T, V, L.ldp, ws + L.Pt, L.ldt, st));
+  // 6. dHidden[T, d] = P[T, V] . W[d, V]^T
+  gemm::Params g3 = {};
+  g3.M = (int)T; g3.N = (int)d; g3.K = (int)V; g3.C = dHidden; g3.ldc = d; g3.status = status;
+  DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(ws + L.P, L.ldp, W, V, g3, st));
+  // 7. dW[d, V] = hidden^T[d, T] . P^T[V, T]^T
+  gemm::Params g4 = {};
+  g4.M = (int)d; g4.N = (int)V; g4.K = (int)T; g4.C = dW; g4.ldc = V; g4.status = status;
+  DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(ws + L.ht, L.ldt, ws + L.Pt, L.ldt, g4, st));
+#undef DPPO_TRY
+  return DPPO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,311 @@
+// bf16 "TN" GEMM on the 5th-generation tensor cores: C[M,N] = A[M,K] * B[N,K]^T, both operands K-major
+// (row-major with K contiguous), fp32 accumulation in tensor memory, epilogue chosen at compile time.
+//
+// One persistent CTA per SM (192 threads):
+//   warp 0      TMA producer: cp.async.bulk.tensor loads of 128x64 (A) and 256x64 (B) bf16 boxes, 128-byte swizzle,
+//               into a 4-stage shared-memory ring (mbarrier complete_tx)
+//   warp 1      allocates the 512 tensor-memory columns and issues tcgen05.mma (cta_group::1, kind::f16, M=128, N=256,
+//               K=16 per instruction); tcgen05.commit releases smem stages and publishes finished accumulators
+//   warps 2-5   epilogue: tcgen05.ld of the accumulator (one row per thread, 32 columns at a time) while the MMA warp
+//               already fills the other 256-column accumulator buffer
+// Tiles are walked M-fastest so that CTAs running at the same time share B strips through L2.
+// Every mbarrier wait is bounded; on expiry the CTA raises DPPO_STATUS_WAIT_LIMIT, skips the rest and frees its TMEM.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/dppo.h"
+
+namespace dppo {
+namespace gemm {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2, B_STAGE_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int THREADS = 192;
+constexpr int TMEM_COLS = 512;
+
+enum { EPI_STORE_F32 = 0, EPI_STATS = 1, EPI_GRAD = 2 };
+
+struct Params {
+  int M, N, K;
+  // EPI_STORE_F32
+  float* C;
+  int64_t ldc;
+  // EPI_STATS: per (row, n-tile) partial (max, sum exp(z - max)); z at the sampled id
+  float2* part;          // [M, tiles_n]
+  float* z_a;            // [M]
+  const int32_t* ids;    // [M] sampled id per row (EPI_STATS, EPI_GRAD)
+  // EPI_GRAD: P[row, col] = sgn * 2^(z*log2e + c2), entry at ids[row] = fix; written as bf16
+  const float* c2;       // [M]
+  const float* sgn;      // [M] +1, -1, or 0 (zero row)
+  const float* fix;      // [M]
+  __nv_bfloat16* P;
+  int64_t ldp;
+  int32_t* status;
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void bar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool bar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait (about 2 s); false = gave up (abort flag set) or somebody else did.
+__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (bar_try(bar, parity)) return true;
+  const unsigned long long t0 = timer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (bar_try(bar, parity)) return true;
+    if ((it & 0xff) == 0) {
+      if (*abort_flag) return false;
+      if (timer_ns() - t0 > 2000000000ull) { *abort_flag = 1; return false; }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+// Shared-memory matrix descriptor: K-major tile with rows of 128 bytes, 128-byte swizzle (8-row groups 1024 bytes apart).
+__device__ __forceinline__ uint64_t make_desc_k_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);       // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                          // leading byte offset (unused with swizzle): 1
+  d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                          // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                          // layout type: 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 128.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ void mma_bf16(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,"
+      "%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                             const __grid_constant__ CUtensorMap map_b, Params p) {
+  extern __shared__ unsigned char smem_raw[];
+  // 1024-byte alignment for the 128-byte swizzle atoms
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + STAGES * STAGE_BYTES);
+  const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + STAGES);
+  const uint32_t tfull0 = smem_addr(bars + 2 * STAGES), tempty0 = smem_addr(bars + 2 * STAGES + 2);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    for (int i = 0; i < STAGES; ++i) { bar_init(full0 + 8 * i, 1); bar_init(empty0 + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { bar_init(tfull0 + 8 * i, 1); bar_init(tempty0 + 8 * i, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {   // the MMA warp owns the tensor memory
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+  const int ntiles = tiles_m * tiles_n;
+  const int kblocks = (p.K + BK - 1) / BK;
+  const uint32_t smem_base = smem_addr(smem);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!bar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t a_dst = smem_base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
+          bar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+          tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
+          tma_load_2d(b_dst, &map_b, kb * BK, n0, full0 + 8 * s);
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+        const uint32_t b = it & 1u, use = it >> 1;
+        if (!bar_wait(tempty0 + 8 * b, (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }   // epilogue drained this buffer
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t tmem_c = tmem_base + b * BN;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!bar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a_src = smem_base + s * STAGE_BYTES, b_src = a_src + A_STAGE_BYTES;
+          const uint64_t adesc = make_desc_k_sw128(a_src), bdesc = make_desc_k_sw128(b_src);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)      // 32 bytes (16 bf16) further along K inside the swizzle atom per step
+            mma_bf16(tmem_c, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), (kb | k) != 0 ? 1u : 0u);
+          mma_commit(empty0 + 8 * s);            // stage free once these MMAs have read it
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (ok) mma_commit(tfull0 + 8 * b);      // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps (TMEM lane quarter = warp % 4)
+    const int q = warp & 3;
+    uint32_t it = 0;
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
+      const int m0 = (tile % tiles_m) * BM, nb = tile / tiles_m, n0 = nb * BN;
+      const uint32_t b = it & 1u, use = it >> 1;
+      const bool ok = __all_sync(0xffffffffu, bar_wait(tfull0 + 8 * b, use & 1u, abort_flag));
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int row = m0 + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * BN;
+      if (EPI == EPI_STORE_F32) {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          if (row_ok) {
+            float* dst = p.C + (int64_t)row * p.ldc + n0 + c;
+            if (n0 + c + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) *reinterpret_cast<uint4*>(dst + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) dst[j] = __uint_as_float(r[j]);
+            }
+          }
+        }
+      } else if (EPI == EPI_STATS) {
+        const int a = row_ok ? p.ids[row] : -1;
+        float m = -INFINITY, s = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          const int col0 = n0 + c;
+          float vm = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            float z = (col0 + j < p.N) ? __uint_as_float(r[j]) : -INFINITY;
+            r[j] = __float_as_uint(z);
+            vm = fmaxf(vm, z);
+          }
+          if (vm > m) { s *= ex2((m - vm) * 1.4426950408889634f); m = vm; }
+          if (m != -INFINITY) {
+            const float nm = -m * 1.4426950408889634f;
+            float acc = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc += ex2(fmaf(__uint_as_float(r[j]), 1.4426950408889634f, nm));
+            s += acc;
+          }
+          if (a >= col0 && a < col0 + 32) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) if (col0 + j == a) p.z_a[row] = __uint_as_float(r[j]);
+          }
+        }
+        if (row_ok) p.part[(int64_t)row * tiles_n + nb] = make_float2(m, s);
+      } else {  // EPI_GRAD
+        const int a = row_ok ? p.ids[row] : -1;
+        const float c2 = row_ok ? p.c2[row] : 0.f, sg = row_ok ? p.sgn[row] : 0.f, fx = row_ok ? p.fix[row] : 0.f;
+        const uint32_t sign2 = (sg < 0.f) ? 0x80008000u : 0u;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          const int col0 = n0 + c;
+          if (row_ok && col0 < p.N) {
+            uint32_t o[16];
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              float v0 = (sg == 0.f) ? 0.f : ex2(fmaf(__uint_as_float(r[j]), 1.4426950408889634f, c2));
+              float v1 = (sg == 0.f) ? 0.f : ex2(fmaf(__uint_as_float(r[j + 1]), 1.4426950408889634f, c2));
+              if (col0 + j == a) v0 = fx * sg;          // the sign flip below restores fix
+              if (col0 + j + 1 == a) v1 = fx * sg;
+              __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+              o[j >> 1] = (*reinterpret_cast<uint32_t*>(&h)) ^ sign2;
+            }
+            __nv_bfloat16* dst = p.P + (int64_t)row * p.ldp + col0;
+            if (col0 + 32 <= p.N) {
+#pragma unroll
+              for (int j = 0; j < 16; j += 4) *reinterpret_cast<uint4*>(dst + 2 * j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+            } else {
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) dst[j] = __ushort_as_bfloat16((unsigned short)((j & 1) ? (o[j >> 1] >> 16) : (o[j >> 1] & 0xffffu)));
+            }
+          }
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) bar_arrive(tempty0 + 8 * b);
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (*abort_flag && tid == 0 && p.status) atomicOr(p.status, DPPO_STATUS_WAIT_LIMIT);
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace gemm
+}  // namespace dppo
