@@ -88,3 +88,60 @@ def test_fused_rejects_misuse():
         dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.BINARY_TV, 0.2,
                                        workspace=torch.empty(1024, dtype=torch.uint8, device=DEV))
     assert e.value.code == -8
+
+
+def test_fused_full_size_masked_subset_and_properties():
+    """The benchmark's fused configuration (T=8192, d=2048, V=151936).  (i) With a token mask that keeps 192 rows the
+    oracle can do everything: loss, mask, divergence, dHidden of the valid rows and the whole dW.  (ii) With all rows
+    valid: sampled rows against the oracle, and properties that hold at any size."""
+    T, d, V = 8192, 2048, 151936
+    b = wl.lm_head_workload(DEV, seed=5)
+    assert b.hidden.shape == (T, d) and b.lm_head.shape == (d, V)
+    ws = torch.empty(dppo.dppo_fused_workspace_bytes(T, d, V), dtype=torch.uint8, device=DEV)
+    W64 = b.lm_head.float().cpu().numpy().astype(np.float64)
+    # ---- (i) masked subset
+    g = torch.Generator().manual_seed(9)
+    keep = torch.sort(torch.randperm(T, generator=g)[:192]).values
+    tok = torch.zeros(T, dtype=torch.uint8)
+    tok[keep] = 1
+    out = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, tok.to(DEV),
+                                         dppo.BINARY_TV, 0.0, workspace=ws, want_stats=True)   # delta = 0: blocked iff moving away
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0 and out["stats"][0].item() == 192
+    idx = keep.numpy()
+    Hk = b.hidden[keep.to(DEV)].float().cpu().numpy().astype(np.float64)
+    ora = O.dppo_fused_lmhead_fwd_bwd(Hk, W64, b.sampled_ids.cpu().numpy()[idx], b.mu_logp.cpu().numpy().astype(np.float64)[idx],
+                                      b.advantages.cpu().numpy().astype(np.float64)[idx], None, O.BINARY_TV, 0.0, 1.0 / 192)
+    # the logits of this workload are nearly uniform (D ~ 1e-6), so every row is inside the 1e-6 exemption band of the
+    # divergence test; the masks are compared directly instead (the decision is the sign of log pi(a) - log mu(a))
+    P.check_scalars(out["divergence"].cpu().numpy()[idx], out["mask"].cpu().numpy()[idx], ora, dict(token_mask=None), 0.0)
+    assert np.array_equal(out["mask"].cpu().numpy()[idx], ora["M"])
+    assert 0 < int((ora["M"] == 0).sum()) < 192
+    P.check_loss(float(out["loss"].item()), ora["loss"], True, ora["row_loss"])
+    aP = np.abs(ora["dlogits"])
+    eh = np.abs(out["dHidden"][keep.to(DEV)].cpu().numpy() - ora["dHidden"])
+    assert np.all(eh <= 2.0 ** -8 * (aP @ np.abs(W64).T) + 1e-7 * np.abs(ora["dHidden"]).max())
+    ew = np.abs(out["dW"].cpu().numpy() - ora["dW"])
+    assert np.all(ew <= 2.0 ** -8 * (np.abs(Hk).T @ aP) + 1e-7 * np.abs(ora["dW"]).max())
+    assert eh.max() <= 4e-3 * np.abs(ora["dHidden"]).max() and ew.max() <= 4e-3 * np.abs(ora["dW"]).max()
+    inv = torch.nonzero(tok == 0)[:, 0][:256].to(DEV)
+    assert not out["dHidden"][inv].any() and not out["divergence"][inv].any()
+    del ora, aP, eh, ew
+    # ---- (ii) all rows valid (the benchmark's launch configuration)
+    out = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None,
+                                         dppo.BINARY_TV, 0.2, workspace=ws)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    rows = keep[:24]
+    ridx = rows.numpy()
+    Hr = b.hidden[rows.to(DEV)].float().cpu().numpy().astype(np.float64)
+    orr = O.dppo_fused_lmhead_fwd_bwd(Hr, W64, b.sampled_ids.cpu().numpy()[ridx], b.mu_logp.cpu().numpy().astype(np.float64)[ridx],
+                                      b.advantages.cpu().numpy().astype(np.float64)[ridx], None, O.BINARY_TV, 0.2, 1.0 / T)
+    P.check_scalars(out["divergence"].cpu().numpy()[ridx], out["mask"].cpu().numpy()[ridx], orr, dict(token_mask=None), 0.2)
+    eh = np.abs(out["dHidden"][rows.to(DEV)].cpu().numpy() - orr["dHidden"])
+    assert np.all(eh <= 2.0 ** -8 * (np.abs(orr["dlogits"]) @ np.abs(W64).T) + 1e-7 * np.abs(orr["dHidden"]).max())
+    # every dlogits row sums to zero, hence every row of dW does (up to the bf16 rounding of dlogits)
+    dW = out["dW"]
+    scale_w = float(dW.abs().sum(dim=1).max().item())
+    assert float(dW.sum(dim=1).abs().max().item()) <= 5e-3 * scale_w
+    assert torch.isfinite(out["dHidden"]).all() and torch.isfinite(dW).all()
