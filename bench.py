@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--variant", default="binary_tv", choices=["binary_tv", "binary_kl"])
     ap.add_argument("--rows", type=int, default=T_ROWS, help="rows per GPU; anything but the default is a reduced case for profiling, not the benchmark workload")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--fused-only", action="store_true", help="run only the fused LM-head measurement (profiling aid)")
+    ap.add_argument("--fused-rows", type=int, default=8192, help="token rows of the fused measurement; anything but 8192 is a reduced profiling case")
+    ap.add_argument("--no-fused", action="store_true", help="skip the fused LM-head measurement (reported as an extra object at N=1)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -54,6 +57,50 @@ def measured_peaks():
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def measured_tensor_peak():
+    """Sustained bf16 dense TFLOP/s (the fused step is a long back-to-back sequence of GEMMs)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json bf16_tflops_sustained)"
+    return 1400.0, "fallback (about 1.4 PFLOP/s sustained, earlier measurement on this pool)"
+
+
+def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
+    """Fused LM-head variant on its own workload: hidden [8192, 2048] x W [2048, 151936], Binary-TV, delta 0.2."""
+    import torch
+    d, V = 2048, VOCAB
+    b = wl.lm_head_workload(dev, seed=5, T=T, d=d, V=V)
+    ws = torch.empty(dppo.dppo_fused_workspace_bytes(T, d, V), dtype=torch.uint8, device=dev)
+    dH = torch.empty((T, d), dtype=torch.float32, device=dev)
+    dW = torch.empty((d, V), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step():
+        return dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None,
+                                              dppo.BINARY_TV, DELTA, workspace=ws, dHidden=dH, dW=dW, status=status)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        out = step()
+    e1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ms = e0.elapsed_time(e1) / steps
+    peak, src = measured_tensor_peak()
+    useful = 6.0 * T * d * V / (ms * 1e-3) / 1e12          # forward + dHidden + dW
+    executed = 8.0 * T * d * V / (ms * 1e-3) / 1e12        # + the recomputation of the logits tiles
+    return {"workload": ("" if T == 8192 else f"REDUCED to {T} rows (profiling case): ") + "fused_lm_head_binary_tv: hidden [8192,2048] bf16 x W [2048,151936] bf16, delta=0.2",
+            "ms_per_step": ms, "tokens_per_s": T / (ms * 1e-3), "steps": steps, "warmup": warmup,
+            "roofline": {"bound": "tensor", "achieved": useful, "peak": peak, "unit": "TFLOP/s", "frac": useful / peak,
+                         "executed_tflops": executed, "executed_frac": executed / peak, "traffic": None,
+                         "peak_source": "of " + src, "flop_count": "useful = 6*T*d*V (forward, dHidden, dW); executed = 8*T*d*V with the recomputed logits"},
+            "gpu_launches_per_step": 10, "loss": float(out["loss"].item())}
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one full-size launch of the row kernel, from the ncu
@@ -192,6 +239,9 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
     variant = dppo.BINARY_TV if args.variant == "binary_tv" else dppo.BINARY_KL
+    if args.fused_only:
+        print(json.dumps({"fused_lm_head": bench_fused(dppo, wl, dev, steps=max(1, min(args.steps, 10)), warmup=max(1, min(args.warmup, 3)), T=args.fused_rows)}))
+        return
 
     # each rank owns T rows of the global batch of world*T rows
     b = wl.qwen_vocab_rows(dev, seed=1 + rank, rows=args.rows) if args.rows != T_ROWS else wl.qwen_vocab_rows(dev, seed=1 + rank)
@@ -284,6 +334,12 @@ def run_ours(args):
                        "h2d_bytes_per_step": T * VOCAB * 2 + T * 12, "d2h_bytes_per_step": T * 5 + 8,
                        "steps": e2e_steps, "note": "dppo_loss_fwd_bwd_host: pinned host logits/ids/mu_logp/advantages in, loss + divergence + mask out; dlogits stay on the device"}
         del h, staging
+
+    if world == 1 and not args.no_fused and T == T_ROWS:
+        del dlogits
+        b.logits = None
+        torch.cuda.empty_cache()
+        line["fused_lm_head"] = bench_fused(dppo, wl, dev)
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import dppo_oracle as O

@@ -4,8 +4,8 @@
 //   1. W^T, hidden^T  (bf16 transposes: every GEMM below then has both operands K-major)
 //   2. stats GEMM     z-tile = hidden . W^T-tile; epilogue: per-row (max, sum exp) of the tile, z at the sampled id
 //   3. scalar kernel  merge the tiles' partials -> lse; ratio, divergence, mask, loss term, gradient coefficients
-//   4. grad GEMM      the same tiles again; epilogue: P = dlogits = g (softmax - onehot) in bf16
-//   5. P^T            (bf16 transpose)
+//   4. grad GEMM      the same tiles again; epilogue: P = dlogits = g (softmax - onehot) in bf16,
+//   5.                written both as P [T, V] and as P^T [V, T]
 //   6. dHidden = P . W     (A = P [T,V], B = W [d,V])          fp32
 //   7. dW = hidden^T . P   (A = hidden^T [d,T], B = P^T [V,T])  fp32
 //
@@ -68,28 +68,56 @@ cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, 
   return cudaGetLastError();
 }
 
-// out[c, r] = in[r, c] for bf16 matrices; 64 x 64 tiles through shared memory.
+// out[c, r] = in[r, c] for bf16 matrices; 64 x 64 tiles through shared memory, 16-byte global accesses when the
+// layout allows (leading dimensions multiples of 8 elements, 16-byte aligned bases), 2-byte accesses at the edges.
 __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* in, int64_t rows, int64_t cols, int64_t ld_in,
-                                                             __nv_bfloat16* out, int64_t ld_out) {
-  __shared__ __nv_bfloat16 tile[64][66];
+                                                             __nv_bfloat16* out, int64_t ld_out, int vec_ok) {
+  __shared__ unsigned short tile[64][72];                 // [r][c], row pitch 144 bytes (16-byte aligned rows)
   const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
-  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
-  for (int i = ty; i < 64; i += 4) {
-    const int64_t r = r0 + i, c = c0 + tx;
-    tile[i][tx] = (r < rows && c < cols) ? in[r * ld_in + c] : __float2bfloat16(0.f);
-  }
-  __syncthreads();
-  for (int i = ty; i < 64; i += 4) {
-    const int64_t c = c0 + i, r = r0 + tx;
-    if (c < cols && r < rows) out[c * ld_out + r] = tile[tx][i];
+  const int tid = threadIdx.x;
+  const unsigned short* src = reinterpret_cast<const unsigned short*>(in);
+  unsigned short* dst = reinterpret_cast<unsigned short*>(out);
+  const bool interior = vec_ok && r0 + 64 <= rows && c0 + 64 <= cols;
+  if (interior) {
+    // 64 rows x 8 vectors of 8 elements: thread -> (row = tid / 8 + 32 * pass, vector = tid % 8)
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass) {
+      const int r = (tid >> 3) + 32 * pass, v = tid & 7;
+      const uint4 x = *reinterpret_cast<const uint4*>(src + (r0 + r) * ld_in + c0 + v * 8);
+      *reinterpret_cast<uint4*>(&tile[r][v * 8]) = x;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass) {
+      const int c = (tid >> 3) + 32 * pass, v = tid & 7;     // output row c, 8 consecutive input rows v*8..v*8+7
+      unsigned short e[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) e[k] = tile[v * 8 + k][c];
+      uint4 x;
+      x.x = e[0] | ((uint32_t)e[1] << 16); x.y = e[2] | ((uint32_t)e[3] << 16);
+      x.z = e[4] | ((uint32_t)e[5] << 16); x.w = e[6] | ((uint32_t)e[7] << 16);
+      *reinterpret_cast<uint4*>(dst + (c0 + c) * ld_out + r0 + v * 8) = x;
+    }
+  } else {
+    const int tx = tid & 63, ty = tid >> 6;
+    for (int i = ty; i < 64; i += 4) {
+      const int64_t r = r0 + i, c = c0 + tx;
+      tile[i][tx] = (r < rows && c < cols) ? src[r * ld_in + c] : (unsigned short)0;
+    }
+    __syncthreads();
+    for (int i = ty; i < 64; i += 4) {
+      const int64_t c = c0 + i, r = r0 + tx;
+      if (c < cols && r < rows) dst[c * ld_out + r] = tile[tx][i];
+    }
   }
 }
 
 cudaError_t transpose_bf16(const void* in, int64_t rows, int64_t cols, int64_t ld_in, void* out, int64_t ld_out, cudaStream_t st) {
   if (rows <= 0 || cols <= 0) return cudaSuccess;
   dim3 grid((unsigned)((cols + 63) / 64), (unsigned)((rows + 63) / 64));
+  const int vec_ok = (ld_in % 8 == 0) && (ld_out % 8 == 0) && ((uintptr_t)in % 16 == 0) && ((uintptr_t)out % 16 == 0);
   transpose_bf16_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(in), rows, cols, ld_in,
-                                              reinterpret_cast<__nv_bfloat16*>(out), ld_out);
+                                              reinterpret_cast<__nv_bfloat16*>(out), ld_out, vec_ok);
   return cudaGetLastError();
 }
 
@@ -254,9 +282,8 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   gemm::Params g2 = {};
   g2.M = (int)T; g2.N = (int)V; g2.K = (int)d; g2.ids = sampled_ids; g2.c2 = c2; g2.sgn = sgn; g2.fix = fix;
   g2.P = reinterpret_cast<__nv_bfloat16*>(ws + L.P); g2.ldp = L.ldp; g2.status = status;
+  g2.Pt = reinterpret_cast<__nv_bfloat16*>(ws + L.Pt); g2.ldpt = L.ldt;       // 5. P^T comes out of the same epilogue
   DPPO_TRY(launch_gemm<gemm::EPI_GRAD>(hidden, d, ws + L.wt, d, g2, st));
-  // 5. P^T
-  DPPO_TRY(transpose_bf16(ws + L.P, T, V, L.ldp, ws + L.Pt, L.ldt, st));
   // 6. dHidden[T, d] = P[T, V] . W[d, V]^T
   gemm::Params g3 = {};
   g3.M = (int)T; g3.N = (int)d; g3.K = (int)V; g3.C = dHidden; g3.ldc = d; g3.status = status;

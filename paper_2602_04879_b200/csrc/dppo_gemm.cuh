@@ -46,6 +46,8 @@ struct Params {
   const float* fix;      // [M]
   __nv_bfloat16* P;
   int64_t ldp;
+  __nv_bfloat16* Pt;     // optional transposed copy [N, ldpt] (same values)
+  int64_t ldpt;
   int32_t* status;
 };
 
@@ -280,6 +282,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
               if (col0 + j + 1 == a) v1 = fx * sg;
               __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
               o[j >> 1] = (*reinterpret_cast<uint32_t*>(&h)) ^ sign2;
+            }
+            if (p.Pt) {
+              // transposed copy: for one column the 32 lanes of the warp hold 32 consecutive rows, i.e. 64 contiguous bytes
+              unsigned short* dt = reinterpret_cast<unsigned short*>(p.Pt) + (int64_t)col0 * p.ldpt + row;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) dt[(int64_t)j * p.ldpt] = (unsigned short)((j & 1) ? (o[j >> 1] >> 16) : (o[j >> 1] & 0xffffu));
             }
             __nv_bfloat16* dst = p.P + (int64_t)row * p.ldp + col0;
             if (col0 + 32 <= p.N) {
