@@ -15,7 +15,8 @@ Reinforcement Learning", DPPO):
 * ``topk_tv`` / ``topk_kl``     divergences of the reduced categoricals    (Eq. topk_tv, Eq. topk_kl).
 * ``full_tv`` / ``full_kl``     exact full-vocabulary divergences          (App. B definitions).
 * ``dppo_mask``                 asymmetric trust-region mask               (Eq. dppo_obj).
-* ``dppo_row`` / ``dppo_loss_fwd_bwd``  surrogate and its logits-gradient   (Eq. dppo_obj, Eq. unified_grad with C = inf).
+* ``dppo_row`` / ``dppo_loss_fwd_bwd``  surrogate and its logits-gradient   (Eq. dppo_obj, Eq. unified_grad; C = inf unless is_cap is given).
+* ``ppo_clip_mask``             ratio-clipping mask of the PPO / GRPO baseline (App. C.1 mask definitions; Eq. ppo-clip).
 * ``dppo_fused_lmhead_fwd_bwd`` the same applied to logits = H W with the chain rule into H and W.
 
 Readings of points the paper leaves open (each is listed in the design notes):
@@ -34,8 +35,8 @@ from __future__ import annotations
 
 import numpy as np
 
-BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL = 0, 1, 2, 3
-VARIANT_NAMES = {BINARY_TV: "binary_tv", BINARY_KL: "binary_kl", TOPK_TV: "topk_tv", TOPK_KL: "topk_kl"}
+BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL, PPO_CLIP = 0, 1, 2, 3, 4
+VARIANT_NAMES = {BINARY_TV: "binary_tv", BINARY_KL: "binary_kl", TOPK_TV: "topk_tv", TOPK_KL: "topk_kl", PPO_CLIP: "ppo_clip"}
 
 
 def _f64(x):
@@ -145,6 +146,14 @@ def dppo_mask(adv, log_pi_a, mu_logp, D, delta):
     return 0 if (away and float(D) > float(delta)) else 1
 
 
+def ppo_clip_mask(adv, r, eps_low, eps_high):
+    """App. C.1, GRPO mask: M = 0 iff (A > 0 and r > 1 + eps_high) or (A < 0 and r < 1 - eps_low); else 1.
+    It is the set where the clipped objective of Eq. ppo-clip has zero gradient."""
+    adv, r = float(adv), float(r)
+    blocked = (adv > 0.0 and r - 1.0 > float(eps_high)) or (adv < 0.0 and 1.0 - r > float(eps_low))
+    return 0 if blocked else 1
+
+
 def divergence(variant, pi, a, mu_logp, topk_ids=None, topk_p=None):
     """D_t of one row for the chosen approximation, given pi[V] (float64 probabilities)."""
     mu_a = float(np.exp(float(mu_logp)))
@@ -161,22 +170,30 @@ def divergence(variant, pi, a, mu_logp, topk_ids=None, topk_p=None):
     raise ValueError(f"unknown variant {variant}")
 
 
-def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=None, want_grad=True):
+def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=None, want_grad=True,
+             is_cap=None, eps_low=None):
     """All per-token quantities of one valid row.
 
-    Returns a dict: lse, log_pi_a, r, D, M, loss (= -s*M*r*A), g (= s*M*r*A) and,
-    if want_grad, dlogits[V] = g * (pi - onehot(a)): the derivative of the loss
-    term with M held constant (Eq. unified_grad with C = inf; d log pi(a)/dz_j =
-    1[j=a] - pi_j).
+    Returns a dict: lse, log_pi_a, r, D, M, loss (= -s*M*w*A), g (= s*M*w*A) with the weight
+    w = min(r, C) of Eq. unified_grad (C = is_cap; None or inf: w = r, which is Eq. dppo_obj) and,
+    if want_grad, dlogits[V] = g * (pi - onehot(a)): Eq. unified_grad, i.e. the derivative of the
+    loss term with M and the truncated weight held constant (d log pi(a)/dz_j = 1[j=a] - pi_j).
+    variant PPO_CLIP: D = |r - 1| and the mask is ppo_clip_mask with eps_high = delta and eps_low
+    (default: delta), the baseline the paper compares against.
     """
     log_pi, lse = log_softmax_row(z)
     pi = np.exp(log_pi)
     a = int(a)
     log_pi_a = float(log_pi[a])
     r = ratio(log_pi_a, mu_logp)
-    D = divergence(variant, pi, a, mu_logp, topk_ids, topk_p)
-    M = dppo_mask(adv, log_pi_a, mu_logp, D, delta)
-    g = float(scale) * M * r * float(adv)
+    if variant == PPO_CLIP:
+        D = abs(r - 1.0)
+        M = ppo_clip_mask(adv, r, delta if eps_low is None else eps_low, delta)
+    else:
+        D = divergence(variant, pi, a, mu_logp, topk_ids, topk_p)
+        M = dppo_mask(adv, log_pi_a, mu_logp, D, delta)
+    w = r if (is_cap is None or not np.isfinite(is_cap) or is_cap <= 0) else min(r, float(is_cap))
+    g = float(scale) * M * w * float(adv)
     out = dict(lse=float(lse), log_pi_a=log_pi_a, r=r, D=D, M=M, loss=-g, g=g)
     if want_grad:
         d = g * pi
@@ -192,7 +209,8 @@ def default_scale(T, token_mask):
 
 
 def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV,
-                      K=0, delta=0.2, loss_scale=None, mu_topk_ids=None, mu_topk_p=None, want_grad=True):
+                      K=0, delta=0.2, loss_scale=None, mu_topk_ids=None, mu_topk_p=None, want_grad=True,
+                      is_cap=None, eps_low=None):
     """The whole path over T rows (Eq. dppo_obj summed over tokens, as a loss to minimise).
 
     logits [T,V]; sampled_ids, mu_logp, advantages [T]; token_mask [T] or None;
@@ -214,7 +232,8 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
         ids = ps = None
         if variant in (TOPK_TV, TOPK_KL) and K > 0:
             ids, ps = mu_topk_ids[t][:K], mu_topk_p[t][:K]
-        o = dppo_row(logits[t], sampled_ids[t], mu_logp[t], advantages[t], variant, delta, s, ids, ps, want_grad)
+        o = dppo_row(logits[t], sampled_ids[t], mu_logp[t], advantages[t], variant, delta, s, ids, ps, want_grad,
+                     is_cap, eps_low)
         D[t], M[t], r[t], row_loss[t] = o["D"], o["M"], o["r"], o["loss"]
         if want_grad:
             dl[t] = o["dlogits"]

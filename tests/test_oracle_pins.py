@@ -389,7 +389,60 @@ def check_fused(O):
     assert abs(fd - o["dW"][0, 4]) < 2e-8
 
 
-CHECKS = [check_worked_example, check_log_softmax, check_binary, check_topk_full_and_bounds,
+def check_is_cap_and_baselines(O):
+    """Eq. unified_grad: weight min(r, C); C = inf is Eq. dppo_obj; delta = inf gives the unmasked PG-IS / CISPO baselines."""
+    rng = np.random.default_rng(9)
+    T, V = 12, 9
+    c = _case(rng, T=T, V=V, K=3, noise=1.2)
+    base = O.dppo_loss_fwd_bwd(c["z"], c["a"], c["mu_logp"], c["adv"], None, O.BINARY_TV, 0, 0.05)
+    same = O.dppo_loss_fwd_bwd(c["z"], c["a"], c["mu_logp"], c["adv"], None, O.BINARY_TV, 0, 0.05, is_cap=float("inf"))
+    assert np.array_equal(base["dlogits"], same["dlogits"]) and base["loss"] == same["loss"]
+    C = float(np.median(base["r"]))
+    cap = O.dppo_loss_fwd_bwd(c["z"], c["a"], c["mu_logp"], c["adv"], None, O.BINARY_TV, 0, 0.05, is_cap=C)
+    assert np.array_equal(cap["M"], base["M"]) and 0 < (base["r"] > C).sum() < T
+    for t in range(T):
+        f = min(1.0, C / base["r"][t])
+        np.testing.assert_allclose(cap["dlogits"][t], f * base["dlogits"][t], rtol=1e-13, atol=1e-18)
+        assert abs(cap["row_loss"][t] - f * base["row_loss"][t]) <= 1e-15
+    # the gradient is that of -s M stopgrad(min(r, C)) A log pi(a)  (autograd, float64)
+    s_ = 1.0 / T
+    zt = torch.tensor(c["z"], dtype=torch.float64, requires_grad=True)
+    lp = torch.log_softmax(zt, dim=1)[torch.arange(T), torch.tensor(c["a"])]
+    w = torch.clamp(torch.exp(lp - torch.tensor(c["mu_logp"])), max=C).detach()
+    (-(s_ * torch.tensor(cap["M"].astype(np.float64)) * w * torch.tensor(c["adv"]) * lp).sum()).backward()
+    np.testing.assert_allclose(cap["dlogits"], zt.grad.numpy(), atol=1e-14)
+    # PG-IS (no mask): delta = +inf
+    pg = O.dppo_loss_fwd_bwd(c["z"], c["a"], c["mu_logp"], c["adv"], None, O.BINARY_KL, 0, float("inf"), is_cap=3.0)
+    assert np.all(pg["M"] == 1)
+
+
+def check_ppo_clip_variant(O):
+    """App. C.1: the GRPO / PPO mask is where the clipped objective of Eq. ppo-clip has zero gradient; with
+    eps_low = eps_high = delta it is the DPPO mask with D replaced by |r - 1|."""
+    for adv in (-1.3, 0.0, 0.7):
+        for r in (0.5, 0.79, 0.81, 0.99, 1.0, 1.01, 1.27, 1.29, 2.5):
+            rt = torch.tensor(r, dtype=torch.float64, requires_grad=True)
+            obj = torch.minimum(rt * adv, torch.clamp(rt, 1 - 0.2, 1 + 0.28) * adv)
+            (gr,) = torch.autograd.grad(obj, rt)
+            M = O.ppo_clip_mask(adv, r, 0.2, 0.28)
+            if adv != 0.0:
+                assert (float(gr) == 0.0) == (M == 0), (adv, r)
+            else:
+                assert M == 1
+            assert O.ppo_clip_mask(adv, r, 0.2, 0.2) == O.dppo_mask(adv, math.log(r), 0.0, abs(r - 1.0), 0.2)
+    rng = np.random.default_rng(10)
+    c = _case(rng, T=40, V=6, K=2, noise=1.0)
+    o = O.dppo_loss_fwd_bwd(c["z"], c["a"], c["mu_logp"], c["adv"], None, O.PPO_CLIP, 0, 0.28, eps_low=0.2)
+    np.testing.assert_allclose(o["D"], np.abs(o["r"] - 1.0), atol=1e-15)
+    exp_M = [O.ppo_clip_mask(c["adv"][t], o["r"][t], 0.2, 0.28) for t in range(40)]
+    assert np.array_equal(o["M"], np.array(exp_M)) and 0 < sum(exp_M) < 40
+    # the low-probability token of the worked example (Sec. 4.2) is clipped by PPO for A > 0 but not by Binary-TV
+    z = np.log([1e-2, 0.495, 0.495])
+    assert O.dppo_row(z, 0, math.log(1e-4), 1.0, O.PPO_CLIP, 0.2, 1.0)["M"] == 0
+    assert O.dppo_row(z, 0, math.log(1e-4), 1.0, O.BINARY_TV, 0.2, 1.0)["M"] == 1
+
+
+CHECKS = [check_is_cap_and_baselines, check_ppo_clip_variant, check_worked_example, check_log_softmax, check_binary, check_topk_full_and_bounds,
           check_topk_other_bucket, check_topk_equality_conditions, check_edge_conventions,
           check_mask_truth_table, check_on_policy, check_gradient, check_brute_force_tiny, check_fused]
 
@@ -472,9 +525,25 @@ def _fused_transposed(m):
     return f
 
 
-MUTANTS.update({"topk_no_dedupe": _no_dedupe, "grad_sign": _grad_sign, "grad_no_onehot": _grad_no_onehot,
+def _cap_as_max(m):
+    orig = m.dppo_row
+
+    def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=None, want_grad=True, is_cap=None, eps_low=None):
+        o = orig(z, a, mu_logp, adv, variant, delta, scale, topk_ids, topk_p, want_grad, None, eps_low)
+        if is_cap is not None and np.isfinite(is_cap):
+            f = max(o["r"], is_cap) / o["r"]
+            o["g"] *= f
+            o["loss"] *= f
+            if "dlogits" in o:
+                o["dlogits"] = o["dlogits"] * f
+        return o
+    return dppo_row
+
+
+MUTANTS.update({"cap_as_max": _cap_as_max, "ppo_eps_swapped": lambda m: (lambda adv, r, el, eh: 0 if ((adv > 0 and r - 1 > el) or (adv < 0 and 1 - r > eh)) else 1),
+                "topk_no_dedupe": _no_dedupe, "grad_sign": _grad_sign, "grad_no_onehot": _grad_no_onehot,
                 "fused_scaled": _fused_transposed})
-MUTANT_TARGET.update({"topk_no_dedupe": "topk_reduced", "grad_sign": "dppo_row", "grad_no_onehot": "dppo_row",
+MUTANT_TARGET.update({"cap_as_max": "dppo_row", "ppo_eps_swapped": "ppo_clip_mask", "topk_no_dedupe": "topk_reduced", "grad_sign": "dppo_row", "grad_no_onehot": "dppo_row",
                       "fused_scaled": "dppo_fused_lmhead_fwd_bwd"})
 
 
