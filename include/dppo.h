@@ -46,7 +46,10 @@ extern "C" {
 #endif
 
 /* Divergence approximations (Sec. 4.4: Binary and Top-K approximation). */
-enum { DPPO_BINARY_TV = 0, DPPO_BINARY_KL = 1, DPPO_TOPK_TV = 2, DPPO_TOPK_KL = 3 };
+enum { DPPO_BINARY_TV = 0, DPPO_BINARY_KL = 1, DPPO_TOPK_TV = 2, DPPO_TOPK_KL = 3,
+       /* baseline the paper compares against: D_t = |r_t - 1| with the PPO / GRPO ratio-clip mask (App. C.1):
+          M_t = 0 iff (A > 0 and r - 1 > delta) or (A < 0 and 1 - r > eps_low); delta plays eps_high */
+       DPPO_PPO_CLIP = 4 };
 /* Element types of the logits / dlogits tensors. */
 enum { DPPO_F32 = 0, DPPO_BF16 = 1 };
 /* opts->dlogits_dtype */
@@ -86,7 +89,10 @@ typedef struct dppo_opts {
   int dlogits_dtype;   /* DPPO_DLOGITS_SAME: dlogits has the logits dtype; DPPO_DLOGITS_F32      */
   int kernel;          /* DPPO_KERNEL_AUTO picks the shared-memory ring kernel when the layout
                           allows 16-byte bulk copies and the scalar kernel otherwise            */
-  int reserved;
+  float is_cap;        /* C of Eq. unified_grad: the importance weight in loss and gradient is min(r_t, C);
+                          <= 0 or +inf: no truncation (Eq. dppo_obj).  The paper's scaling runs use C = 5,
+                          CISPO / PG-TIS is C = 3 with delta = +inf (no mask)                            */
+  float eps_low;       /* DPPO_PPO_CLIP only: lower clip range; <= 0: same as delta                      */
 } dppo_opts;
 
 /* Bytes of device scratch dppo_loss_fwd_bwd needs for T rows (256-byte aligned
@@ -109,7 +115,8 @@ size_t dppo_workspace_bytes(int64_t T);
  *                  a member and exp(mu_logp) otherwise.
  *  advantages      [T] per-token advantage A_t.
  *  token_mask      [T] bytes, non-zero = valid row; NULL = all rows valid.
- *  variant, K, delta   divergence approximation, list width, threshold (mask test is D_t > delta).
+ *  variant, K, delta   divergence approximation, list width, threshold (mask test is D_t > delta).  delta = +inf
+ *                  disables the mask (the PG-IS / CISPO baselines of App. C.1).
  *  opts            NULL = defaults.
  *  loss            [1]  out: -s * sum_t M_t r_t A_t.
  *  divergence      [T]  out: D_t (0 for invalid rows; +inf possible for KL when pi puts zero mass
@@ -203,7 +210,7 @@ size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V);
  *
  *  hidden   [T, d] bf16 row-major;  W  [d, V] bf16 row-major (LM head);  d and V multiples of 8, 16-byte aligned.
  *  sampled_ids, mu_logp, advantages, token_mask, delta, opts, loss, divergence, mask, stats, status: as for
- *           dppo_loss_fwd_bwd.  variant: DPPO_BINARY_TV or DPPO_BINARY_KL (others: DPPO_ERR_VARIANT).
+ *           dppo_loss_fwd_bwd.  variant: DPPO_BINARY_TV, DPPO_BINARY_KL or DPPO_PPO_CLIP (Top-K: DPPO_ERR_VARIANT).
  *  dHidden  [T, d] fp32 out: d loss / d hidden = dlogits . W^T.
  *  dW       [d, V] fp32 out: d loss / d W = hidden^T . dlogits (overwritten, not accumulated).
  *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V) bytes; it holds W^T, hidden^T, the

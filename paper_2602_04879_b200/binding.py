@@ -13,19 +13,19 @@ from ctypes import POINTER, c_char_p, c_float, c_int, c_int32, c_int64, c_size_t
 
 import torch
 
-BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL = 0, 1, 2, 3
+BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL, PPO_CLIP = 0, 1, 2, 3, 4
 F32, BF16 = 0, 1
 DLOGITS_SAME, DLOGITS_F32 = 0, 1
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_RING = 0, 1, 2
 STATUS_BAD_SAMPLED_ID, STATUS_BAD_TOPK_ID, STATUS_NONFINITE_ROW, STATUS_WAIT_LIMIT = 1, 2, 4, 8
-VARIANTS = {"binary_tv": BINARY_TV, "binary_kl": BINARY_KL, "topk_tv": TOPK_TV, "topk_kl": TOPK_KL}
+VARIANTS = {"binary_tv": BINARY_TV, "binary_kl": BINARY_KL, "topk_tv": TOPK_TV, "topk_kl": TOPK_KL, "ppo_clip": PPO_CLIP}
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdppo.so")
 _lib = None
 
 
 class DppoOpts(ctypes.Structure):
-    _fields_ = [("loss_scale", c_float), ("dlogits_dtype", c_int), ("kernel", c_int), ("reserved", c_int)]
+    _fields_ = [("loss_scale", c_float), ("dlogits_dtype", c_int), ("kernel", c_int), ("is_cap", c_float), ("eps_low", c_float)]
 
 
 class DppoError(RuntimeError):
@@ -99,7 +99,7 @@ def dppo_workspace_bytes(T):
 
 def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, K=0, delta=0.2,
                       mu_topk_ids=None, mu_topk_p=None, loss_scale=0.0, dlogits_f32=False, kernel=KERNEL_AUTO,
-                      dlogits=None, want_stats=False, workspace=None, status=None, stream=None):
+                      dlogits=None, want_stats=False, workspace=None, status=None, stream=None, is_cap=0.0, eps_low=0.0):
     """Calls ``dppo_loss_fwd_bwd`` on CUDA tensors.  Output tensors are allocated with torch unless
     given.  Returns dict(loss[1], divergence[T], mask[T], dlogits[T,V], stats[8] or None, status[1]);
     nothing is synchronised."""
@@ -124,7 +124,7 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
                         ("mu_topk_ids", mu_topk_ids, torch.int32), ("mu_topk_p", mu_topk_p, torch.float32)):
         if t is not None:
             assert t.is_cuda and t.dtype == dt and t.is_contiguous(), name
-    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), 0)
+    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), float(is_cap), float(eps_low))
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     with torch.cuda.device(dev):
         rc = lib().dppo_loss_fwd_bwd(_ptr(logits), T, V, logits.stride(0) if T > 0 else V, _dtype_code(logits),
@@ -143,7 +143,8 @@ def dppo_fused_workspace_bytes(T, d, V):
 
 
 def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, delta=0.2,
-                              loss_scale=0.0, want_stats=False, workspace=None, dHidden=None, dW=None, status=None, stream=None):
+                              loss_scale=0.0, want_stats=False, workspace=None, dHidden=None, dW=None, status=None, stream=None,
+                              is_cap=0.0, eps_low=0.0):
     """Calls ``dppo_fused_lmhead_fwd_bwd`` on CUDA tensors: hidden [T,d] bf16, W [d,V] bf16.  Returns
     dict(loss[1], divergence[T], mask[T], dHidden[T,d] fp32, dW[d,V] fp32, stats, status); nothing is synchronised."""
     assert hidden.is_cuda and W.is_cuda and hidden.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
@@ -163,7 +164,7 @@ def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token
         status = torch.zeros(1, dtype=torch.int32, device=dev)
     if workspace is None:
         workspace = torch.empty(dppo_fused_workspace_bytes(T, d, V), dtype=torch.uint8, device=dev)
-    opts = DppoOpts(float(loss_scale), 0, 0, 0)
+    opts = DppoOpts(float(loss_scale), 0, 0, float(is_cap), float(eps_low))
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     with torch.cuda.device(dev):
         rc = lib().dppo_fused_lmhead_fwd_bwd(_ptr(hidden), _ptr(W), T, d, V, _ptr(sampled_ids), _ptr(mu_logp), _ptr(advantages),
@@ -216,7 +217,7 @@ def dppo_loss_fwd_bwd_static_ws(logits, sampled_ids, mu_logp, advantages, token_
                    dlogits=torch.empty((T, V), dtype=torch.float32 if dlogits_f32 else logits.dtype, device=dev),
                    status=torch.zeros(1, dtype=torch.int32, device=dev), stats=None)
     dl = out["dlogits"]
-    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), 0)
+    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), 0.0, 0.0)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     with torch.cuda.device(dev):
         rc = lib().dppo_loss_fwd_bwd_static_ws(_ptr(logits), T, V, logits.stride(0) if T > 0 else V, _dtype_code(logits),
@@ -261,7 +262,7 @@ def dppo_loss_fwd_bwd_host(logits, sampled_ids, mu_logp, advantages, token_mask=
             dl = torch.empty((T, V), dtype=torch.float32 if dlogits_f32 else logits.dtype).pin_memory()
     loss = c_float(0.0)
     status = c_int32(0)
-    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), 0)
+    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), 0.0, 0.0)
     with torch.cuda.device(staging.device):
         rc = lib().dppo_loss_fwd_bwd_host(_ptr(logits), T, V, dt, _ptr(sampled_ids), _ptr(mu_logp), _ptr(mu_topk_ids),
                                           _ptr(mu_topk_p), _ptr(advantages), _ptr(token_mask), int(variant), int(K),

@@ -54,7 +54,7 @@ int dppo_loss_fwd_bwd(const void* logits, int64_t T, int64_t V, int64_t logits_r
   if (T < 0 || V < 1 || K < 0 || (int64_t)K > V) return DPPO_ERR_SHAPE;
   if (logits_dtype != DPPO_F32 && logits_dtype != DPPO_BF16) return DPPO_ERR_DTYPE;
   if (o.dlogits_dtype != DPPO_DLOGITS_SAME && o.dlogits_dtype != DPPO_DLOGITS_F32) return DPPO_ERR_DTYPE;
-  if (variant < DPPO_BINARY_TV || variant > DPPO_TOPK_KL) return DPPO_ERR_VARIANT;
+  if (variant < DPPO_BINARY_TV || variant > DPPO_PPO_CLIP) return DPPO_ERR_VARIANT;
   if (o.kernel < DPPO_KERNEL_AUTO || o.kernel > DPPO_KERNEL_RING) return DPPO_ERR_UNSUPPORTED;
   if (!loss || !status) return DPPO_ERR_NULL;
   if (T > 0 && (!logits || !sampled_ids || !mu_logp || !advantages || !divergence || !mask || !dlogits)) return DPPO_ERR_NULL;
@@ -71,7 +71,7 @@ int dppo_loss_fwd_bwd(const void* logits, int64_t T, int64_t V, int64_t logits_r
   p.logits = logits; p.T = T; p.V = V; p.ld_in = logits_row_stride;
   p.sampled_ids = sampled_ids; p.mu_logp = mu_logp; p.topk_ids = mu_topk_ids; p.topk_p = mu_topk_p;
   p.adv = advantages; p.token_mask = token_mask;
-  p.variant = variant; p.K = K; p.delta = delta; p.loss_scale = o.loss_scale;
+  p.variant = variant; p.K = K; p.delta = delta; p.loss_scale = o.loss_scale; p.is_cap = o.is_cap; p.eps_low = o.eps_low;
   p.dlogits = dlogits; p.ld_out = dlogits_row_stride;
   p.divergence = divergence; p.mask = mask; p.loss = loss; p.stats = stats; p.status = status;
   char* ws = reinterpret_cast<char*>(workspace);
@@ -142,7 +142,7 @@ int dppo_loss_fwd_bwd_host(const void* logits, int64_t T, int64_t V, int logits_
   if (T < 0 || V < 1 || K < 0 || (int64_t)K > V || rows_per_chunk < 1) return DPPO_ERR_SHAPE;
   if (logits_dtype != DPPO_F32 && logits_dtype != DPPO_BF16) return DPPO_ERR_DTYPE;
   if (o.dlogits_dtype != DPPO_DLOGITS_SAME && o.dlogits_dtype != DPPO_DLOGITS_F32) return DPPO_ERR_DTYPE;
-  if (variant < DPPO_BINARY_TV || variant > DPPO_TOPK_KL) return DPPO_ERR_VARIANT;
+  if (variant < DPPO_BINARY_TV || variant > DPPO_PPO_CLIP) return DPPO_ERR_VARIANT;
   if (!loss_host || !status_host) return DPPO_ERR_NULL;
   if (T > 0 && (!logits || !sampled_ids || !mu_logp || !advantages || !divergence_host || !mask_host)) return DPPO_ERR_NULL;
   const bool topk = (variant == DPPO_TOPK_TV || variant == DPPO_TOPK_KL);

@@ -34,6 +34,8 @@ struct RowParams {
   int variant, K;
   float delta;
   float loss_scale;          // > 0: caller's s
+  float is_cap;              // C of Eq. unified_grad (<= 0 or inf: none)
+  float eps_low;             // lower clip range of DPPO_PPO_CLIP (<= 0: delta)
   void* dlogits;
   int64_t ld_out;
   float* divergence;
@@ -105,7 +107,12 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
   const double mu_a = exp(mu_logp);
   const double r = exp(lpa - mu_logp);                // Eq. ppo-clip
   double D;
-  if (p.variant == DPPO_BINARY_TV) {
+  bool ppo_blocked = false;
+  if (p.variant == DPPO_PPO_CLIP) {                   // baseline: ratio clipping (App. C.1), D reported as |r - 1|
+    D = fabs(r - 1.0);
+    const double eh = (double)p.delta, el = (p.eps_low > 0.f) ? (double)p.eps_low : (double)p.delta;
+    ppo_blocked = (adv > 0.0 && r - 1.0 > eh) || (adv < 0.0 && 1.0 - r > el);
+  } else if (p.variant == DPPO_BINARY_TV) {
     D = fabs(mu_a - pi_a);                            // Eq. binary_tv
   } else if (p.variant == DPPO_BINARY_KL) {           // Eq. binary_kl
     double first = (mu_a > 0.0) ? mu_a * (mu_logp - lpa) : 0.0;
@@ -150,10 +157,12 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
   }
   // Eq. dppo_obj: blocked iff D > delta and the ratio already left 1 on the side the advantage pushes.
   const bool away = (adv > 0.0 && lpa > mu_logp) || (adv < 0.0 && lpa < mu_logp);
-  const int M = (away && D > (double)p.delta) ? 0 : 1;
+  const int M = (p.variant == DPPO_PPO_CLIP) ? (ppo_blocked ? 0 : 1) : ((away && D > (double)p.delta) ? 0 : 1);
+  // Eq. unified_grad: the importance weight in loss and gradient is min(r, C)
+  const double w = (p.is_cap > 0.f && isfinite(p.is_cap)) ? fmin(r, (double)p.is_cap) : r;
   D_out = (float)D;
   M_out = M;
-  g_out = scale * (double)M * r * adv;
+  g_out = scale * (double)M * w * adv;
   r_out = (float)r;
   absdiff_out = (float)fabs(mu_a - pi_a);
   pi_a_out = pi_a;

@@ -234,7 +234,7 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   dppo_opts o = {};
   if (opts) o = *opts;
   if (T < 0 || d < 1 || V < 1 || T > (int64_t)1 << 30 || V > (int64_t)1 << 30 || d > (int64_t)1 << 30) return DPPO_ERR_SHAPE;
-  if (variant != DPPO_BINARY_TV && variant != DPPO_BINARY_KL) return DPPO_ERR_VARIANT;
+  if (variant != DPPO_BINARY_TV && variant != DPPO_BINARY_KL && variant != DPPO_PPO_CLIP) return DPPO_ERR_VARIANT;
   if (!loss || !status || !W || !dW) return DPPO_ERR_NULL;
   if (T > 0 && (!hidden || !sampled_ids || !mu_logp || !advantages || !divergence || !mask || !dHidden)) return DPPO_ERR_NULL;
   if (((uintptr_t)hidden % 16) || ((uintptr_t)W % 16) || (d % 8) || (V % 8)) return DPPO_ERR_ALIGN;
@@ -246,7 +246,7 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
 
   RowParams p = {};
   p.T = T; p.V = V; p.sampled_ids = sampled_ids; p.mu_logp = mu_logp; p.adv = advantages; p.token_mask = token_mask;
-  p.variant = variant; p.K = 0; p.delta = delta; p.loss_scale = o.loss_scale;
+  p.variant = variant; p.K = 0; p.delta = delta; p.loss_scale = o.loss_scale; p.is_cap = o.is_cap; p.eps_low = o.eps_low;
   p.divergence = divergence; p.mask = mask; p.loss = loss; p.stats = stats; p.status = status;
   char* lws = ws + L.loss_ws;
   const size_t per = round_up((size_t)T * sizeof(float), kAlign);

@@ -45,9 +45,9 @@ def host_inputs(batch, rows=None):
     )
 
 
-def run_oracle(h, variant, K, delta, scale, want_grad=True):
+def run_oracle(h, variant, K, delta, scale, want_grad=True, is_cap=None, eps_low=None):
     return O.dppo_loss_fwd_bwd(h["logits"], h["sampled_ids"], h["mu_logp"], h["advantages"], h["token_mask"],
-                               variant, K, delta, scale, h["mu_topk_ids"], h["mu_topk_p"], want_grad)
+                               variant, K, delta, scale, h["mu_topk_ids"], h["mu_topk_p"], want_grad, is_cap, eps_low)
 
 
 def bf16_round(x):
@@ -59,7 +59,7 @@ def bf16_ulp(x):
     return 2.0 ** (np.floor(np.log2(ax)) - 7)
 
 
-def check_scalars(gpu_D, gpu_M, ora, h, delta, variant_is_topk=False):
+def check_scalars(gpu_D, gpu_M, ora, h, delta, variant_is_topk=False, eps_low=None):
     """Mask / divergence parity on the rows of `ora`.  Returns the number of exempted rows."""
     gpu_D = np.asarray(gpu_D, dtype=np.float64)
     gpu_M = np.asarray(gpu_M)
@@ -73,6 +73,8 @@ def check_scalars(gpu_D, gpu_M, ora, h, delta, variant_is_topk=False):
     valid = np.ones_like(oM, dtype=bool) if h["token_mask"] is None else (h["token_mask"] != 0)
     log_r = np.log(np.where(ora["r"] > 0, ora["r"], 1.0))
     exempt = valid & ((np.abs(oD - delta) <= MASK_BAND) | (np.abs(log_r) <= MASK_BAND))
+    if eps_low is not None:
+        exempt |= valid & (np.abs(oD - eps_low) <= MASK_BAND)
     bad = diff & ~exempt
     assert not bad.any(), f"mask differs on rows {np.nonzero(bad)[0][:10]} (D={oD[bad][:5]}, delta={delta})"
     return int(exempt.sum()), float(err.max() if err.size else 0.0)

@@ -79,10 +79,10 @@ def test_misuse_is_rejected_before_launch(binding):
     assert _call(B, variant=2, K=65, tk_ids=1 << 8, tk_p=1 << 9) == -2
     assert _call(B, K=-1) == -2
     assert _call(B, dt=7) == -3
-    assert _call(B, opts=B.DppoOpts(0.0, 5, 0, 0)) == -3
-    assert _call(B, variant=4) == -4
+    assert _call(B, opts=B.DppoOpts(0.0, 5, 0, 0.0, 0.0)) == -3
+    assert _call(B, variant=5) == -4
     assert _call(B, variant=-1) == -4
-    assert _call(B, opts=B.DppoOpts(0.0, 0, 9, 0)) == -11
+    assert _call(B, opts=B.DppoOpts(0.0, 0, 9, 0.0, 0.0)) == -11
     assert _call(B, logits=None) == -1
     assert _call(B, loss=None) == -1
     assert _call(B, status=None) == -1
@@ -95,11 +95,11 @@ def test_misuse_is_rejected_before_launch(binding):
     assert _call(B, ws=None) == -8
     assert _call(B, ws=0xA0010) == -8
     assert _call(B, ws_bytes=100) == -8
-    assert _call(B, dl=0x10000, opts=B.DppoOpts(0.0, B.DLOGITS_F32, 0, 0)) == -9
+    assert _call(B, dl=0x10000, opts=B.DppoOpts(0.0, B.DLOGITS_F32, 0, 0.0, 0.0)) == -9
     assert _call(B, dl=0x10000, ld_out=128) == -9
     # forcing the bulk-copy kernel on a layout it cannot take
-    assert _call(B, V=63, ld=63, ld_out=63, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0)) == -7
-    assert _call(B, logits=0x10002, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0)) == -7
+    assert _call(B, V=63, ld=63, ld_out=63, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0.0, 0.0)) == -7
+    assert _call(B, logits=0x10002, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0.0, 0.0)) == -7
 
 
 def test_missing_library_fails_loudly(binding, monkeypatch, tmp_path):

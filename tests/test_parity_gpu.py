@@ -14,10 +14,11 @@ DEV = "cuda:0"
 KERNELS = {"ring": dppo.KERNEL_RING, "generic": dppo.KERNEL_GENERIC}
 
 
-def _run(batch, variant, K, delta, kernel, dlogits_f32=False, loss_scale=0.0, want_stats=True, dlogits=None):
+def _run(batch, variant, K, delta, kernel, dlogits_f32=False, loss_scale=0.0, want_stats=True, dlogits=None, is_cap=0.0, eps_low=0.0):
     out = dppo.dppo_loss_fwd_bwd(batch.logits, batch.sampled_ids, batch.mu_logp, batch.advantages, batch.token_mask,
                                  variant, K, delta, batch.mu_topk_ids, batch.mu_topk_p, loss_scale=loss_scale,
-                                 dlogits_f32=dlogits_f32, kernel=kernel, want_stats=want_stats, dlogits=dlogits)
+                                 dlogits_f32=dlogits_f32, kernel=kernel, want_stats=want_stats, dlogits=dlogits,
+                                 is_cap=is_cap, eps_low=eps_low)
     torch.cuda.synchronize()
     return out
 
@@ -35,12 +36,14 @@ def _stress_delta(D):
     return float(np.float32(0.5 * (d[i] + d[i + 1])))
 
 
-def _full_check(batch, variant, K, delta, kernel, dlogits_f32=False, loss_scale=0.0, expect_blocked=None):
-    out = _run(batch, variant, K, delta, kernel, dlogits_f32, loss_scale)
+def _full_check(batch, variant, K, delta, kernel, dlogits_f32=False, loss_scale=0.0, expect_blocked=None, is_cap=0.0, eps_low=0.0):
+    out = _run(batch, variant, K, delta, kernel, dlogits_f32, loss_scale, is_cap=is_cap, eps_low=eps_low)
     assert int(out["status"].item()) == 0
     h = P.host_inputs(batch)
-    ora = P.run_oracle(h, variant, K, delta, None if loss_scale == 0.0 else loss_scale)
-    n_exempt, d_err = P.check_scalars(out["divergence"].cpu().numpy(), out["mask"].cpu().numpy(), ora, h, delta)
+    ora = P.run_oracle(h, variant, K, delta, None if loss_scale == 0.0 else loss_scale, is_cap=is_cap if is_cap > 0 else None,
+                       eps_low=eps_low if eps_low > 0 else None)
+    n_exempt, d_err = P.check_scalars(out["divergence"].cpu().numpy(), out["mask"].cpu().numpy(), ora, h, delta,
+                                      eps_low=eps_low if eps_low > 0 else None)
     bf16_in = batch.logits.dtype == torch.bfloat16
     info = P.check_loss(float(out["loss"].item()), ora["loss"], bf16_in, ora["row_loss"])
     dinfo = P.check_dlogits(out["dlogits"], ora["dlogits"], out_is_bf16=(bf16_in and not dlogits_f32))
@@ -96,6 +99,26 @@ def test_qwen_fp32_gradient_and_generic_kernel(qwen_rows):
     assert info["max_err_over_max"] < 2e-5
     _full_check(qwen_rows, dppo.BINARY_TV, 0, 0.02, dppo.KERNEL_GENERIC)
     _full_check(qwen_rows, dppo.TOPK_KL, 64, 0.02, dppo.KERNEL_GENERIC, dlogits_f32=True)
+
+
+@pytest.mark.parametrize("kernel", sorted(KERNELS))
+def test_truncated_importance_weight_and_ppo_clip_baseline(kernel, qwen_rows):
+    """min(r, C) of Eq. unified_grad, the unmasked PG-IS / CISPO baselines (delta = inf) and the PPO ratio-clip mask."""
+    b = wl.Batch(qwen_rows.logits, qwen_rows.sampled_ids, qwen_rows.mu_logp, qwen_rows.advantages, None)
+    base = _run(b, dppo.BINARY_TV, 0, 1.0, KERNELS[kernel])
+    h = P.host_inputs(b)
+    r = P.run_oracle(h, O.BINARY_TV, 0, 1.0, None, want_grad=False)["r"]
+    C = float(np.float32(np.median(r)))                      # about half of the rows are truncated
+    _, ora, _ = _full_check(b, dppo.BINARY_TV, 0, 0.02, KERNELS[kernel], is_cap=C)
+    assert 0.3 < np.mean(ora["r"] > C) < 0.7
+    out, ora, _ = _full_check(b, dppo.BINARY_KL, 0, float("inf"), KERNELS[kernel], is_cap=3.0)     # CISPO / PG-TIS
+    assert np.all(ora["M"] == 1)
+    # PPO / GRPO clip with the paper's ranges: few rows clipped at noise 0.1; a tight range clips a good share
+    _full_check(b, dppo.PPO_CLIP, 0, 0.28, KERNELS[kernel], eps_low=0.2)
+    rr = np.sort(np.abs(r - 1.0))
+    eh = float(np.float32(0.5 * (rr[len(rr) // 2] + rr[len(rr) // 2 + 1])))
+    el = float(np.float32(0.5 * (rr[len(rr) // 3] + rr[len(rr) // 3 + 1])))
+    _full_check(b, dppo.PPO_CLIP, 0, eh, KERNELS[kernel], eps_low=el, expect_blocked=lambda k, n: 0.1 * n < k < 0.5 * n)
 
 
 # ------------------------------------------------------------------------------------- config 3
