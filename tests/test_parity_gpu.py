@@ -310,3 +310,46 @@ def test_full_size_binary_tv_sampled_rows():
     assert sums <= 2e-3 * mx * 40
     blocked = torch.nonzero(out["mask"] == 0)[:, 0]
     assert not out["dlogits"][blocked].any()
+
+
+def test_full_size_topk_tv_k20_sampled_rows():
+    """Config 3 at full size (T=16384, V=151936, bf16, TopK-TV, K=20, delta=0.2): sampled rows against the oracle."""
+    T = 16384
+    b = wl.qwen_vocab_rows(DEV, seed=1, K=20)
+    out = _run(b, dppo.TOPK_TV, 20, 0.2, dppo.KERNEL_AUTO)
+    assert int(out["status"].item()) == 0
+    rows = np.sort(np.random.default_rng(3).choice(T, 40, replace=False))
+    h = P.host_inputs(b, rows)
+    ora = P.run_oracle(h, O.TOPK_TV, 20, 0.2, 1.0 / T)
+    P.check_scalars(out["divergence"].cpu().numpy()[rows], out["mask"].cpu().numpy()[rows], ora, h, 0.2)
+    mx = float(out["dlogits"].abs().max().item())
+    P.check_dlogits(out["dlogits"][torch.as_tensor(rows, device=DEV)], ora["dlogits"], out_is_bf16=True, max_abs=mx)
+    # stress threshold on the same tensors: the mask of the sampled rows still agrees
+    d_all = out["divergence"]
+    delta = _stress_delta(d_all[torch.as_tensor(rows, device=DEV)])
+    out2 = _run(b, dppo.TOPK_TV, 20, delta, dppo.KERNEL_AUTO)
+    ora2 = P.run_oracle(h, O.TOPK_TV, 20, delta, 1.0 / T, want_grad=False)
+    P.check_scalars(out2["divergence"].cpu().numpy()[rows], out2["mask"].cpu().numpy()[rows], ora2, h, delta)
+    assert 0 < int((ora2["M"] == 0).sum()) < len(rows)
+
+
+def test_full_size_ragged_topk_kl_k64_one_response():
+    """Config 4, one padded response block at full size (8192 rows x V=151936, K=64, rollout noise 0.3, delta=0.05),
+    with the global token-mean scale of the 64-response batch, as the whole batch would be streamed."""
+    lengths = wl.ragged_lengths()
+    n_valid = int(sum(lengths))
+    i = 7                                          # a response of medium length
+    L = int(lengths[i])
+    b = wl.ragged_response(DEV, i, lengths)
+    b.logits[L:] = float("nan")                    # a kernel that read the padding would be caught
+    out = _run(b, dppo.TOPK_KL, 64, 0.05, dppo.KERNEL_AUTO, loss_scale=1.0 / n_valid)
+    assert int(out["status"].item()) == 0 and out["stats"][0].item() == L
+    rows = np.sort(np.random.default_rng(4).choice(L, 40, replace=False))
+    h = P.host_inputs(b, rows)
+    h["token_mask"] = None
+    ora = P.run_oracle(h, O.TOPK_KL, 64, 0.05, 1.0 / n_valid)
+    P.check_scalars(out["divergence"].cpu().numpy()[rows], out["mask"].cpu().numpy()[rows], ora, h, 0.05)
+    assert 0 < int((ora["M"] == 0).sum())          # this workload does leave the trust region
+    mx = float(out["dlogits"][:L].abs().max().item())
+    P.check_dlogits(out["dlogits"][torch.as_tensor(rows, device=DEV)], ora["dlogits"], out_is_bf16=True, max_abs=mx)
+    assert not out["dlogits"][L:].any() and not out["mask"][L:].any() and not out["divergence"][L:].any()
