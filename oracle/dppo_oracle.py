@@ -17,6 +17,7 @@ Reinforcement Learning", DPPO):
 * ``dppo_mask``                 asymmetric trust-region mask               (Eq. dppo_obj).
 * ``dppo_row`` / ``dppo_loss_fwd_bwd``  surrogate and its logits-gradient   (Eq. dppo_obj, Eq. unified_grad; C = inf unless is_cap is given).
 * ``ppo_clip_mask``             ratio-clipping mask of the PPO / GRPO baseline (App. C.1 mask definitions; Eq. ppo-clip).
+* ``minimal_mask``              the ablation mask of Sec. 5.3: negative samples whose probability dropped by >= delta.
 * ``dppo_fused_lmhead_fwd_bwd`` the same applied to logits = H W with the chain rule into H and W.
 
 Readings of points the paper leaves open (each is listed in the design notes):
@@ -35,8 +36,8 @@ from __future__ import annotations
 
 import numpy as np
 
-BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL, PPO_CLIP = 0, 1, 2, 3, 4
-VARIANT_NAMES = {BINARY_TV: "binary_tv", BINARY_KL: "binary_kl", TOPK_TV: "topk_tv", TOPK_KL: "topk_kl", PPO_CLIP: "ppo_clip"}
+BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL, PPO_CLIP, MINIMAL_MASK = 0, 1, 2, 3, 4, 5
+VARIANT_NAMES = {BINARY_TV: "binary_tv", BINARY_KL: "binary_kl", TOPK_TV: "topk_tv", TOPK_KL: "topk_kl", PPO_CLIP: "ppo_clip", MINIMAL_MASK: "minimal_mask"}
 
 
 def _f64(x):
@@ -154,6 +155,11 @@ def ppo_clip_mask(adv, r, eps_low, eps_high):
     return 0 if blocked else 1
 
 
+def minimal_mask(adv, mu_a, pi_a, delta):
+    """Sec. 5.3 (source of instability): M = 0 iff A < 0 and mu(a) - pi(a) >= delta; else 1."""
+    return 0 if (float(adv) < 0.0 and float(mu_a) - float(pi_a) >= float(delta)) else 1
+
+
 def divergence(variant, pi, a, mu_logp, topk_ids=None, topk_p=None):
     """D_t of one row for the chosen approximation, given pi[V] (float64 probabilities)."""
     mu_a = float(np.exp(float(mu_logp)))
@@ -179,7 +185,8 @@ def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=No
     if want_grad, dlogits[V] = g * (pi - onehot(a)): Eq. unified_grad, i.e. the derivative of the
     loss term with M and the truncated weight held constant (d log pi(a)/dz_j = 1[j=a] - pi_j).
     variant PPO_CLIP: D = |r - 1| and the mask is ppo_clip_mask with eps_high = delta and eps_low
-    (default: delta), the baseline the paper compares against.
+    (default: delta), the baseline the paper compares against.  variant MINIMAL_MASK: D = mu(a) - pi(a)
+    (signed) and the mask of Sec. 5.3.
     """
     log_pi, lse = log_softmax_row(z)
     pi = np.exp(log_pi)
@@ -189,6 +196,10 @@ def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=No
     if variant == PPO_CLIP:
         D = abs(r - 1.0)
         M = ppo_clip_mask(adv, r, delta if eps_low is None else eps_low, delta)
+    elif variant == MINIMAL_MASK:
+        mu_a = float(np.exp(float(mu_logp)))
+        D = mu_a - float(pi[a])                      # signed drop of the sampled token's probability
+        M = minimal_mask(adv, mu_a, pi[a], delta)
     else:
         D = divergence(variant, pi, a, mu_logp, topk_ids, topk_p)
         M = dppo_mask(adv, log_pi_a, mu_logp, D, delta)

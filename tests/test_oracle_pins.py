@@ -442,7 +442,23 @@ def check_ppo_clip_variant(O):
     assert O.dppo_row(z, 0, math.log(1e-4), 1.0, O.BINARY_TV, 0.2, 1.0)["M"] == 1
 
 
-CHECKS = [check_is_cap_and_baselines, check_ppo_clip_variant, check_worked_example, check_log_softmax, check_binary, check_topk_full_and_bounds,
+def check_minimal_mask(O):
+    """Sec. 5.3: only negative samples whose sampled-token probability dropped by at least delta are blocked."""
+    for adv, mu, pi, delta, expect in ((-1.0, 0.9, 0.3, 0.5, 0), (-1.0, 0.9, 0.4, 0.5, 0), (-1.0, 0.9, 0.41, 0.5, 1),
+                                       (1.0, 0.9, 0.1, 0.5, 1), (-1.0, 0.3, 0.9, 0.5, 1), (0.0, 0.9, 0.1, 0.5, 1),
+                                       (-1.0, 0.99, 0.18, 0.8, 0), (-1.0, 0.99, 0.20, 0.8, 1)):
+        assert O.minimal_mask(adv, mu, pi, delta) == expect, (adv, mu, pi, delta)
+        z = np.log(np.array([pi, (1 - pi) * 0.25, (1 - pi) * 0.75]))
+        o = O.dppo_row(z, 0, math.log(mu), adv, O.MINIMAL_MASK, delta, 0.5)
+        assert o["M"] == expect and abs(o["D"] - (mu - pi)) < 1e-12
+        # the blocked set is inside the DPPO Binary-TV blocked set at the same threshold (it adds "A < 0" and the sign)
+        if expect == 0:
+            assert O.dppo_row(z, 0, math.log(mu), adv, O.BINARY_TV, delta - 1e-9, 0.5)["M"] == 0
+        g_expect = 0.5 * expect * (pi / mu) * adv
+        assert abs(o["g"] - g_expect) < 1e-12
+
+
+CHECKS = [check_minimal_mask, check_is_cap_and_baselines, check_ppo_clip_variant, check_worked_example, check_log_softmax, check_binary, check_topk_full_and_bounds,
           check_topk_other_bucket, check_topk_equality_conditions, check_edge_conventions,
           check_mask_truth_table, check_on_policy, check_gradient, check_brute_force_tiny, check_fused]
 
@@ -540,10 +556,11 @@ def _cap_as_max(m):
     return dppo_row
 
 
-MUTANTS.update({"cap_as_max": _cap_as_max, "ppo_eps_swapped": lambda m: (lambda adv, r, el, eh: 0 if ((adv > 0 and r - 1 > el) or (adv < 0 and 1 - r > eh)) else 1),
+MUTANTS.update({"minimal_mask_positive_side": lambda m: (lambda adv, mu, pi, delta: 0 if (adv > 0 and mu - pi >= delta) else 1),
+                "cap_as_max": _cap_as_max, "ppo_eps_swapped": lambda m: (lambda adv, r, el, eh: 0 if ((adv > 0 and r - 1 > el) or (adv < 0 and 1 - r > eh)) else 1),
                 "topk_no_dedupe": _no_dedupe, "grad_sign": _grad_sign, "grad_no_onehot": _grad_no_onehot,
                 "fused_scaled": _fused_transposed})
-MUTANT_TARGET.update({"cap_as_max": "dppo_row", "ppo_eps_swapped": "ppo_clip_mask", "topk_no_dedupe": "topk_reduced", "grad_sign": "dppo_row", "grad_no_onehot": "dppo_row",
+MUTANT_TARGET.update({"minimal_mask_positive_side": "minimal_mask", "cap_as_max": "dppo_row", "ppo_eps_swapped": "ppo_clip_mask", "topk_no_dedupe": "topk_reduced", "grad_sign": "dppo_row", "grad_no_onehot": "dppo_row",
                       "fused_scaled": "dppo_fused_lmhead_fwd_bwd"})
 
 
