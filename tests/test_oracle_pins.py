@@ -444,10 +444,11 @@ def check_ppo_clip_variant(O):
 
 def check_minimal_mask(O):
     """Sec. 5.3: only negative samples whose sampled-token probability dropped by at least delta are blocked."""
-    for adv, mu, pi, delta, expect in ((-1.0, 0.9, 0.3, 0.5, 0), (-1.0, 0.9, 0.4, 0.5, 0), (-1.0, 0.9, 0.41, 0.5, 1),
+    for adv, mu, pi, delta, expect in ((-1.0, 0.9, 0.3, 0.5, 0), (-1.0, 0.9, 0.39, 0.5, 0), (-1.0, 0.9, 0.41, 0.5, 1),
                                        (1.0, 0.9, 0.1, 0.5, 1), (-1.0, 0.3, 0.9, 0.5, 1), (0.0, 0.9, 0.1, 0.5, 1),
                                        (-1.0, 0.99, 0.18, 0.8, 0), (-1.0, 0.99, 0.20, 0.8, 1)):
         assert O.minimal_mask(adv, mu, pi, delta) == expect, (adv, mu, pi, delta)
+        assert O.minimal_mask(-1.0, 0.75, 0.25, 0.5) == 0          # ">=": exactly delta is blocked (exact in binary)
         z = np.log(np.array([pi, (1 - pi) * 0.25, (1 - pi) * 0.75]))
         o = O.dppo_row(z, 0, math.log(mu), adv, O.MINIMAL_MASK, delta, 0.5)
         assert o["M"] == expect and abs(o["D"] - (mu - pi)) < 1e-12
