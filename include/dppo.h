@@ -49,7 +49,9 @@ extern "C" {
 enum { DPPO_BINARY_TV = 0, DPPO_BINARY_KL = 1, DPPO_TOPK_TV = 2, DPPO_TOPK_KL = 3,
        /* baseline the paper compares against: D_t = |r_t - 1| with the PPO / GRPO ratio-clip mask (App. C.1):
           M_t = 0 iff (A > 0 and r - 1 > delta) or (A < 0 and 1 - r > eps_low); delta plays eps_high */
-       DPPO_PPO_CLIP = 4 };
+       DPPO_PPO_CLIP = 4,
+       /* ablation of Sec. 5.3: D_t = mu(a_t) - pi(a_t) (signed), M_t = 0 iff A_t < 0 and D_t >= delta */
+       DPPO_MINIMAL_MASK = 5 };
 /* Element types of the logits / dlogits tensors. */
 enum { DPPO_F32 = 0, DPPO_BF16 = 1 };
 /* opts->dlogits_dtype */
@@ -210,7 +212,7 @@ size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V);
  *
  *  hidden   [T, d] bf16 row-major;  W  [d, V] bf16 row-major (LM head);  d and V multiples of 8, 16-byte aligned.
  *  sampled_ids, mu_logp, advantages, token_mask, delta, opts, loss, divergence, mask, stats, status: as for
- *           dppo_loss_fwd_bwd.  variant: DPPO_BINARY_TV, DPPO_BINARY_KL or DPPO_PPO_CLIP (Top-K: DPPO_ERR_VARIANT).
+ *           dppo_loss_fwd_bwd.  variant: any but the Top-K ones (those: DPPO_ERR_VARIANT).
  *  dHidden  [T, d] fp32 out: d loss / d hidden = dlogits . W^T.
  *  dW       [d, V] fp32 out: d loss / d W = hidden^T . dlogits (overwritten, not accumulated).
  *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V) bytes; it holds W^T, hidden^T, the

@@ -112,6 +112,9 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
     D = fabs(r - 1.0);
     const double eh = (double)p.delta, el = (p.eps_low > 0.f) ? (double)p.eps_low : (double)p.delta;
     ppo_blocked = (adv > 0.0 && r - 1.0 > eh) || (adv < 0.0 && 1.0 - r > el);
+  } else if (p.variant == DPPO_MINIMAL_MASK) {        // ablation of Sec. 5.3: signed drop of the sampled token's probability
+    D = mu_a - pi_a;
+    ppo_blocked = (adv < 0.0 && D >= (double)p.delta);
   } else if (p.variant == DPPO_BINARY_TV) {
     D = fabs(mu_a - pi_a);                            // Eq. binary_tv
   } else if (p.variant == DPPO_BINARY_KL) {           // Eq. binary_kl
@@ -157,7 +160,7 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
   }
   // Eq. dppo_obj: blocked iff D > delta and the ratio already left 1 on the side the advantage pushes.
   const bool away = (adv > 0.0 && lpa > mu_logp) || (adv < 0.0 && lpa < mu_logp);
-  const int M = (p.variant == DPPO_PPO_CLIP) ? (ppo_blocked ? 0 : 1) : ((away && D > (double)p.delta) ? 0 : 1);
+  const int M = (p.variant == DPPO_PPO_CLIP || p.variant == DPPO_MINIMAL_MASK) ? (ppo_blocked ? 0 : 1) : ((away && D > (double)p.delta) ? 0 : 1);
   // Eq. unified_grad: the importance weight in loss and gradient is min(r, C)
   const double w = (p.is_cap > 0.f && isfinite(p.is_cap)) ? fmin(r, (double)p.is_cap) : r;
   D_out = (float)D;

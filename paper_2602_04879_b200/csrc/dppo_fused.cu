@@ -234,7 +234,8 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   dppo_opts o = {};
   if (opts) o = *opts;
   if (T < 0 || d < 1 || V < 1 || T > (int64_t)1 << 30 || V > (int64_t)1 << 30 || d > (int64_t)1 << 30) return DPPO_ERR_SHAPE;
-  if (variant != DPPO_BINARY_TV && variant != DPPO_BINARY_KL && variant != DPPO_PPO_CLIP) return DPPO_ERR_VARIANT;
+  if (variant != DPPO_BINARY_TV && variant != DPPO_BINARY_KL && variant != DPPO_PPO_CLIP && variant != DPPO_MINIMAL_MASK)
+    return DPPO_ERR_VARIANT;
   if (!loss || !status || !W || !dW) return DPPO_ERR_NULL;
   if (T > 0 && (!hidden || !sampled_ids || !mu_logp || !advantages || !divergence || !mask || !dHidden)) return DPPO_ERR_NULL;
   if (((uintptr_t)hidden % 16) || ((uintptr_t)W % 16) || (d % 8) || (V % 8)) return DPPO_ERR_ALIGN;

@@ -119,6 +119,12 @@ def test_truncated_importance_weight_and_ppo_clip_baseline(kernel, qwen_rows):
     eh = float(np.float32(0.5 * (rr[len(rr) // 2] + rr[len(rr) // 2 + 1])))
     el = float(np.float32(0.5 * (rr[len(rr) // 3] + rr[len(rr) // 3 + 1])))
     _full_check(b, dppo.PPO_CLIP, 0, eh, KERNELS[kernel], eps_low=el, expect_blocked=lambda k, n: 0.1 * n < k < 0.5 * n)
+    # minimal mask of Sec. 5.3 (signed D = mu(a) - pi(a); only negative samples are ever blocked)
+    dd = np.exp(h["mu_logp"]) - r * np.exp(h["mu_logp"])
+    pos = np.sort(dd[(dd > 0) & (h["advantages"] < 0)])
+    dm = float(np.float32(0.5 * (pos[len(pos) // 2] + pos[len(pos) // 2 + 1])))
+    out, ora, _ = _full_check(b, dppo.MINIMAL_MASK, 0, dm, KERNELS[kernel], expect_blocked=lambda k, n: 0 < k < 0.5 * n)
+    assert np.all(h["advantages"][ora["M"] == 0] < 0)
 
 
 # ------------------------------------------------------------------------------------- config 3
