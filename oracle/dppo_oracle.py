@@ -14,6 +14,8 @@ Reinforcement Learning", DPPO):
 * ``topk_reduced``              A'_t = TopK(mu, K) u {a_t} plus "other"    (Sec. 4.4, Top-K Approximation).
 * ``topk_tv`` / ``topk_kl``     divergences of the reduced categoricals    (Eq. topk_tv, Eq. topk_kl).
 * ``full_tv`` / ``full_kl``     exact full-vocabulary divergences          (App. B definitions).
+* ``exact_divergence_row``      what the approximations stand in for, from two logits rows: full TV, full KL(mu||pi)
+                                (App. B) and the entropy of pi (a run metric of App. E).
 * ``dppo_mask``                 asymmetric trust-region mask               (Eq. dppo_obj).
 * ``dppo_row`` / ``dppo_loss_fwd_bwd``  surrogate and its logits-gradient   (Eq. dppo_obj, Eq. unified_grad; C = inf unless is_cap is given).
 * ``ppo_clip_mask``             ratio-clipping mask of the PPO / GRPO baseline (App. C.1 mask definitions; Eq. ppo-clip).
@@ -133,6 +135,20 @@ def full_tv(mu, pi):
 def full_kl(mu, pi):
     """Exact KL(mu || pi) over the whole vocabulary  (App. B)."""
     return float(sum(_xlogx_over_y(x, y) for x, y in zip(_f64(mu), _f64(pi))))
+
+
+def exact_divergence_row(z, z_mu):
+    """Full-vocabulary quantities of one state from the trainer's and the rollout policy's logits rows:
+    TV = 1/2 sum |mu - pi|, KL(mu || pi) = sum mu log(mu / pi)  (App. B definitions) and the entropy
+    -sum pi log pi of the trainer policy.  Returns (tv, kl, entropy)."""
+    log_pi, _ = log_softmax_row(z)
+    log_mu, _ = log_softmax_row(z_mu)
+    pi, mu = np.exp(log_pi), np.exp(log_mu)
+    tv = full_tv(mu, pi)
+    with np.errstate(invalid="ignore"):              # 0 * log 0 = 0 (entries with probability zero)
+        kl = float(np.sum(np.where(mu > 0, mu * (log_mu - log_pi), 0.0)))   # log domain: no 0/0 on underflow
+        ent = -float(np.sum(np.where(pi > 0, pi * log_pi, 0.0)))
+    return tv, kl, ent
 
 
 def dppo_mask(adv, log_pi_a, mu_logp, D, delta):

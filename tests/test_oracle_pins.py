@@ -459,7 +459,31 @@ def check_minimal_mask(O):
         assert abs(o["g"] - g_expect) < 1e-12
 
 
-CHECKS = [check_minimal_mask, check_is_cap_and_baselines, check_ppo_clip_variant, check_worked_example, check_log_softmax, check_binary, check_topk_full_and_bounds,
+def check_exact_divergence(O):
+    """Full TV / KL / entropy from two logits rows against library routines and the App. B ordering."""
+    rng = np.random.default_rng(11)
+    for V in (2, 9, 500):
+        z = 3 * rng.standard_normal(V)
+        zm = z + rng.standard_normal(V)
+        tv, kl, ent = O.exact_divergence_row(z, zm)
+        pi, mu = scipy.special.softmax(z), scipy.special.softmax(zm)
+        assert abs(tv - 0.5 * np.abs(mu - pi).sum()) < 1e-13
+        assert abs(kl - scipy.stats.entropy(mu, pi)) < 1e-12
+        assert abs(ent - scipy.stats.entropy(pi)) < 1e-12
+        assert abs(kl - O.full_kl(mu, pi)) < 1e-12 and tv * tv <= 0.5 * kl + 1e-15
+        a = int(rng.integers(0, V))
+        assert O.binary_tv(mu[a], pi[a]) <= tv + 1e-15 and O.binary_kl(mu[a], pi[a]) <= kl + 1e-13
+    tv, kl, ent = O.exact_divergence_row(np.zeros(64), np.zeros(64))
+    assert tv == 0.0 and abs(kl) < 1e-15 and abs(ent - math.log(64)) < 1e-13
+    # direction: KL(mu || pi), not the reverse
+    z, zm = np.log([0.7, 0.2, 0.1]), np.log([0.1, 0.3, 0.6])
+    assert abs(O.exact_divergence_row(z, zm)[1] - (0.1 * math.log(0.1 / 0.7) + 0.3 * math.log(0.3 / 0.2) + 0.6 * math.log(0.6 / 0.1))) < 1e-12
+    # huge offsets and a -inf entry do not produce nan
+    tv, kl, ent = O.exact_divergence_row(np.array([800.0, 799.0, -np.inf]), np.array([-300.0, -301.0, -np.inf]))
+    assert np.isfinite(tv) and np.isfinite(ent) and np.isfinite(kl)
+
+
+CHECKS = [check_exact_divergence, check_minimal_mask, check_is_cap_and_baselines, check_ppo_clip_variant, check_worked_example, check_log_softmax, check_binary, check_topk_full_and_bounds,
           check_topk_other_bucket, check_topk_equality_conditions, check_edge_conventions,
           check_mask_truth_table, check_on_policy, check_gradient, check_brute_force_tiny, check_fused]
 
