@@ -234,6 +234,22 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
 int dppo_gemm_tn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,
                       int32_t* status, void* cuda_stream);
 
+/*
+ * Exact full-vocabulary divergence between the rollout policy and the trainer policy, and the trainer policy's
+ * entropy, streamed from the two logits tensors (App. B defines the exact TV and KL that the Binary / Top-K forms bound
+ * from below; App. E lists entropy and |pi - mu| among the run metrics).  No probability tensor is materialised.
+ *
+ *  logits, mu_logits  [T, V] row-major (row strides in elements, >= V), both of `dtype` (DPPO_F32 or DPPO_BF16).
+ *  token_mask         [T] bytes or NULL; rows with a zero byte are not read and give 0.
+ *  tv, kl, entropy    [T] out: 1/2 sum_j |mu_j - pi_j|,  sum_j mu_j log(mu_j / pi_j),  -sum_j pi_j log pi_j.
+ *  status             device word; DPPO_STATUS_NONFINITE_ROW if a row's log-sum-exp is not finite (outputs 0).
+ * Needs no workspace.  Each row is read twice (the second time normally from L2).
+ */
+int dppo_exact_divergence(const void* logits, const void* mu_logits, int64_t T, int64_t V,
+                          int64_t logits_row_stride, int64_t mu_row_stride, int dtype,
+                          const uint8_t* token_mask, float* tv, float* kl, float* entropy,
+                          int32_t* status, void* cuda_stream);
+
 /* Name of an error code (static string, never NULL). */
 const char* dppo_error_string(int code);
 

@@ -64,6 +64,9 @@ def lib():
         L.dppo_fused_lmhead_fwd_bwd.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
                                                 c_void_p, c_int, c_float, POINTER(DppoOpts), c_void_p, c_void_p, c_void_p,
                                                 c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.dppo_exact_divergence.restype = c_int
+        L.dppo_exact_divergence.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p,
+                                            c_void_p, c_void_p, c_void_p, c_void_p]
         L.dppo_gemm_tn_bf16.restype = c_int
         L.dppo_gemm_tn_bf16.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_int, c_int, c_int, c_void_p, c_int64,
                                         c_void_p, c_void_p]
@@ -174,6 +177,28 @@ def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token
     if rc != 0:
         raise DppoError(rc, "dppo_fused_lmhead_fwd_bwd")
     return dict(loss=loss, divergence=D, mask=M, dHidden=dHidden, dW=dW, stats=stats, status=status)
+
+
+def dppo_exact_divergence(logits, mu_logits, token_mask=None, status=None, stream=None):
+    """Calls ``dppo_exact_divergence``: per-row exact TV, KL(mu||pi) and entropy of pi from two [T,V] CUDA logits tensors
+    of the same dtype.  Returns dict(tv, kl, entropy, status)."""
+    assert logits.is_cuda and mu_logits.is_cuda and logits.dtype == mu_logits.dtype and logits.shape == mu_logits.shape
+    assert logits.stride(1) == 1 and mu_logits.stride(1) == 1
+    T, V = logits.shape
+    dev = logits.device
+    tv = torch.empty(T, dtype=torch.float32, device=dev)
+    kl = torch.empty(T, dtype=torch.float32, device=dev)
+    ent = torch.empty(T, dtype=torch.float32, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    with torch.cuda.device(dev):
+        rc = lib().dppo_exact_divergence(_ptr(logits), _ptr(mu_logits), T, V, logits.stride(0) if T > 0 else V,
+                                         mu_logits.stride(0) if T > 0 else V, _dtype_code(logits), _ptr(token_mask), _ptr(tv),
+                                         _ptr(kl), _ptr(ent), _ptr(status), c_void_p(st.cuda_stream))
+    if rc != 0:
+        raise DppoError(rc, "dppo_exact_divergence")
+    return dict(tv=tv, kl=kl, entropy=ent, status=status)
 
 
 def dppo_gemm_tn_bf16(A, B, C=None, status=None, stream=None):

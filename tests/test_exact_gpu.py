@@ -1,0 +1,71 @@
+"""Exact full-vocabulary TV / KL / entropy kernel against the float64 oracle (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2602_04879_b200 as dppo
+from oracle import dppo_oracle as O
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _pair(T, V, dtype, seed, noise):
+    g = torch.Generator(device=DEV).manual_seed(seed)
+    z = (3.0 * torch.randn((T, V), generator=g, device=DEV)).to(dtype)
+    zm = (z.float() + noise * torch.randn((T, V), generator=g, device=DEV)).to(dtype)
+    return z, zm
+
+
+def _check(z, zm, tok=None, rows=None):
+    out = dppo.dppo_exact_divergence(z, zm, tok)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    T = z.shape[0]
+    rows = range(T) if rows is None else rows
+    zh, zmh = z.float().cpu().numpy().astype(np.float64), zm.float().cpu().numpy().astype(np.float64)
+    tv, kl, ent = out["tv"].cpu().numpy(), out["kl"].cpu().numpy(), out["entropy"].cpu().numpy()
+    for t in rows:
+        if tok is not None and tok[t].item() == 0:
+            assert tv[t] == 0 and kl[t] == 0 and ent[t] == 0
+            continue
+        o_tv, o_kl, o_ent = O.exact_divergence_row(zh[t], zmh[t])
+        assert abs(tv[t] - o_tv) <= 1e-5 and abs(kl[t] - o_kl) <= 1e-5 and abs(ent[t] - o_ent) <= 2e-5 * max(1.0, o_ent), t
+    return out
+
+
+@pytest.mark.parametrize("T,V,dtype", [(37, 4096, torch.float32), (50, 1001, torch.bfloat16), (64, 151936, torch.bfloat16), (5, 8, torch.float32)])
+def test_exact_divergence_matches_oracle(T, V, dtype):
+    z, zm = _pair(T, V, dtype, seed=T + V, noise=0.5)
+    tok = (torch.arange(T, device=DEV) % 5 != 2).to(torch.uint8)
+    out = _check(z, zm, tok)
+    # App. B: the Binary approximation never exceeds the exact divergence
+    a = torch.randint(0, V, (T,), device=DEV, dtype=torch.int32)
+    mu_logp = torch.log_softmax(zm.float(), 1).gather(1, a.long()[:, None])[:, 0].contiguous()
+    adv = torch.ones(T, device=DEV)
+    b_tv = dppo.dppo_loss_fwd_bwd(z, a, mu_logp, adv, tok, dppo.BINARY_TV, 0, 1.0)["divergence"]
+    b_kl = dppo.dppo_loss_fwd_bwd(z, a, mu_logp, adv, tok, dppo.BINARY_KL, 0, 1.0)["divergence"]
+    assert torch.all(b_tv <= out["tv"] + 1e-5) and torch.all(b_kl <= out["kl"] + 1e-5)
+
+
+def test_exact_divergence_edge_cases():
+    z, zm = _pair(8, 512, torch.float32, seed=3, noise=0.2)
+    # identical policies: zero divergence, entropy of uniform logits = log V
+    out = dppo.dppo_exact_divergence(z, z.clone())
+    assert out["tv"].abs().max().item() <= 1e-6 and out["kl"].abs().max().item() <= 1e-6
+    u = torch.zeros((3, 512), device=DEV)
+    out = dppo.dppo_exact_divergence(u, u.clone())
+    assert torch.allclose(out["entropy"], torch.full((3,), float(np.log(512)), device=DEV), atol=1e-5)
+    # -inf entries are probability zero; a nan row only raises the status bit
+    z2, zm2 = z.clone(), zm.clone()
+    z2[:, 5::7] = float("-inf")
+    zm2[:, 5::7] = float("-inf")
+    _check(z2, zm2)
+    z2[3, 0] = float("nan")
+    out = dppo.dppo_exact_divergence(z2, zm2)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == dppo.binding.STATUS_NONFINITE_ROW and out["tv"][3].item() == 0
+    # strided views
+    wide = torch.zeros((8, 600), device=DEV)
+    wide[:, :512] = z
+    _check(wide[:, :512], zm)
