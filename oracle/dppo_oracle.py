@@ -268,14 +268,16 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
 
 
 def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None,
-                              variant=BINARY_TV, delta=0.2, loss_scale=None):
+                              variant=BINARY_TV, delta=0.2, loss_scale=None, K=0, mu_topk_ids=None, mu_topk_p=None,
+                              is_cap=None, eps_low=None):
     """LM-head variant: logits = hidden @ W in float64 (never rounded), then the path above,
     then the chain rule: dHidden = dlogits @ W^T, dW = hidden^T @ dlogits.
     """
     H = _f64(hidden)
     Wm = _f64(W)
     z = H @ Wm
-    o = dppo_loss_fwd_bwd(z, sampled_ids, mu_logp, advantages, token_mask, variant, 0, delta, loss_scale)
+    o = dppo_loss_fwd_bwd(z, sampled_ids, mu_logp, advantages, token_mask, variant, K, delta, loss_scale,
+                          mu_topk_ids, mu_topk_p, True, is_cap, eps_low)
     o["dHidden"] = o["dlogits"] @ Wm.T
     o["dW"] = H.T @ o["dlogits"]
     return o
