@@ -202,26 +202,28 @@ int dppo_loss_fwd_bwd_static_ws(const void* logits, int64_t T, int64_t V, int64_
                                 float* stats, int32_t* status, void* cuda_stream);
 
 /* Bytes of device workspace dppo_fused_lmhead_fwd_bwd needs (256-byte aligned pointer expected). */
-size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V);
+size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V, int K);
 
 /*
  * Fused LM-head variant (not in the paper, which takes the trainer's logits as given; the loss is Eq. dppo_obj
- * with the Binary approximations of Eq. binary_tv / Eq. binary_kl, the gradient Eq. unified_grad with C = infinity):
+ * with any of the divergence approximations of Sec. 4.4, the gradient Eq. unified_grad):
  * logits = hidden x W are produced tile by tile on the tensor cores and consumed in the accumulator epilogue, so the
  * [T, V] logits are never written to memory; the gradient is propagated to hidden and W.
  *
  *  hidden   [T, d] bf16 row-major;  W  [d, V] bf16 row-major (LM head);  d and V multiples of 8, 16-byte aligned.
  *  sampled_ids, mu_logp, advantages, token_mask, delta, opts, loss, divergence, mask, stats, status: as for
- *           dppo_loss_fwd_bwd.  variant: any but the Top-K ones (those: DPPO_ERR_VARIANT).
+ *           dppo_loss_fwd_bwd.  mu_topk_ids / mu_topk_p [T, K]: as for dppo_loss_fwd_bwd (Top-K variants; the K
+ *           logits per row are recomputed as dot products, K is ignored by the other variants).
  *  dHidden  [T, d] fp32 out: d loss / d hidden = dlogits . W^T.
  *  dW       [d, V] fp32 out: d loss / d W = hidden^T . dlogits (overwritten, not accumulated).
- *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V) bytes; it holds W^T, hidden^T, the
+ *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V, K) bytes; it holds W^T, hidden^T, the
  *           bf16 gradient with respect to the logits and its transpose (about 4 T V + 2 d V bytes).
  * The gradient with respect to the logits is rounded to bf16 before the two gradient GEMMs (fp32 accumulation).
  */
 int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int64_t d, int64_t V,
-                              const int32_t* sampled_ids, const float* mu_logp, const float* advantages,
-                              const uint8_t* token_mask, int variant, float delta, const dppo_opts* opts,
+                              const int32_t* sampled_ids, const float* mu_logp,
+                              const int32_t* mu_topk_ids, const float* mu_topk_p, const float* advantages,
+                              const uint8_t* token_mask, int variant, int K, float delta, const dppo_opts* opts,
                               float* loss, float* divergence, uint8_t* mask, float* dHidden, float* dW,
                               float* stats, int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 

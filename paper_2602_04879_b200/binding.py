@@ -59,10 +59,11 @@ def lib():
                                              c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                              c_void_p, c_size_t, c_int64]
         L.dppo_fused_workspace_bytes.restype = c_size_t
-        L.dppo_fused_workspace_bytes.argtypes = [c_int64, c_int64, c_int64]
+        L.dppo_fused_workspace_bytes.argtypes = [c_int64, c_int64, c_int64, c_int]
         L.dppo_fused_lmhead_fwd_bwd.restype = c_int
         L.dppo_fused_lmhead_fwd_bwd.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
-                                                c_void_p, c_int, c_float, POINTER(DppoOpts), c_void_p, c_void_p, c_void_p,
+                                                c_void_p, c_void_p, c_void_p, c_int, c_int, c_float, POINTER(DppoOpts),
+                                                c_void_p, c_void_p, c_void_p,
                                                 c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.dppo_exact_divergence.restype = c_int
         L.dppo_exact_divergence.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p,
@@ -141,13 +142,13 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
     return dict(loss=loss, divergence=D, mask=M, dlogits=dlogits, stats=stats, status=status)
 
 
-def dppo_fused_workspace_bytes(T, d, V):
-    return int(lib().dppo_fused_workspace_bytes(int(T), int(d), int(V)))
+def dppo_fused_workspace_bytes(T, d, V, K=0):
+    return int(lib().dppo_fused_workspace_bytes(int(T), int(d), int(V), int(K)))
 
 
 def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, delta=0.2,
                               loss_scale=0.0, want_stats=False, workspace=None, dHidden=None, dW=None, status=None, stream=None,
-                              is_cap=0.0, eps_low=0.0):
+                              is_cap=0.0, eps_low=0.0, K=0, mu_topk_ids=None, mu_topk_p=None):
     """Calls ``dppo_fused_lmhead_fwd_bwd`` on CUDA tensors: hidden [T,d] bf16, W [d,V] bf16.  Returns
     dict(loss[1], divergence[T], mask[T], dHidden[T,d] fp32, dW[d,V] fp32, stats, status); nothing is synchronised."""
     assert hidden.is_cuda and W.is_cuda and hidden.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
@@ -166,12 +167,13 @@ def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
     if workspace is None:
-        workspace = torch.empty(dppo_fused_workspace_bytes(T, d, V), dtype=torch.uint8, device=dev)
+        workspace = torch.empty(dppo_fused_workspace_bytes(T, d, V, K), dtype=torch.uint8, device=dev)
     opts = DppoOpts(float(loss_scale), 0, 0, float(is_cap), float(eps_low))
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     with torch.cuda.device(dev):
-        rc = lib().dppo_fused_lmhead_fwd_bwd(_ptr(hidden), _ptr(W), T, d, V, _ptr(sampled_ids), _ptr(mu_logp), _ptr(advantages),
-                                             _ptr(token_mask), int(variant), float(delta), ctypes.byref(opts), _ptr(loss),
+        rc = lib().dppo_fused_lmhead_fwd_bwd(_ptr(hidden), _ptr(W), T, d, V, _ptr(sampled_ids), _ptr(mu_logp),
+                                             _ptr(mu_topk_ids), _ptr(mu_topk_p), _ptr(advantages),
+                                             _ptr(token_mask), int(variant), int(K), float(delta), ctypes.byref(opts), _ptr(loss),
                                              _ptr(D), _ptr(M), _ptr(dHidden), _ptr(dW), _ptr(stats), _ptr(status),
                                              _ptr(workspace), workspace.numel(), c_void_p(st.cuda_stream))
     if rc != 0:

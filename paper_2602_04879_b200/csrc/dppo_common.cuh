@@ -93,7 +93,7 @@ __device__ __forceinline__ double xlogx_over_y(double x, double y) {
 
 // Per-row scalar stage, run by ONE full warp (all 32 lanes call it with the same arguments).
 //   lse        log-sum-exp of the row (double, from fp32 partial sums)
-//   z_at(id)   fp32 value of this row's logit `id` (global read)
+//   z_at(id, k)  fp32 value of this row's logit `id`; k is its position in the top-K list, -1 for the sampled id
 // Returns on every lane the same values.  `flags` receives DPPO_STATUS_* bits found here.
 template <typename ZAt>
 __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, int a, double lse, double scale,
@@ -102,7 +102,7 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
   const int lane = threadIdx.x & 31;
   const double mu_logp = (double)p.mu_logp[t];
   const double adv = (double)p.adv[t];
-  const double lpa = (double)z_at(a) - lse;           // log pi(a_t)
+  const double lpa = (double)z_at(a, -1) - lse;           // log pi(a_t)
   const double pi_a = exp(lpa);
   const double mu_a = exp(mu_logp);
   const double r = exp(lpa - mu_logp);                // Eq. ppo-clip
@@ -130,7 +130,7 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
       int id = ids[k];
       if (id < 0 || (int64_t)id >= p.V) { bad = 1; continue; }
       double pm = (double)ps[k];
-      double lpk = (double)z_at(id) - lse;
+      double lpk = (double)z_at(id, k) - lse;
       double pk = exp(lpk);
       sum_mu += pm;
       sum_pi += pk;

@@ -4,6 +4,7 @@
 //   1. W^T, hidden^T  (bf16 transposes: every GEMM below then has both operands K-major)
 //   2. stats GEMM     z-tile = hidden . W^T-tile; epilogue: per-row (max, sum exp) of the tile, z at the sampled id
 //   3. scalar kernel  merge the tiles' partials -> lse; ratio, divergence, mask, loss term, gradient coefficients
+//                     (Top-K variants: the K logits per row come from a small gather-dot kernel over rows of W^T)
 //   4. grad GEMM      the same tiles again; epilogue: P = dlogits = g (softmax - onehot) in bf16,
 //   5.                written both as P [T, V] and as P^T [V, T]
 //   6. dHidden = P . W     (A = P [T,V], B = W [d,V])          fp32
@@ -121,9 +122,37 @@ cudaError_t transpose_bf16(const void* in, int64_t rows, int64_t cols, int64_t l
   return cudaGetLastError();
 }
 
+// z_topk[t, k] = hidden[t, :] . W^T[ids[t, k], :]: the logits at the rollout policy's top-K ids, one warp per (t, k).
+// W^T rows are contiguous, so each dot product reads two 2d-byte rows with 16-byte loads (d is a multiple of 8).
+__global__ void __launch_bounds__(256) fused_topk_logits_kernel(const __nv_bfloat16* hidden, const __nv_bfloat16* wt, int64_t T,
+                                                                int64_t d, int64_t V, const int32_t* ids, int K, float* z_topk) {
+  const int lane = threadIdx.x & 31;
+  const int64_t w = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (w >= T * K) return;
+  const int64_t t = w / K;
+  const int id = ids[w];
+  float acc = 0.f;
+  if (id >= 0 && (int64_t)id < V) {
+    const uint4* h = reinterpret_cast<const uint4*>(hidden + t * d);
+    const uint4* r = reinterpret_cast<const uint4*>(wt + (int64_t)id * d);
+    for (int64_t j = lane; j < d / 8; j += 32) {
+      const uint4 x = h[j], y = r[j];
+      const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        acc = fmaf(__uint_as_float(xs[i] << 16), __uint_as_float(ys[i] << 16), acc);
+        acc = fmaf(__uint_as_float(xs[i] & 0xffff0000u), __uint_as_float(ys[i] & 0xffff0000u), acc);
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) z_topk[w] = acc;       // out-of-range ids give 0 here and raise the status bit in the scalar stage
+}
+
 // One warp per row: merge the stats GEMM's per-tile partials, then the same scalar stage as the streaming kernels.
 __global__ void __launch_bounds__(256) fused_scalar_kernel(RowParams p, const float2* part, int tiles_n, const float* z_a,
-                                                           float* c2, float* sgn, float* fix) {
+                                                           const float* z_topk, float* c2, float* sgn, float* fix) {
   const int lane = threadIdx.x & 31;
   const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (t >= p.T) return;
@@ -155,9 +184,11 @@ __global__ void __launch_bounds__(256) fused_scalar_kernel(RowParams p, const fl
       double pi_a;
       int f2 = 0;
       const float za = z_a[t];
-      auto z_at = [&](int) { return za; };          // Binary variants only touch the sampled id
+      const float* zk = z_topk ? z_topk + t * (int64_t)p.K : nullptr;
+      auto z_at = [&](int, int k) { return k < 0 ? za : zk[k]; };   // sampled id, or position k of the top-K list
       row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
-      coef = make_coef(g, lse, pi_a);
+      if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
+      else coef = make_coef(g, lse, pi_a);
     }
   }
   if (lane == 0) {
@@ -177,11 +208,11 @@ constexpr size_t kAlign = 256;
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct FusedLayout {
-  size_t wt, ht, P, Pt, part, z_a, c2, sgn, fix, loss_ws, total;
+  size_t wt, ht, P, Pt, part, z_a, z_topk, c2, sgn, fix, loss_ws, total;
   int64_t ldp, ldt;
   int tiles_n;
 };
-FusedLayout fused_layout(int64_t T, int64_t d, int64_t V) {
+FusedLayout fused_layout(int64_t T, int64_t d, int64_t V, int K) {
   FusedLayout L;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += round_up(bytes ? bytes : 1, kAlign); return o; };
@@ -194,6 +225,7 @@ FusedLayout fused_layout(int64_t T, int64_t d, int64_t V) {
   L.Pt = take((size_t)V * L.ldt * 2);
   L.part = take((size_t)T * L.tiles_n * sizeof(float2));
   L.z_a = take((size_t)T * 4);
+  L.z_topk = take((size_t)T * (K > 0 ? K : 0) * 4);
   L.c2 = take((size_t)T * 4);
   L.sgn = take((size_t)T * 4);
   L.fix = take((size_t)T * 4);
@@ -207,9 +239,9 @@ FusedLayout fused_layout(int64_t T, int64_t d, int64_t V) {
 
 extern "C" {
 
-size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V) {
-  if (T < 0 || d < 1 || V < 1) return 0;
-  return dppo::fused_layout(T, d, V).total;
+size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V, int K) {
+  if (T < 0 || d < 1 || V < 1 || K < 0) return 0;
+  return dppo::fused_layout(T, d, V, K).total;
 }
 
 int dppo_gemm_tn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,
@@ -226,28 +258,33 @@ int dppo_gemm_tn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, in
 }
 
 int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int64_t d, int64_t V,
-                              const int32_t* sampled_ids, const float* mu_logp, const float* advantages,
-                              const uint8_t* token_mask, int variant, float delta, const dppo_opts* opts,
+                              const int32_t* sampled_ids, const float* mu_logp,
+                              const int32_t* mu_topk_ids, const float* mu_topk_p, const float* advantages,
+                              const uint8_t* token_mask, int variant, int K, float delta, const dppo_opts* opts,
                               float* loss, float* divergence, uint8_t* mask, float* dHidden, float* dW,
                               float* stats, int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   using namespace dppo;
   dppo_opts o = {};
   if (opts) o = *opts;
   if (T < 0 || d < 1 || V < 1 || T > (int64_t)1 << 30 || V > (int64_t)1 << 30 || d > (int64_t)1 << 30) return DPPO_ERR_SHAPE;
-  if (variant != DPPO_BINARY_TV && variant != DPPO_BINARY_KL && variant != DPPO_PPO_CLIP && variant != DPPO_MINIMAL_MASK)
-    return DPPO_ERR_VARIANT;
+  if (variant < DPPO_BINARY_TV || variant > DPPO_MINIMAL_MASK) return DPPO_ERR_VARIANT;
+  const bool topk = (variant == DPPO_TOPK_TV || variant == DPPO_TOPK_KL);
+  if (!topk) K = 0;
+  if (K < 0 || (int64_t)K > V) return DPPO_ERR_SHAPE;
+  if (topk && K > 0 && T > 0 && (!mu_topk_ids || !mu_topk_p)) return DPPO_ERR_TOPK;
   if (!loss || !status || !W || !dW) return DPPO_ERR_NULL;
   if (T > 0 && (!hidden || !sampled_ids || !mu_logp || !advantages || !divergence || !mask || !dHidden)) return DPPO_ERR_NULL;
   if (((uintptr_t)hidden % 16) || ((uintptr_t)W % 16) || (d % 8) || (V % 8)) return DPPO_ERR_ALIGN;
   if (((uintptr_t)dHidden % 16) || ((uintptr_t)dW % 16)) return DPPO_ERR_ALIGN;
-  const FusedLayout L = fused_layout(T, d, V);
+  const FusedLayout L = fused_layout(T, d, V, K);
   if (!workspace || ((uintptr_t)workspace % kAlign) || workspace_bytes < L.total) return DPPO_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   char* ws = reinterpret_cast<char*>(workspace);
 
   RowParams p = {};
   p.T = T; p.V = V; p.sampled_ids = sampled_ids; p.mu_logp = mu_logp; p.adv = advantages; p.token_mask = token_mask;
-  p.variant = variant; p.K = 0; p.delta = delta; p.loss_scale = o.loss_scale; p.is_cap = o.is_cap; p.eps_low = o.eps_low;
+  p.variant = variant; p.K = K; p.topk_ids = mu_topk_ids; p.topk_p = mu_topk_p;
+  p.delta = delta; p.loss_scale = o.loss_scale; p.is_cap = o.is_cap; p.eps_low = o.eps_low;
   p.divergence = divergence; p.mask = mask; p.loss = loss; p.stats = stats; p.status = status;
   char* lws = ws + L.loss_ws;
   const size_t per = round_up((size_t)T * sizeof(float), kAlign);
@@ -276,7 +313,14 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   g1.M = (int)T; g1.N = (int)V; g1.K = (int)d; g1.part = part; g1.z_a = z_a; g1.ids = sampled_ids; g1.status = status;
   DPPO_TRY(launch_gemm<gemm::EPI_STATS>(hidden, d, ws + L.wt, d, g1, st));
   // 3. per-row scalars, loss
-  fused_scalar_kernel<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(p, part, L.tiles_n, z_a, c2, sgn, fix);
+  float* z_topk = nullptr;
+  if (K > 0) {      // logits at the rollout policy's top-K ids: T x K dot products against rows of W^T
+    z_topk = reinterpret_cast<float*>(ws + L.z_topk);
+    fused_topk_logits_kernel<<<(unsigned)((T * K + 7) / 8), 256, 0, st>>>(
+        reinterpret_cast<const __nv_bfloat16*>(hidden), reinterpret_cast<const __nv_bfloat16*>(ws + L.wt), T, d, V, mu_topk_ids, K, z_topk);
+    DPPO_TRY(cudaGetLastError());
+  }
+  fused_scalar_kernel<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(p, part, L.tiles_n, z_a, z_topk, c2, sgn, fix);
   DPPO_TRY(cudaGetLastError());
   DPPO_TRY(launch_finalize(p, st));
   // 4. gradient with respect to the logits, bf16, [T, ldp]

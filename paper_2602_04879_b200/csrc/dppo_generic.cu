@@ -158,7 +158,7 @@ __global__ void __launch_bounds__(kGenericThreads) dppo_row_generic_kernel(RowPa
         } else {
           double pi_a;
           int f2 = 0;
-          auto z_at = [&](int id) { return to_f32<InT>(zrow[id]); };
+          auto z_at = [&](int id, int) { return to_f32<InT>(zrow[id]); };
           row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
           if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
           else coef = make_coef(g, lse, pi_a);

@@ -493,7 +493,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           } else {
             double pi_a;
             int f2 = 0;
-            auto z_at = [&](int id) { return id == a ? z_a : to_f32<InT>(zrow[id]); };
+            auto z_at = [&](int id, int) { return id == a ? z_a : to_f32<InT>(zrow[id]); };
             row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
             if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
             else coef = make_coef(g, lse, pi_a);

@@ -172,13 +172,13 @@ def ragged_response(device, i, lengths, seed=3, max_len=8192, V=QWEN3_VOCAB, dty
                                                                    n_valid_total=int(sum(lengths))))
 
 
-def lm_head_workload(device, seed=5, T=8192, d=2048, V=QWEN3_VOCAB, resp_len=512, sigma_w=0.02, sigma_mu=0.1):
+def lm_head_workload(device, seed=5, T=8192, d=2048, V=QWEN3_VOCAB, resp_len=512, sigma_w=0.02, sigma_mu=0.1, K=0):
     """hidden [T,d] bf16 ~ N(0,1), LM head W [d,V] bf16 ~ sigma_w*N(0,1); the rollout side is built from
     hidden x W (fp32 accumulation, computed here only to generate inputs) + sigma_mu*N(0,1)."""
     g = _gen(device, seed, 0)
     H = torch.randn((T, d), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
     W = (sigma_w * torch.randn((d, V), generator=g, device=device, dtype=torch.float32)).to(torch.bfloat16)
-    a_l, ml_l = [], []
+    a_l, ml_l, id_l, p_l = [], [], [], []
     Wf = W.to(torch.float32) if device == "cpu" or str(device) == "cpu" else None
     for r0 in range(0, T, BLOCK_ROWS):
         n = min(BLOCK_ROWS, T - r0)
@@ -188,11 +188,14 @@ def lm_head_workload(device, seed=5, T=8192, d=2048, V=QWEN3_VOCAB, resp_len=512
         else:
             z = (H[r0:r0 + n] @ W).to(torch.float32)
         z = z + sigma_mu * torch.randn((n, V), generator=gb, device=device, dtype=torch.float32)
-        a, ml, _, _ = _rollout_side(z, 0, gb)
+        a, ml, ids, ps = _rollout_side(z, K, gb)
         a_l.append(a)
         ml_l.append(ml)
+        id_l.append(ids)
+        p_l.append(ps)
     adv = _group_advantages(max(1, T // resp_len), 1, seed, "pm1").repeat_interleave(resp_len)[:T].to(device)
     if adv.shape[0] < T:
         adv = torch.cat([adv, adv.new_ones(T - adv.shape[0])])
-    return Batch(None, torch.cat(a_l), torch.cat(ml_l), adv.contiguous(), None, hidden=H, lm_head=W,
-                 meta=dict(name="lm_head_binary_tv", delta=0.2))
+    return Batch(None, torch.cat(a_l), torch.cat(ml_l), adv.contiguous(), None,
+                 torch.cat(id_l) if K > 0 else None, torch.cat(p_l) if K > 0 else None, hidden=H, lm_head=W,
+                 meta=dict(name="lm_head_binary_tv", delta=0.2, K=K))

@@ -33,21 +33,24 @@ def test_gemm_tn_bf16_matches_fp64_product(M, N, K):
     assert torch.equal(Cw[:, :N], C) and torch.all(Cw[:, N:] == 7.0)
 
 
-def _fused_case(T, d, V, seed, resp_len):
-    b = wl.lm_head_workload(DEV, seed=seed, T=T, d=d, V=V, resp_len=resp_len, sigma_w=0.02 * (2048 / d) ** 0.5)
-    return b
+def _fused_case(T, d, V, seed, resp_len, K=0, sigma_w=None):
+    sw = 0.02 * (2048 / d) ** 0.5 if sigma_w is None else sigma_w
+    return wl.lm_head_workload(DEV, seed=seed, T=T, d=d, V=V, resp_len=resp_len, sigma_w=sw, K=K)
 
 
-def _check_fused(b, variant, delta, tok=None):
+def _check_fused(b, variant, delta, tok=None, K=0, is_cap=0.0):
     out = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, tok, variant, delta,
-                                         want_stats=True)
+                                         want_stats=True, K=K, mu_topk_ids=b.mu_topk_ids, mu_topk_p=b.mu_topk_p, is_cap=is_cap)
     torch.cuda.synchronize()
     assert int(out["status"].item()) == 0
     H = b.hidden.float().cpu().numpy().astype(np.float64)
     W = b.lm_head.float().cpu().numpy().astype(np.float64)
     tokh = None if tok is None else tok.cpu().numpy()
     ora = O.dppo_fused_lmhead_fwd_bwd(H, W, b.sampled_ids.cpu().numpy(), b.mu_logp.cpu().numpy().astype(np.float64),
-                                      b.advantages.cpu().numpy().astype(np.float64), tokh, variant, delta)
+                                      b.advantages.cpu().numpy().astype(np.float64), tokh, variant, delta, None, K,
+                                      None if b.mu_topk_ids is None else b.mu_topk_ids.cpu().numpy(),
+                                      None if b.mu_topk_p is None else b.mu_topk_p.cpu().numpy().astype(np.float64),
+                                      is_cap if is_cap > 0 else None)
     h = dict(token_mask=tokh)
     P.check_scalars(out["divergence"].cpu().numpy(), out["mask"].cpu().numpy(), ora, h, delta)
     P.check_loss(float(out["loss"].item()), ora["loss"], True, ora["row_loss"])
@@ -79,10 +82,39 @@ def test_fused_matches_oracle_small(T, d, V):
     _check_fused(b, dppo.BINARY_KL, 1e-9, tok)
 
 
+@pytest.mark.parametrize("variant", [dppo.TOPK_TV, dppo.TOPK_KL])
+def test_fused_topk_variants_match_oracle(variant):
+    """Top-K divergences in the fused path: peaked logits (larger LM-head scale) so that the top-K lists carry mass."""
+    T, d, V, K = 256, 128, 2048, 20
+    b = _fused_case(T, d, V, seed=43, resp_len=8, K=K, sigma_w=0.35)
+    out, ora = _check_fused(b, variant, 1.0, K=K)
+    Dm = np.sort(ora["D"])
+    gaps = Dm[T // 2 - 6:T // 2 + 6]
+    i = int(np.argmax(np.diff(gaps)))
+    delta = float(np.float32(0.5 * (gaps[i] + gaps[i + 1])))
+    tok = (torch.arange(T, device=DEV) % 5 != 1).to(torch.uint8)
+    out2, ora2 = _check_fused(b, variant, delta, tok, K=K, is_cap=1.05)
+    valid = tok.cpu().numpy() != 0
+    assert 0 < int(((ora2["M"] == 0) & valid).sum()) < int(valid.sum())
+    # App. B: Top-K refines Binary
+    bin_out = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, variant - 2, 1.0)
+    assert torch.all(bin_out["divergence"] <= out["divergence"] + 1e-5)      # equality happens; 1e-5 is the tolerance of D
+    # an out-of-range list entry raises the status bit and drops the row
+    bad = b.mu_topk_ids.clone()
+    bad[7, 3] = V + 5
+    o3 = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, variant, 1.0,
+                                        K=K, mu_topk_ids=bad, mu_topk_p=b.mu_topk_p)
+    torch.cuda.synchronize()
+    assert int(o3["status"].item()) == dppo.binding.STATUS_BAD_TOPK_ID and not o3["dHidden"][7].any()
+
+
 def test_fused_rejects_misuse():
     b = _fused_case(128, 64, 512, seed=42, resp_len=8)
     with pytest.raises(dppo.DppoError) as e:
-        dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.TOPK_TV, 0.2)
+        dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.TOPK_TV, 0.2, K=4)
+    assert e.value.code == -5
+    with pytest.raises(dppo.DppoError) as e:
+        dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, 9, 0.2)
     assert e.value.code == -4
     with pytest.raises(dppo.DppoError) as e:
         dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.BINARY_TV, 0.2,
