@@ -104,7 +104,7 @@ def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one full-size launch of the row kernel, from the ncu
-# capture summarised in profiles/dppo_row_ring_kernel_bf16_V151936.md, and the hash of the kernel sources it was
+# capture summarised under profiles/ (row ring kernel, V = 151936), and the hash of the kernel sources it was
 # taken with: once the kernel changes the figure no longer applies and None is reported.
 TRAFFIC_BYTES_PER_LAUNCH = 5514331733 + 4917249707
 TRAFFIC_KERNEL_SHA = "72311896fc13c8ed"

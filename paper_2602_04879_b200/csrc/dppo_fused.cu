@@ -64,7 +64,12 @@ cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, 
   cudaError_t e = cudaFuncSetAttribute(gemm::gemm_tn_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int64_t ntiles = (int64_t)((p.M + gemm::BM - 1) / gemm::BM) * ((p.N + gemm::BN - 1) / gemm::BN);
-  const int grid = (int)(ntiles < sms ? ntiles : sms);
+  if (EPI == gemm::EPI_STORE_F32 && p.splits > 1) {
+    cudaError_t ez = cudaMemset2DAsync(p.C, (size_t)p.ldc * sizeof(float), 0, (size_t)p.N * sizeof(float), (size_t)p.M, st);
+    if (ez != cudaSuccess) return ez;
+  }
+  const int64_t nunits = ntiles * ((EPI == gemm::EPI_STORE_F32 && p.splits > 1) ? p.splits : 1);
+  const int grid = (int)(nunits < sms ? nunits : sms);
   gemm::gemm_tn_kernel<EPI><<<grid, gemm::THREADS, gemm::SMEM_BYTES, st>>>(ma, mb, p);
   return cudaGetLastError();
 }
@@ -332,6 +337,17 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   // 6. dHidden[T, d] = P[T, V] . W[d, V]^T
   gemm::Params g3 = {};
   g3.M = (int)T; g3.N = (int)d; g3.K = (int)V; g3.C = dHidden; g3.ldc = d; g3.status = status;
+  {
+    // Few output tiles, very long K: when the tiles do not fill whole waves of SMs, cut K in two so that the halves do
+    // (two partial sums added into zeros: the result does not depend on which lands first).
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int64_t tiles = ((T + gemm::BM - 1) / gemm::BM) * ((d + gemm::BN - 1) / gemm::BN);
+    const double eff1 = (double)tiles / (double)(((tiles + sms - 1) / sms) * sms);
+    const double eff2 = (double)(2 * tiles) / (double)(((2 * tiles + sms - 1) / sms) * sms);
+    g3.splits = (eff2 > eff1 + 0.05 && V >= 4 * gemm::BK) ? 2 : 1;
+  }
   DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(ws + L.P, L.ldp, W, V, g3, st));
   // 7. dW[d, V] = hidden^T[d, T] . P^T[V, T]^T
   gemm::Params g4 = {};

@@ -36,6 +36,7 @@ struct Params {
   // EPI_STORE_F32
   float* C;
   int64_t ldc;
+  int splits;            // EPI_STORE_F32: K is cut into this many parts whose results are added into a zeroed C (0/1: none)
   // EPI_STATS: per (row, n-tile) partial (max, sum exp(z - max)); z at the sampled id
   float2* part;          // [M, tiles_n]
   float* z_a;            // [M]
@@ -159,6 +160,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
   const int ntiles = tiles_m * tiles_n;
   const int kblocks = (p.K + BK - 1) / BK;
+  // work unit u = part * ntiles + tile: all tiles of one K part are in flight together and share operand strips
+  const int splits = (EPI == EPI_STORE_F32 && p.splits > 1) ? p.splits : 1;
+  const int kper = (kblocks + splits - 1) / splits;
+  const int nunits = ntiles * splits;
   const uint32_t smem_base = smem_addr(smem);
 
   if (warp == 0) {
@@ -167,9 +172,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+      for (int u = blockIdx.x; u < nunits && ok; u += gridDim.x) {
+        const int tile = u % ntiles, part = u / ntiles;
         const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
-        for (int kb = 0; kb < kblocks; ++kb) {
+        const int kb0 = part * kper, kb1 = (kb0 + kper < kblocks) ? kb0 + kper : kblocks;
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!bar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = smem_base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
           bar_expect_tx(full0 + 8 * s, STAGE_BYTES);
@@ -186,19 +193,21 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       uint32_t ph = 0;
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+      for (int u = blockIdx.x; u < nunits && ok; u += gridDim.x, ++it) {
+        const int part = u / ntiles;
+        const int kb0 = part * kper, kb1 = (kb0 + kper < kblocks) ? kb0 + kper : kblocks;
         const uint32_t b = it & 1u, use = it >> 1;
         if (!bar_wait(tempty0 + 8 * b, (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }   // epilogue drained this buffer
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t tmem_c = tmem_base + b * BN;
-        for (int kb = 0; kb < kblocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!bar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t a_src = smem_base + s * STAGE_BYTES, b_src = a_src + A_STAGE_BYTES;
           const uint64_t adesc = make_desc_k_sw128(a_src), bdesc = make_desc_k_sw128(b_src);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)      // 32 bytes (16 bf16) further along K inside the swizzle atom per step
-            mma_bf16(tmem_c, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), (kb | k) != 0 ? 1u : 0u);
+            mma_bf16(tmem_c, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), (kb != kb0 || k != 0) ? 1u : 0u);
           mma_commit(empty0 + 8 * s);            // stage free once these MMAs have read it
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
@@ -209,7 +218,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
     // ------------------------------------------------------------------ epilogue warps (TMEM lane quarter = warp % 4)
     const int q = warp & 3;
     uint32_t it = 0;
-    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
+    for (int u = blockIdx.x; u < nunits; u += gridDim.x, ++it) {
+      const int tile = u % ntiles;
       const int m0 = (tile % tiles_m) * BM, nb = tile / tiles_m, n0 = nb * BN;
       const uint32_t b = it & 1u, use = it >> 1;
       const bool ok = __all_sync(0xffffffffu, bar_wait(tfull0 + 8 * b, use & 1u, abort_flag));
@@ -225,7 +235,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
           tmem_ld32(taddr + c, r);
           if (row_ok) {
             float* dst = p.C + (int64_t)row * p.ldc + n0 + c;
-            if (n0 + c + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+            if (splits > 1) {              // partial sum over a K part: add into the zeroed output
+#pragma unroll
+              for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) atomicAdd(dst + j, __uint_as_float(r[j]));
+            } else if (n0 + c + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
 #pragma unroll
               for (int j = 0; j < 32; j += 4) *reinterpret_cast<uint4*>(dst + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
             } else {
