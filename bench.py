@@ -100,7 +100,7 @@ def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
             "roofline": {"bound": "tensor", "achieved": useful, "peak": peak, "unit": "TFLOP/s", "frac": useful / peak,
                          "executed_tflops": executed, "executed_frac": executed / peak, "traffic": None,
                          "peak_source": "of " + src, "flop_count": "useful = 6*T*d*V (forward, dHidden, dW); executed = 8*T*d*V with the recomputed logits"},
-            "gpu_launches_per_step": 10, "loss": float(out["loss"].item())}
+            "gpu_launches_per_step": 8, "loss": float(out["loss"].item())}
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one full-size launch of the row kernel, from the ncu

@@ -216,8 +216,8 @@ size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V, int K);
  *           logits per row are recomputed as dot products, K is ignored by the other variants).
  *  dHidden  [T, d] fp32 out: d loss / d hidden = dlogits . W^T.
  *  dW       [d, V] fp32 out: d loss / d W = hidden^T . dlogits (overwritten, not accumulated).
- *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V, K) bytes; it holds W^T, hidden^T, the
- *           bf16 gradient with respect to the logits and its transpose (about 4 T V + 2 d V bytes).
+ *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V, K) bytes; it holds hidden^T and the
+ *           bf16 gradient with respect to the logits (about 2 T V bytes; plus W^T, 2 d V bytes, for Top-K variants).
  * The gradient with respect to the logits is rounded to bf16 before the two gradient GEMMs (fp32 accumulation).
  */
 int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int64_t d, int64_t V,
@@ -234,6 +234,10 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
  * bounded wait that ran out (may be NULL).
  */
 int dppo_gemm_tn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,
+                      int32_t* status, void* cuda_stream);
+
+/* The same with B given as [K, N] row-major (N contiguous, row stride ldb): C[M, N] = A[M, K] . B[K, N]. */
+int dppo_gemm_nn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,
                       int32_t* status, void* cuda_stream);
 
 /*

@@ -71,6 +71,8 @@ def lib():
         L.dppo_gemm_tn_bf16.restype = c_int
         L.dppo_gemm_tn_bf16.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_int, c_int, c_int, c_void_p, c_int64,
                                         c_void_p, c_void_p]
+        L.dppo_gemm_nn_bf16.restype = c_int
+        L.dppo_gemm_nn_bf16.argtypes = L.dppo_gemm_tn_bf16.argtypes
         L.dppo_loss_fwd_bwd_static_ws.restype = c_int
         L.dppo_loss_fwd_bwd_static_ws.argtypes = L.dppo_loss_fwd_bwd.argtypes[:22] + [c_void_p]
         _lib = L
@@ -219,6 +221,25 @@ def dppo_gemm_tn_bf16(A, B, C=None, status=None, stream=None):
                                      c_void_p(st.cuda_stream))
     if rc != 0:
         raise DppoError(rc, "dppo_gemm_tn_bf16")
+    return C, status
+
+
+def dppo_gemm_nn_bf16(A, B, C=None, status=None, stream=None):
+    """C[M,N] fp32 = A[M,K] . B[K,N] for bf16 CUDA matrices (last dimension contiguous)."""
+    assert A.is_cuda and B.is_cuda and A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16
+    assert A.stride(1) == 1 and B.stride(1) == 1 and A.shape[1] == B.shape[0]
+    M, K = A.shape
+    N = B.shape[1]
+    if C is None:
+        C = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=A.device)
+    st = stream if stream is not None else torch.cuda.current_stream(A.device)
+    with torch.cuda.device(A.device):
+        rc = lib().dppo_gemm_nn_bf16(_ptr(A), A.stride(0), _ptr(B), B.stride(0), M, N, K, _ptr(C), C.stride(0), _ptr(status),
+                                     c_void_p(st.cuda_stream))
+    if rc != 0:
+        raise DppoError(rc, "dppo_gemm_nn_bf16")
     return C, status
 
 

@@ -1,18 +1,18 @@
 // Fused LM-head variant of the DPPO loss: logits = hidden x W are produced tile by tile on the tensor cores and
 // consumed in the accumulators' epilogue, so the [T, V] logits never exist in memory.
 //
-//   1. W^T, hidden^T  (bf16 transposes: every GEMM below then has both operands K-major)
-//   2. stats GEMM     z-tile = hidden . W^T-tile; epilogue: per-row (max, sum exp) of the tile, z at the sampled id
+//   1. hidden^T       (bf16 transpose, 2 T d bytes; W^T only for the Top-K variants' gather)
+//   2. stats GEMM     z-tile = hidden . W-tile (B = W [d, V] as an MN-major operand); epilogue: per-row (max, sum exp)
+//                     of the tile, z at the sampled id
 //   3. scalar kernel  merge the tiles' partials -> lse; ratio, divergence, mask, loss term, gradient coefficients
 //                     (Top-K variants: the K logits per row come from a small gather-dot kernel over rows of W^T)
-//   4. grad GEMM      the same tiles again; epilogue: P = dlogits = g (softmax - onehot) in bf16,
-//   5.                written both as P [T, V] and as P^T [V, T]
-//   6. dHidden = P . W     (A = P [T,V], B = W [d,V])          fp32
-//   7. dW = hidden^T . P   (A = hidden^T [d,T], B = P^T [V,T])  fp32
+//   4. grad GEMM      the same tiles again; epilogue: P = dlogits = g (softmax - onehot) in bf16, [T, V]
+//   5. dHidden = P . W^T   (A = P [T,V], B = W [d,V] K-major)                 fp32
+//   6. dW = hidden^T . P   (A = hidden^T [d,T], B = P [T,V] as MN-major)      fp32
 //
 // dHidden and dW are d = thousands of columns wide, far more than the 512 accumulator columns of tensor memory, so they
 // cannot be accumulated on chip across the vocabulary; the bf16 gradient P (not the logits) is therefore staged in the
-// caller's workspace between steps 4 and 6/7.
+// caller's workspace between steps 4 and 5/6.
 #include <mutex>
 
 #include "dppo_common.cuh"
@@ -46,22 +46,24 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
   if (!enc) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {(cuuint32_t)gemm::BK, (cuuint32_t)box_rows};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};       // 64 bf16 = 128 bytes = the swizzle span
   cuuint32_t estr[2] = {1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int EPI>
+// B_MN = false: B is [N, K] with leading dimension ldb; B_MN = true: B is [K, N] with leading dimension ldb.
+template <int EPI, bool B_MN = false>
 cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
   if (p.M <= 0 || p.N <= 0 || p.K <= 0) return cudaSuccess;
   CUtensorMap ma, mb;
-  if (!make_map(&ma, A, p.M, p.K, lda, gemm::BM) || !make_map(&mb, B, p.N, p.K, ldb, gemm::BN)) return cudaErrorInvalidValue;
+  if (!make_map(&ma, A, p.M, p.K, lda, gemm::BM)) return cudaErrorInvalidValue;
+  if (!(B_MN ? make_map(&mb, B, p.K, p.N, ldb, gemm::BK) : make_map(&mb, B, p.N, p.K, ldb, gemm::BN))) return cudaErrorInvalidValue;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  cudaError_t e = cudaFuncSetAttribute(gemm::gemm_tn_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::SMEM_BYTES);
+  cudaError_t e = cudaFuncSetAttribute(gemm::gemm_tn_kernel<EPI, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int64_t ntiles = (int64_t)((p.M + gemm::BM - 1) / gemm::BM) * ((p.N + gemm::BN - 1) / gemm::BN);
   if (EPI == gemm::EPI_STORE_F32 && p.splits > 1) {
@@ -70,7 +72,7 @@ cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, 
   }
   const int64_t nunits = ntiles * ((EPI == gemm::EPI_STORE_F32 && p.splits > 1) ? p.splits : 1);
   const int grid = (int)(nunits < sms ? nunits : sms);
-  gemm::gemm_tn_kernel<EPI><<<grid, gemm::THREADS, gemm::SMEM_BYTES, st>>>(ma, mb, p);
+  gemm::gemm_tn_kernel<EPI, B_MN><<<grid, gemm::THREADS, gemm::SMEM_BYTES, st>>>(ma, mb, p);
   return cudaGetLastError();
 }
 
@@ -224,10 +226,10 @@ FusedLayout fused_layout(int64_t T, int64_t d, int64_t V, int K) {
   L.ldp = (V + 7) / 8 * 8;
   L.ldt = (T + 7) / 8 * 8;
   L.tiles_n = (int)((V + gemm::BN - 1) / gemm::BN);
-  L.wt = take((size_t)V * d * 2);
+  L.wt = take(K > 0 ? (size_t)V * d * 2 : 0);      // W^T is only needed to gather the top-K logits
   L.ht = take((size_t)d * L.ldt * 2);
   L.P = take((size_t)T * L.ldp * 2);
-  L.Pt = take((size_t)V * L.ldt * 2);
+  L.Pt = 0;
   L.part = take((size_t)T * L.tiles_n * sizeof(float2));
   L.z_a = take((size_t)T * 4);
   L.z_topk = take((size_t)T * (K > 0 ? K : 0) * 4);
@@ -259,6 +261,19 @@ int dppo_gemm_tn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, in
   dppo::gemm::Params p = {};
   p.M = M; p.N = N; p.K = K; p.C = C; p.ldc = ldc; p.status = status;
   return dppo::launch_gemm<dppo::gemm::EPI_STORE_F32>(A, lda, B, ldb, p, reinterpret_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? DPPO_OK : DPPO_ERR_CUDA;
+}
+
+int dppo_gemm_nn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,
+                      int32_t* status, void* cuda_stream) {
+  if (M < 0 || N < 0 || K < 0) return DPPO_ERR_SHAPE;
+  if (M == 0 || N == 0) return DPPO_OK;
+  if (!A || !B || !C) return DPPO_ERR_NULL;
+  if (lda < K || ldb < N || ldc < N) return DPPO_ERR_STRIDE;
+  if (((uintptr_t)A % 16) || ((uintptr_t)B % 16) || (lda % 8) || (ldb % 8) || ((uintptr_t)C % 4)) return DPPO_ERR_ALIGN;
+  dppo::gemm::Params p = {};
+  p.M = M; p.N = N; p.K = K; p.C = C; p.ldc = ldc; p.status = status;
+  return dppo::launch_gemm<dppo::gemm::EPI_STORE_F32, true>(A, lda, B, ldb, p, reinterpret_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
              ? DPPO_OK : DPPO_ERR_CUDA;
 }
 
@@ -310,13 +325,13 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   float *z_a = reinterpret_cast<float*>(ws + L.z_a), *c2 = reinterpret_cast<float*>(ws + L.c2);
   float *sgn = reinterpret_cast<float*>(ws + L.sgn), *fix = reinterpret_cast<float*>(ws + L.fix);
   // 1. transposes of the operands
-  DPPO_TRY(transpose_bf16(W, d, V, V, ws + L.wt, d, st));
+  if (K > 0) DPPO_TRY(transpose_bf16(W, d, V, V, ws + L.wt, d, st));
   DPPO_TRY(transpose_bf16(hidden, T, d, d, ws + L.ht, L.ldt, st));
   // 2. statistics of the logits
   DPPO_TRY(cudaMemsetAsync(z_a, 0, (size_t)T * 4, st));
   gemm::Params g1 = {};
   g1.M = (int)T; g1.N = (int)V; g1.K = (int)d; g1.part = part; g1.z_a = z_a; g1.ids = sampled_ids; g1.status = status;
-  DPPO_TRY(launch_gemm<gemm::EPI_STATS>(hidden, d, ws + L.wt, d, g1, st));
+  DPPO_TRY((launch_gemm<gemm::EPI_STATS, true>(hidden, d, W, V, g1, st)));      // B = W [d, V], MN-major
   // 3. per-row scalars, loss
   float* z_topk = nullptr;
   if (K > 0) {      // logits at the rollout policy's top-K ids: T x K dot products against rows of W^T
@@ -332,9 +347,8 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   gemm::Params g2 = {};
   g2.M = (int)T; g2.N = (int)V; g2.K = (int)d; g2.ids = sampled_ids; g2.c2 = c2; g2.sgn = sgn; g2.fix = fix;
   g2.P = reinterpret_cast<__nv_bfloat16*>(ws + L.P); g2.ldp = L.ldp; g2.status = status;
-  g2.Pt = reinterpret_cast<__nv_bfloat16*>(ws + L.Pt); g2.ldpt = L.ldt;       // 5. P^T comes out of the same epilogue
-  DPPO_TRY(launch_gemm<gemm::EPI_GRAD>(hidden, d, ws + L.wt, d, g2, st));
-  // 6. dHidden[T, d] = P[T, V] . W[d, V]^T
+  DPPO_TRY((launch_gemm<gemm::EPI_GRAD, true>(hidden, d, W, V, g2, st)));
+  // 5. dHidden[T, d] = P[T, V] . W[d, V]^T
   gemm::Params g3 = {};
   g3.M = (int)T; g3.N = (int)d; g3.K = (int)V; g3.C = dHidden; g3.ldc = d; g3.status = status;
   {
@@ -349,10 +363,10 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
     g3.splits = (eff2 > eff1 + 0.05 && V >= 4 * gemm::BK) ? 2 : 1;
   }
   DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(ws + L.P, L.ldp, W, V, g3, st));
-  // 7. dW[d, V] = hidden^T[d, T] . P^T[V, T]^T
+  // 6. dW[d, V] = hidden^T[d, T] . P[T, V]
   gemm::Params g4 = {};
   g4.M = (int)d; g4.N = (int)V; g4.K = (int)T; g4.C = dW; g4.ldc = V; g4.status = status;
-  DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(ws + L.ht, L.ldt, ws + L.Pt, L.ldt, g4, st));
+  DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(ws + L.ht, L.ldt, ws + L.P, L.ldp, g4, st)));   // B = P [T, V], MN-major
 #undef DPPO_TRY
   return DPPO_OK;
 }

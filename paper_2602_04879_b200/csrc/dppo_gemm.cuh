@@ -100,13 +100,26 @@ __device__ __forceinline__ uint64_t make_desc_k_sw128(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                          // layout type: 128-byte swizzle
   return d;
 }
-// Instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 128.
+// Shared-memory matrix descriptor of an MN-major operand tile (the operand is stored [K, MN] with MN contiguous): the
+// tile is a row of 64-element (128-byte) wide column blocks, each block 64 k-rows of 128 bytes (8 KB, swizzled in 8-row
+// groups of 1024 bytes); consecutive blocks along MN are `block_bytes` apart.
+__device__ __forceinline__ uint64_t make_desc_mn_sw128(uint32_t saddr, uint32_t block_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);       // start address, 16-byte units
+  d |= (uint64_t)(block_bytes >> 4) << 16;         // leading byte offset: next 64-element block along MN
+  d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset: next group of 8 k-rows
+  d |= (uint64_t)1 << 46;                          // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                          // layout type: 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: D = f32, A = B = bf16, A K-major, B K-major or MN-major (bit 16), N = 256, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+constexpr uint32_t kIdescBmn = kIdesc | (1u << 16);
 
-__device__ __forceinline__ void mma_bf16(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+__device__ __forceinline__ void mma_bf16(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-      ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate) : "memory");
+      ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -128,7 +141,9 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-template <int EPI>
+// B_MN = false: B given as [N, K] (K contiguous).  B_MN = true: B given as [K, N] (N contiguous, "NN" product); its tile is
+// then loaded as four boxes of 64 columns x 64 k-rows.
+template <int EPI, bool B_MN>
 __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a,
                                                              const __grid_constant__ CUtensorMap map_b, Params p) {
   extern __shared__ unsigned char smem_raw[];
@@ -181,7 +196,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
           const uint32_t a_dst = smem_base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
           bar_expect_tx(full0 + 8 * s, STAGE_BYTES);
           tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
-          tma_load_2d(b_dst, &map_b, kb * BK, n0, full0 + 8 * s);
+          if (B_MN) {
+#pragma unroll
+            for (int i = 0; i < BN / 64; ++i) tma_load_2d(b_dst + i * (64 * BK * 2), &map_b, n0 + i * 64, kb * BK, full0 + 8 * s);
+          } else {
+            tma_load_2d(b_dst, &map_b, kb * BK, n0, full0 + 8 * s);
+          }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
       }
@@ -204,10 +224,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
           if (!bar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t a_src = smem_base + s * STAGE_BYTES, b_src = a_src + A_STAGE_BYTES;
-          const uint64_t adesc = make_desc_k_sw128(a_src), bdesc = make_desc_k_sw128(b_src);
+          const uint64_t adesc = make_desc_k_sw128(a_src);
+          const uint64_t bdesc = B_MN ? make_desc_mn_sw128(b_src, 64 * BK * 2) : make_desc_k_sw128(b_src);
+          // per step of 16 along K: K-major operands move 32 bytes inside the swizzle atom, an MN-major one 16 k-rows (2048 bytes)
+          constexpr uint64_t kStepB = B_MN ? (uint64_t)(16 * 128 >> 4) : 2ull;
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)      // 32 bytes (16 bf16) further along K inside the swizzle atom per step
-            mma_bf16(tmem_c, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), (kb != kb0 || k != 0) ? 1u : 0u);
+          for (int k = 0; k < BK / 16; ++k)
+            mma_bf16(tmem_c, adesc + (uint64_t)(k * 2), bdesc + kStepB * k, B_MN ? kIdescBmn : kIdesc, (kb != kb0 || k != 0) ? 1u : 0u);
           mma_commit(empty0 + 8 * s);            // stage free once these MMAs have read it
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }

@@ -33,6 +33,20 @@ def test_gemm_tn_bf16_matches_fp64_product(M, N, K):
     assert torch.equal(Cw[:, :N], C) and torch.all(Cw[:, N:] == 7.0)
 
 
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (128, 256, 256), (300, 520, 200), (256, 1024, 1024), (264, 4104, 1000)])
+def test_gemm_nn_bf16_matches_fp64_product(M, N, K):
+    """B given as [K, N]: the MN-major operand path of the tensor-core GEMM."""
+    g = torch.Generator(device=DEV).manual_seed(M * 5 + N * 11 + K)
+    A = torch.randn((M, K), generator=g, device=DEV).to(torch.bfloat16)
+    B = torch.randn((K, N), generator=g, device=DEV).to(torch.bfloat16)
+    C, status = dppo.dppo_gemm_nn_bf16(A, B)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = A.double().cpu().numpy() @ B.double().cpu().numpy()
+    err = np.abs(C.cpu().numpy() - ref).max()
+    assert err <= 2e-5 * np.abs(ref).max() + 1e-4, err
+
+
 def _fused_case(T, d, V, seed, resp_len, K=0, sigma_w=None):
     sw = 0.02 * (2048 / d) ** 0.5 if sigma_w is None else sigma_w
     return wl.lm_head_workload(DEV, seed=seed, T=T, d=d, V=V, resp_len=resp_len, sigma_w=sw, K=K)
