@@ -106,8 +106,8 @@ def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one full-size launch of the row kernel, from the ncu
 # capture summarised under profiles/ (row ring kernel, V = 151936), and the hash of the kernel sources it was
 # taken with: once the kernel changes the figure no longer applies and None is reported.
-TRAFFIC_BYTES_PER_LAUNCH = 5514331733 + 4917249707
-TRAFFIC_KERNEL_SHA = "72311896fc13c8ed"
+TRAFFIC_BYTES_PER_LAUNCH = 5521499819 + 4917211648
+TRAFFIC_KERNEL_SHA = "4f41c1ae413adf92"
 
 
 def measured_traffic():
@@ -175,20 +175,25 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------------------- oracle arm
 
-def oracle_tokens_per_s(rows, seed, variant_code):
-    """Times the float64 oracle, as it stands, on `rows` rows of the workload generated on the CPU."""
+def oracle_tokens_per_s(rows, seed, variant_code, chunk=1024):
+    """Times the float64 oracle, as it stands, on the first `rows` rows of the workload, generated on the CPU and
+    handed over `chunk` rows at a time (bounded host memory); only the oracle calls are timed."""
     import numpy as np
     import torch
     from paper_2602_04879_b200 import workloads as wl
     from oracle import dppo_oracle as O
-    b = wl.qwen_vocab_rows("cpu", seed=seed, rows=rows)
-    z = b.logits.float().numpy().astype(np.float64)
-    ids = b.sampled_ids.numpy()
-    mu = b.mu_logp.numpy().astype(np.float64)
-    adv = b.advantages.numpy().astype(np.float64)
-    t0 = time.perf_counter()
-    O.dppo_loss_fwd_bwd(z, ids, mu, adv, None, variant_code, 0, DELTA, 1.0 / T_ROWS)
-    dt = time.perf_counter() - t0
+    dt = 0.0
+    for row0 in range(0, rows, chunk):
+        n = min(chunk, rows - row0)
+        b = wl.qwen_vocab_rows("cpu", seed=seed, row0=row0, rows=n)
+        z = b.logits.float().numpy().astype(np.float64)
+        ids = b.sampled_ids.numpy()
+        mu = b.mu_logp.numpy().astype(np.float64)
+        adv = b.advantages.numpy().astype(np.float64)
+        t0 = time.perf_counter()
+        O.dppo_loss_fwd_bwd(z, ids, mu, adv, None, variant_code, 0, DELTA, 1.0 / T_ROWS)
+        dt += time.perf_counter() - t0
+        del b, z
     return rows / dt, dt, torch.get_num_threads()
 
 
@@ -344,7 +349,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import dppo_oracle as O
         code = O.BINARY_TV if args.variant == "binary_tv" else O.BINARY_KL
-        rows = 1536
+        rows = min(T, 12288)                  # about 10 s of float64 numpy at the full size
         tps, dt, _ = oracle_tokens_per_s(rows, 1, code)
         line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": 1, "kind": "oracle",
                                 "sample": f"first {rows} rows of the workload regenerated on the CPU, {dt:.1f} s of float64 numpy"}
