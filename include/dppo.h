@@ -216,9 +216,14 @@ size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V, int K);
  *           logits per row are recomputed as dot products, K is ignored by the other variants).
  *  dHidden  [T, d] fp32 out: d loss / d hidden = dlogits . W^T.
  *  dW       [d, V] fp32 out: d loss / d W = hidden^T . dlogits (overwritten, not accumulated).
- *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V, K) bytes; it holds hidden^T and the
- *           bf16 gradient with respect to the logits (about 2 T V bytes; plus W^T, 2 d V bytes, for Top-K variants).
+ *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V, K) bytes; it holds a packed copy of hidden
+ *           and its transpose and the bf16 gradient with respect to the logits (about 2 T V bytes; plus W^T,
+ *           2 d V bytes, for Top-K variants).
  * The gradient with respect to the logits is rounded to bf16 before the two gradient GEMMs (fp32 accumulation).
+ * Rows whose gradient is zero (token_mask 0, blocked by the trust-region mask, zero advantage) are left out of the three
+ * backward GEMMs: the remaining rows are packed on the device, their count is never read by the host, and the call
+ * stays asynchronous.  Rows with token_mask 0 are left out of the forward GEMM as well.  The outputs are the same as
+ * without packing: such rows of dHidden are zero.
  */
 int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int64_t d, int64_t V,
                               const int32_t* sampled_ids, const float* mu_logp,

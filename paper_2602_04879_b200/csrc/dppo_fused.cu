@@ -1,14 +1,16 @@
 // Fused LM-head variant of the DPPO loss: logits = hidden x W are produced tile by tile on the tensor cores and
 // consumed in the accumulators' epilogue, so the [T, V] logits never exist in memory.
 //
-//   1. hidden^T       (bf16 transpose, 2 T d bytes; W^T only for the Top-K variants' gather)
+//   1. (token mask given) the valid rows of hidden packed together; (Top-K variants) W^T for the gather
 //   2. stats GEMM     z-tile = hidden . W-tile (B = W [d, V] as an MN-major operand); epilogue: per-row (max, sum exp)
 //                     of the tile, z at the sampled id
 //   3. scalar kernel  merge the tiles' partials -> lse; ratio, divergence, mask, loss term, gradient coefficients
 //                     (Top-K variants: the K logits per row come from a small gather-dot kernel over rows of W^T)
-//   4. grad GEMM      the same tiles again; epilogue: P = dlogits = g (softmax - onehot) in bf16, [T, V]
-//   5. dHidden = P . W^T   (A = P [T,V], B = W [d,V] K-major)                 fp32
-//   6. dW = hidden^T . P   (A = hidden^T [d,T], B = P [T,V] as MN-major)      fp32
+//   4. packing        rows with a non-zero gradient, in order, packed together (hidden rows, coefficients) and transposed;
+//                     their count stays on the device and bounds the tile loops of the three GEMMs below
+//   5. grad GEMM      the same tiles again; epilogue: P = dlogits = g (softmax - onehot) in bf16, [rows, V]
+//   6. dHidden = P . W^T   (A = P, B = W [d,V] K-major), rows scattered back        fp32
+//   7. dW = hidden^T . P   (A = packed hidden^T, B = P as MN-major)                 fp32
 //
 // dHidden and dW are d = thousands of columns wide, far more than the 512 accumulator columns of tensor memory, so they
 // cannot be accumulated on chip across the vocabulary; the bf16 gradient P (not the logits) is therefore staged in the
@@ -66,11 +68,15 @@ cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, 
   cudaError_t e = cudaFuncSetAttribute(gemm::gemm_tn_kernel<EPI, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int64_t ntiles = (int64_t)((p.M + gemm::BM - 1) / gemm::BM) * ((p.N + gemm::BN - 1) / gemm::BN);
-  if (EPI == gemm::EPI_STORE_F32 && p.splits > 1) {
+  p.sms = sms;
+  int max_splits = 1;
+  if (EPI == gemm::EPI_STORE_F32) max_splits = p.splits > 1 ? p.splits : (p.splits < 0 ? 2 : 1);
+  // partial sums are added into zeros; with a row map the rows that no tile row maps to stay zero
+  if (EPI == gemm::EPI_STORE_F32 && (max_splits > 1 || p.row_map)) {
     cudaError_t ez = cudaMemset2DAsync(p.C, (size_t)p.ldc * sizeof(float), 0, (size_t)p.N * sizeof(float), (size_t)p.M, st);
     if (ez != cudaSuccess) return ez;
   }
-  const int64_t nunits = ntiles * ((EPI == gemm::EPI_STORE_F32 && p.splits > 1) ? p.splits : 1);
+  const int64_t nunits = ntiles * max_splits;
   const int grid = (int)(nunits < sms ? nunits : sms);
   gemm::gemm_tn_kernel<EPI, B_MN><<<grid, gemm::THREADS, gemm::SMEM_BYTES, st>>>(ma, mb, p);
   return cudaGetLastError();
@@ -157,9 +163,68 @@ __global__ void __launch_bounds__(256) fused_topk_logits_kernel(const __nv_bfloa
   if (lane == 0) z_topk[w] = acc;       // out-of-range ids give 0 here and raise the status bit in the scalar stage
 }
 
+// Stable compaction of the rows to keep (one block): idx[i] = i-th kept row, pos[t] = its place in idx or -1, *n = count.
+// A row is kept when its token_mask byte is non-zero (mask8 given) or when its gradient sign is non-zero (sgn given).
+__global__ void __launch_bounds__(1024) fused_compact_rows_kernel(const uint8_t* mask8, const float* sgn, int64_t T, int32_t* idx,
+                                                                  int32_t* pos, int32_t* n) {
+  __shared__ int warp_tot[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t per = (T + 1023) / 1024;
+  const int64_t t0 = (int64_t)tid * per, t1 = (t0 + per < T) ? t0 + per : T;
+  auto keep = [&](int64_t t) { return mask8 ? (mask8[t] != 0) : (sgn[t] != 0.f); };
+  int cnt = 0;
+  for (int64_t t = t0; t < t1; ++t) cnt += keep(t) ? 1 : 0;
+  int incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int v = warp_tot[lane], w = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int u = __shfl_up_sync(0xffffffffu, w, o); if (lane >= o) w += u; }
+    warp_tot[lane] = w - v;                     // exclusive offset of each warp
+    if (lane == 31) *n = w;
+  }
+  __syncthreads();
+  int at = warp_tot[warp] + incl - cnt;
+  for (int64_t t = t0; t < t1; ++t) {
+    if (keep(t)) { idx[at] = (int32_t)t; pos[t] = at; ++at; }
+    else pos[t] = -1;
+  }
+}
+
+// Row i of the compact copies = row idx[i] of the sources for i < *n, zeros after that (one block per row).
+struct GatherArgs {
+  const int32_t* idx;
+  const int32_t* n;
+  int64_t d;
+  const __nv_bfloat16* src;      // [T, d]
+  __nv_bfloat16* dst;            // [T, d]
+  const int32_t* ids_in;
+  int32_t* ids_out;
+  const float* f_in[3];          // optional per-row floats (null: skipped)
+  float* f_out[3];
+};
+__global__ void __launch_bounds__(256) fused_gather_rows_kernel(GatherArgs g) {
+  const int64_t i = blockIdx.x;
+  const bool live = i < (int64_t)*g.n;
+  const int64_t t = live ? g.idx[i] : 0;
+  const uint4* src = reinterpret_cast<const uint4*>(g.src + t * g.d);
+  uint4* dst = reinterpret_cast<uint4*>(g.dst + i * g.d);
+  for (int64_t j = threadIdx.x; j < g.d / 8; j += blockDim.x) dst[j] = live ? src[j] : make_uint4(0, 0, 0, 0);
+  if (threadIdx.x == 0) {
+    g.ids_out[i] = live ? g.ids_in[t] : 0;
+#pragma unroll
+    for (int k = 0; k < 3; ++k)
+      if (g.f_in[k]) g.f_out[k][i] = live ? g.f_in[k][t] : 0.f;
+  }
+}
+
 // One warp per row: merge the stats GEMM's per-tile partials, then the same scalar stage as the streaming kernels.
+// `pos` (optional) maps a row to its row in the statistics (rows compacted by the token mask; -1: not there).
 __global__ void __launch_bounds__(256) fused_scalar_kernel(RowParams p, const float2* part, int tiles_n, const float* z_a,
-                                                           const float* z_topk, float* c2, float* sgn, float* fix) {
+                                                           const int32_t* pos, const float* z_topk, float* c2, float* sgn, float* fix) {
   const int lane = threadIdx.x & 31;
   const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (t >= p.T) return;
@@ -173,14 +238,16 @@ __global__ void __launch_bounds__(256) fused_scalar_kernel(RowParams p, const fl
   double g = 0.0;
   RowCoef coef;
   coef.c2 = 0.f; coef.sgn = 0.f; coef.fix = 0.f; coef.zero_row = 1;
+  const int64_t ts = pos ? (int64_t)pos[t] : t;       // row of the statistics
+  if (ts < 0) valid = false;
   if (valid) {
     float mm = -INFINITY;
-    for (int i = lane; i < tiles_n; i += 32) mm = fmaxf(mm, part[t * tiles_n + i].x);
+    for (int i = lane; i < tiles_n; i += 32) mm = fmaxf(mm, part[ts * tiles_n + i].x);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
     double S = 0.0;
     for (int i = lane; i < tiles_n; i += 32) {
-      const float2 pr = part[t * tiles_n + i];
+      const float2 pr = part[ts * tiles_n + i];
       if (pr.y > 0.f || pr.y != pr.y) S += (double)pr.y * exp((double)pr.x - (double)mm);
     }
     S = warp_sum(S);
@@ -190,7 +257,7 @@ __global__ void __launch_bounds__(256) fused_scalar_kernel(RowParams p, const fl
     } else {
       double pi_a;
       int f2 = 0;
-      const float za = z_a[t];
+      const float za = z_a[ts];
       const float* zk = z_topk ? z_topk + t * (int64_t)p.K : nullptr;
       auto z_at = [&](int, int k) { return k < 0 ? za : zk[k]; };   // sampled id, or position k of the top-K list
       row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
@@ -215,7 +282,7 @@ constexpr size_t kAlign = 256;
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct FusedLayout {
-  size_t wt, ht, P, Pt, part, z_a, z_topk, c2, sgn, fix, loss_ws, total;
+  size_t wt, ht, hc, P, Pt, part, z_a, z_topk, c2, sgn, fix, c2c, sgnc, fixc, ids_c, idx, pos, nlive, loss_ws, total;
   int64_t ldp, ldt;
   int tiles_n;
 };
@@ -228,6 +295,7 @@ FusedLayout fused_layout(int64_t T, int64_t d, int64_t V, int K) {
   L.tiles_n = (int)((V + gemm::BN - 1) / gemm::BN);
   L.wt = take(K > 0 ? (size_t)V * d * 2 : 0);      // W^T is only needed to gather the top-K logits
   L.ht = take((size_t)d * L.ldt * 2);
+  L.hc = take((size_t)T * d * 2);                  // hidden rows compacted (valid rows, then rows with a gradient)
   L.P = take((size_t)T * L.ldp * 2);
   L.Pt = 0;
   L.part = take((size_t)T * L.tiles_n * sizeof(float2));
@@ -236,6 +304,13 @@ FusedLayout fused_layout(int64_t T, int64_t d, int64_t V, int K) {
   L.c2 = take((size_t)T * 4);
   L.sgn = take((size_t)T * 4);
   L.fix = take((size_t)T * 4);
+  L.c2c = take((size_t)T * 4);                     // the same per-row values in compact row order
+  L.sgnc = take((size_t)T * 4);
+  L.fixc = take((size_t)T * 4);
+  L.ids_c = take((size_t)T * 4);
+  L.idx = take((size_t)T * 4);
+  L.pos = take((size_t)T * 4);
+  L.nlive = take(2 * sizeof(int32_t));
   L.loss_ws = take(dppo_workspace_bytes(T));
   L.total = off;
   return L;
@@ -324,48 +399,71 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   float2* part = reinterpret_cast<float2*>(ws + L.part);
   float *z_a = reinterpret_cast<float*>(ws + L.z_a), *c2 = reinterpret_cast<float*>(ws + L.c2);
   float *sgn = reinterpret_cast<float*>(ws + L.sgn), *fix = reinterpret_cast<float*>(ws + L.fix);
-  // 1. transposes of the operands
+  int32_t *idx = reinterpret_cast<int32_t*>(ws + L.idx), *pos = reinterpret_cast<int32_t*>(ws + L.pos);
+  int32_t *nlive = reinterpret_cast<int32_t*>(ws + L.nlive), *ids_c = reinterpret_cast<int32_t*>(ws + L.ids_c);
+  const __nv_bfloat16* hid = reinterpret_cast<const __nv_bfloat16*>(hidden);
+  __nv_bfloat16* hc = reinterpret_cast<__nv_bfloat16*>(ws + L.hc);
+  auto gather = [&](const int32_t* n, bool coefs) {
+    GatherArgs ga = {};
+    ga.idx = idx; ga.n = n; ga.d = d; ga.src = hid; ga.dst = hc; ga.ids_in = sampled_ids; ga.ids_out = ids_c;
+    if (coefs) {
+      ga.f_in[0] = c2; ga.f_in[1] = sgn; ga.f_in[2] = fix;
+      ga.f_out[0] = reinterpret_cast<float*>(ws + L.c2c); ga.f_out[1] = reinterpret_cast<float*>(ws + L.sgnc);
+      ga.f_out[2] = reinterpret_cast<float*>(ws + L.fixc);
+    }
+    fused_gather_rows_kernel<<<(unsigned)T, 256, 0, st>>>(ga);
+    return cudaGetLastError();
+  };
+  // 1. W^T for the Top-K gather; with a token mask, the valid rows of hidden packed together for the statistics
   if (K > 0) DPPO_TRY(transpose_bf16(W, d, V, V, ws + L.wt, d, st));
-  DPPO_TRY(transpose_bf16(hidden, T, d, d, ws + L.ht, L.ldt, st));
+  const void* a_stats = hidden;
+  const int32_t* ids_stats = sampled_ids;
+  const int32_t *m_stats = nullptr, *pos_stats = nullptr;
+  if (token_mask) {
+    fused_compact_rows_kernel<<<1, 1024, 0, st>>>(token_mask, nullptr, T, idx, pos, nlive);
+    DPPO_TRY(cudaGetLastError());
+    DPPO_TRY(gather(nlive, false));
+    a_stats = hc; ids_stats = ids_c; m_stats = nlive; pos_stats = pos;
+  }
   // 2. statistics of the logits
   DPPO_TRY(cudaMemsetAsync(z_a, 0, (size_t)T * 4, st));
   gemm::Params g1 = {};
-  g1.M = (int)T; g1.N = (int)V; g1.K = (int)d; g1.part = part; g1.z_a = z_a; g1.ids = sampled_ids; g1.status = status;
-  DPPO_TRY((launch_gemm<gemm::EPI_STATS, true>(hidden, d, W, V, g1, st)));      // B = W [d, V], MN-major
+  g1.M = (int)T; g1.N = (int)V; g1.K = (int)d; g1.part = part; g1.z_a = z_a; g1.ids = ids_stats; g1.status = status;
+  g1.m_live = m_stats;
+  DPPO_TRY((launch_gemm<gemm::EPI_STATS, true>(a_stats, d, W, V, g1, st)));      // B = W [d, V], MN-major
   // 3. per-row scalars, loss
   float* z_topk = nullptr;
   if (K > 0) {      // logits at the rollout policy's top-K ids: T x K dot products against rows of W^T
     z_topk = reinterpret_cast<float*>(ws + L.z_topk);
     fused_topk_logits_kernel<<<(unsigned)((T * K + 7) / 8), 256, 0, st>>>(
-        reinterpret_cast<const __nv_bfloat16*>(hidden), reinterpret_cast<const __nv_bfloat16*>(ws + L.wt), T, d, V, mu_topk_ids, K, z_topk);
+        hid, reinterpret_cast<const __nv_bfloat16*>(ws + L.wt), T, d, V, mu_topk_ids, K, z_topk);
     DPPO_TRY(cudaGetLastError());
   }
-  fused_scalar_kernel<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(p, part, L.tiles_n, z_a, z_topk, c2, sgn, fix);
+  fused_scalar_kernel<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(p, part, L.tiles_n, z_a, pos_stats, z_topk, c2, sgn, fix);
   DPPO_TRY(cudaGetLastError());
   DPPO_TRY(launch_finalize(p, st));
-  // 4. gradient with respect to the logits, bf16, [T, ldp]
+  // 4. rows whose gradient is zero (invalid, blocked by the mask, zero advantage) drop out of the backward: the rows
+  //    that remain are packed together, so the three GEMMs below run over *n_act rows instead of T
+  int32_t* n_act = nlive + 1;
+  fused_compact_rows_kernel<<<1, 1024, 0, st>>>(nullptr, sgn, T, idx, pos, n_act);
+  DPPO_TRY(cudaGetLastError());
+  DPPO_TRY(gather(n_act, true));
+  DPPO_TRY(transpose_bf16(hc, T, d, d, ws + L.ht, L.ldt, st));
+  // 5. gradient with respect to the logits of the packed rows, bf16, [T, ldp] (zero rows from *n_act to the tile's end)
   gemm::Params g2 = {};
-  g2.M = (int)T; g2.N = (int)V; g2.K = (int)d; g2.ids = sampled_ids; g2.c2 = c2; g2.sgn = sgn; g2.fix = fix;
-  g2.P = reinterpret_cast<__nv_bfloat16*>(ws + L.P); g2.ldp = L.ldp; g2.status = status;
-  DPPO_TRY((launch_gemm<gemm::EPI_GRAD, true>(hidden, d, W, V, g2, st)));
-  // 5. dHidden[T, d] = P[T, V] . W[d, V]^T
+  g2.M = (int)T; g2.N = (int)V; g2.K = (int)d; g2.ids = ids_c; g2.c2 = reinterpret_cast<float*>(ws + L.c2c);
+  g2.sgn = reinterpret_cast<float*>(ws + L.sgnc); g2.fix = reinterpret_cast<float*>(ws + L.fixc);
+  g2.P = reinterpret_cast<__nv_bfloat16*>(ws + L.P); g2.ldp = L.ldp; g2.status = status; g2.m_live = n_act;
+  DPPO_TRY((launch_gemm<gemm::EPI_GRAD, true>(hc, d, W, V, g2, st)));
+  // 6. dHidden[idx[i], :] = P[i, :] . W[d, V]^T; the other rows stay zero.  Few output tiles, very long K: K is cut in
+  //    two when that fills the waves better (two partial sums added into zeros, in either order the same result).
   gemm::Params g3 = {};
   g3.M = (int)T; g3.N = (int)d; g3.K = (int)V; g3.C = dHidden; g3.ldc = d; g3.status = status;
-  {
-    // Few output tiles, very long K: when the tiles do not fill whole waves of SMs, cut K in two so that the halves do
-    // (two partial sums added into zeros: the result does not depend on which lands first).
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int64_t tiles = ((T + gemm::BM - 1) / gemm::BM) * ((d + gemm::BN - 1) / gemm::BN);
-    const double eff1 = (double)tiles / (double)(((tiles + sms - 1) / sms) * sms);
-    const double eff2 = (double)(2 * tiles) / (double)(((2 * tiles + sms - 1) / sms) * sms);
-    g3.splits = (eff2 > eff1 + 0.05 && V >= 4 * gemm::BK) ? 2 : 1;
-  }
+  g3.m_live = n_act; g3.row_map = idx; g3.splits = -1;
   DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(ws + L.P, L.ldp, W, V, g3, st));
-  // 6. dW[d, V] = hidden^T[d, T] . P[T, V]
+  // 7. dW[d, V] = packed hidden^T[d, n_act] . P[n_act, V]
   gemm::Params g4 = {};
-  g4.M = (int)d; g4.N = (int)V; g4.K = (int)T; g4.C = dW; g4.ldc = V; g4.status = status;
+  g4.M = (int)d; g4.N = (int)V; g4.K = (int)T; g4.C = dW; g4.ldc = V; g4.status = status; g4.k_live = n_act;
   DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(ws + L.ht, L.ldt, ws + L.P, L.ldp, g4, st)));   // B = P [T, V], MN-major
 #undef DPPO_TRY
   return DPPO_OK;

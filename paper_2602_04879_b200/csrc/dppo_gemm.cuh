@@ -36,7 +36,15 @@ struct Params {
   // EPI_STORE_F32
   float* C;
   int64_t ldc;
-  int splits;            // EPI_STORE_F32: K is cut into this many parts whose results are added into a zeroed C (0/1: none)
+  int splits;            // EPI_STORE_F32: K is cut into this many parts whose results are added into a zeroed C (0/1: none;
+                         // < 0: two parts when that fills the waves of `sms` CTAs better, decided from the live tile count)
+  int sms;               // CTAs the split decision assumes (splits < 0)
+  // Live extents, read from device memory at kernel start (null: the static M / K).  Rows of A at and beyond *m_live
+  // get no output tile (at least one tile is always processed); K blocks at and beyond *k_live are not read (at least
+  // one is), so the operands must hold zeros from *k_live to the end of that block.
+  const int* m_live;
+  const int* k_live;
+  const int* row_map;    // EPI_STORE_F32: output row of tile row i (null: i); rows >= *m_live are not stored
   // EPI_STATS: per (row, n-tile) partial (max, sum exp(z - max)); z at the sampled id
   float2* part;          // [M, tiles_n]
   float* z_a;            // [M]
@@ -172,11 +180,23 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+  int m_lim = p.M, k_lim = p.K;
+  if (p.m_live) { const int v = *p.m_live; m_lim = v < 0 ? 0 : (v < p.M ? v : p.M); }
+  if (p.k_live) { const int v = *p.k_live; k_lim = v < 0 ? 0 : (v < p.K ? v : p.K); }
+  const int tiles_m = m_lim > 0 ? (m_lim + BM - 1) / BM : 1, tiles_n = (p.N + BN - 1) / BN;
   const int ntiles = tiles_m * tiles_n;
-  const int kblocks = (p.K + BK - 1) / BK;
+  const int kblocks = k_lim > 0 ? (k_lim + BK - 1) / BK : 1;
   // work unit u = part * ntiles + tile: all tiles of one K part are in flight together and share operand strips
-  const int splits = (EPI == EPI_STORE_F32 && p.splits > 1) ? p.splits : 1;
+  int splits = 1;
+  if (EPI == EPI_STORE_F32) {
+    if (p.splits > 1) splits = p.splits;
+    else if (p.splits < 0 && p.sms > 0 && kblocks >= 8) {
+      // few output tiles, very long K: cut K in two when the halves fill whole waves of CTAs better
+      const float w1 = (float)ntiles / (float)(((ntiles + p.sms - 1) / p.sms) * p.sms);
+      const float w2 = (float)(2 * ntiles) / (float)(((2 * ntiles + p.sms - 1) / p.sms) * p.sms);
+      if (w2 > w1 + 0.05f) splits = 2;
+    }
+  }
   const int kper = (kblocks + splits - 1) / splits;
   const int nunits = ntiles * splits;
   const uint32_t smem_base = smem_addr(smem);
@@ -249,7 +269,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int row = m0 + q * 32 + lane;
-      const bool row_ok = row < p.M;
+      // the gradient epilogue fills its whole tile (zero rows past the live extent feed the next GEMM's last K block)
+      const bool row_ok = (EPI == EPI_STORE_F32) ? row < m_lim : row < p.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * BN;
       if (EPI == EPI_STORE_F32) {
 #pragma unroll 1
@@ -257,7 +278,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
           uint32_t r[32];
           tmem_ld32(taddr + c, r);
           if (row_ok) {
-            float* dst = p.C + (int64_t)row * p.ldc + n0 + c;
+            float* dst = p.C + (int64_t)(p.row_map ? p.row_map[row] : row) * p.ldc + n0 + c;
             if (splits > 1) {              // partial sum over a K part: add into the zeroed output
 #pragma unroll
               for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) atomicAdd(dst + j, __uint_as_float(r[j]));

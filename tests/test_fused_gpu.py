@@ -122,6 +122,37 @@ def test_fused_topk_variants_match_oracle(variant):
     assert int(o3["status"].item()) == dppo.binding.STATUS_BAD_TOPK_ID and not o3["dHidden"][7].any()
 
 
+def test_fused_backward_skips_rows_without_gradient():
+    """Rows with zero advantage, rows blocked by the mask and invalid rows drop out of the backward GEMMs (the kept rows are
+    packed on the device); the outputs must not change: zeros in dHidden for those rows, the same dW."""
+    T, d, V = 600, 128, 1536
+    b = _fused_case(T, d, V, seed=47, resp_len=8)
+    adv = b.advantages.clone()
+    adv[(torch.arange(T, device=DEV) // 8) % 3 == 0] = 0.0           # every third response has zero advantage
+    b.advantages = adv
+    out0, ora0 = _check_fused(b, dppo.BINARY_TV, 0.2)
+    Dm = np.sort(ora0["D"])
+    delta = float(np.float32(0.5 * (Dm[T // 2] + Dm[T // 2 + 1])))
+    tok = (torch.arange(T, device=DEV) % 11 != 4).to(torch.uint8)
+    out, ora = _check_fused(b, dppo.BINARY_TV, delta, tok)
+    zero = (ora["M"] == 0) | (tok.cpu().numpy() == 0) | (adv.cpu().numpy() == 0)
+    kept = int((~zero).sum())
+    assert 0 < kept < T and kept % 64 != 0
+    assert not out["dHidden"][torch.from_numpy(zero).to(DEV)].any()
+    assert out["dHidden"][torch.from_numpy(~zero).to(DEV)].abs().sum(dim=1).min().item() > 0
+    # nothing left at all: zero advantages everywhere
+    b.advantages = torch.zeros_like(adv)
+    o2 = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, tok, dppo.BINARY_TV, delta)
+    torch.cuda.synchronize()
+    assert int(o2["status"].item()) == 0 and float(o2["loss"].item()) == 0.0
+    assert not o2["dHidden"].any() and not o2["dW"].any()
+    assert np.array_equal(o2["divergence"].cpu().numpy(), out["divergence"].cpu().numpy())
+    # no valid row at all
+    o3 = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, adv, torch.zeros_like(tok), dppo.BINARY_TV, delta)
+    torch.cuda.synchronize()
+    assert int(o3["status"].item()) == 0 and not o3["dHidden"].any() and not o3["dW"].any() and not o3["mask"].any()
+
+
 def test_fused_rejects_misuse():
     b = _fused_case(128, 64, 512, seed=42, resp_len=8)
     with pytest.raises(dppo.DppoError) as e:
