@@ -233,6 +233,14 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
                               float* stats, int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Tuning switch of the tensor-core GEMM (process-wide; the paper has no counterpart): 2 (default) computes 256 x 256
+ * tiles on pairs of SMs (tcgen05 cta_group::2, each SM stages half of the B tile), 1 computes 128 x 256 tiles on single
+ * SMs.  Any other value only queries.  Returns the previous setting.  The results of the two modes are the same up to
+ * the order of the fp32 additions inside the tensor cores.
+ */
+int dppo_gemm_cta_group(int cta_group);
+
+/*
  * The tensor-core GEMM the fused variant is built from, exposed for testing and reuse:
  * C[M, N] (fp32, row stride ldc) = A[M, K] . B[N, K]^T with A and B bf16 row-major (row strides lda, ldb elements,
  * multiples of 8; 16-byte aligned bases), fp32 accumulation.  status: device word, DPPO_STATUS_WAIT_LIMIT on a

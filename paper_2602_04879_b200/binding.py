@@ -73,6 +73,8 @@ def lib():
                                         c_void_p, c_void_p]
         L.dppo_gemm_nn_bf16.restype = c_int
         L.dppo_gemm_nn_bf16.argtypes = L.dppo_gemm_tn_bf16.argtypes
+        L.dppo_gemm_cta_group.restype = c_int
+        L.dppo_gemm_cta_group.argtypes = [c_int]
         L.dppo_loss_fwd_bwd_static_ws.restype = c_int
         L.dppo_loss_fwd_bwd_static_ws.argtypes = L.dppo_loss_fwd_bwd.argtypes[:22] + [c_void_p]
         _lib = L
@@ -241,6 +243,12 @@ def dppo_gemm_nn_bf16(A, B, C=None, status=None, stream=None):
     if rc != 0:
         raise DppoError(rc, "dppo_gemm_nn_bf16")
     return C, status
+
+
+def dppo_gemm_cta_group(cta_group=0):
+    """Sets the tensor-core GEMM's mode (2: pairs of SMs per 256 x 256 tile, the default; 1: single SMs); any other value
+    only queries.  Returns the previous setting."""
+    return int(lib().dppo_gemm_cta_group(int(cta_group)))
 
 
 STATIC_WS_MAX_ROWS = 65536

@@ -15,6 +15,7 @@
 // dHidden and dW are d = thousands of columns wide, far more than the 512 accumulator columns of tensor memory, so they
 // cannot be accumulated on chip across the vocabulary; the bf16 gradient P (not the logits) is therefore staged in the
 // caller's workspace between steps 4 and 5/6.
+#include <atomic>
 #include <mutex>
 
 #include "dppo_common.cuh"
@@ -55,19 +56,22 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// B_MN = false: B is [N, K] with leading dimension ldb; B_MN = true: B is [K, N] with leading dimension ldb.
-template <int EPI, bool B_MN = false>
-cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
-  if (p.M <= 0 || p.N <= 0 || p.K <= 0) return cudaSuccess;
+// 1: one CTA per tile (cta_group::1); 2: pairs of CTAs per 256 x 256 tile (cta_group::2).  Set by dppo_gemm_cta_group.
+std::atomic<int> g_cta_group{2};
+
+template <int EPI, bool B_MN, int CG>
+cudaError_t launch_gemm_cg(const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
+  using C = gemm::Cfg<CG>;
   CUtensorMap ma, mb;
   if (!make_map(&ma, A, p.M, p.K, lda, gemm::BM)) return cudaErrorInvalidValue;
-  if (!(B_MN ? make_map(&mb, B, p.K, p.N, ldb, gemm::BK) : make_map(&mb, B, p.N, p.K, ldb, gemm::BN))) return cudaErrorInvalidValue;
+  if (!(B_MN ? make_map(&mb, B, p.K, p.N, ldb, gemm::BK) : make_map(&mb, B, p.N, p.K, ldb, C::B_COLS))) return cudaErrorInvalidValue;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  cudaError_t e = cudaFuncSetAttribute(gemm::gemm_tn_kernel<EPI, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::SMEM_BYTES);
+  auto kernel = gemm::gemm_tn_kernel<EPI, B_MN, CG>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  const int64_t ntiles = (int64_t)((p.M + gemm::BM - 1) / gemm::BM) * ((p.N + gemm::BN - 1) / gemm::BN);
+  const int64_t ntiles = (int64_t)((p.M + C::TILE_M - 1) / C::TILE_M) * ((p.N + gemm::BN - 1) / gemm::BN);
   p.sms = sms;
   int max_splits = 1;
   if (EPI == gemm::EPI_STORE_F32) max_splits = p.splits > 1 ? p.splits : (p.splits < 0 ? 2 : 1);
@@ -77,9 +81,27 @@ cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, 
     if (ez != cudaSuccess) return ez;
   }
   const int64_t nunits = ntiles * max_splits;
-  const int grid = (int)(nunits < sms ? nunits : sms);
-  gemm::gemm_tn_kernel<EPI, B_MN><<<grid, gemm::THREADS, gemm::SMEM_BYTES, st>>>(ma, mb, p);
-  return cudaGetLastError();
+  const int slots = sms / CG;                               // CTA groups that can be resident at once
+  const int groups = (int)(nunits < slots ? nunits : slots);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(groups * CG));
+  cfg.blockDim = dim3(gemm::THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (CG > 1) ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, ma, mb, p);
+}
+
+// B_MN = false: B is [N, K] with leading dimension ldb; B_MN = true: B is [K, N] with leading dimension ldb.
+template <int EPI, bool B_MN = false>
+cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
+  if (p.M <= 0 || p.N <= 0 || p.K <= 0) return cudaSuccess;
+  return g_cta_group.load() == 2 ? launch_gemm_cg<EPI, B_MN, 2>(A, lda, B, ldb, p, st)
+                                 : launch_gemm_cg<EPI, B_MN, 1>(A, lda, B, ldb, p, st);
 }
 
 // out[c, r] = in[r, c] for bf16 matrices; 64 x 64 tiles through shared memory, 16-byte global accesses when the
@@ -324,6 +346,12 @@ extern "C" {
 size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V, int K) {
   if (T < 0 || d < 1 || V < 1 || K < 0) return 0;
   return dppo::fused_layout(T, d, V, K).total;
+}
+
+int dppo_gemm_cta_group(int cta_group) {
+  const int prev = dppo::g_cta_group.load();
+  if (cta_group == 1 || cta_group == 2) dppo::g_cta_group.store(cta_group);
+  return prev;
 }
 
 int dppo_gemm_tn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,

@@ -10,6 +10,14 @@
 //               already fills the other 256-column accumulator buffer
 // Tiles are walked M-fastest so that CTAs running at the same time share B strips through L2.
 // Every mbarrier wait is bounded; on expiry the CTA raises DPPO_STATUS_WAIT_LIMIT, skips the rest and frees its TMEM.
+//
+// CG = 2 runs the same roles on pairs of CTAs (a cluster of two SMs) with tcgen05.mma.cta_group::2: one work unit is a
+// 256 x 256 tile, each CTA stages its own 128 rows of A and only half of the B tile (128 of the 256 columns) and
+// accumulates its 128 rows x 256 columns in its own tensor memory; the tensor cores of both SMs read both halves of B.
+// That halves the shared-memory fill per flop for B and makes room for 6 stages.  The even CTA of the pair (the leader)
+// issues the MMAs; the loads of both CTAs report to the leader's "full" barrier, tcgen05.commit multicasts the "stage
+// free" and "accumulator ready" arrivals to both CTAs, and the epilogue warps of both CTAs release the accumulator buffer
+// on the leader's barrier.  No multicast loads are used.
 #pragma once
 
 #include <cuda.h>
@@ -22,12 +30,20 @@
 namespace dppo {
 namespace gemm {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
-constexpr int A_STAGE_BYTES = BM * BK * 2, B_STAGE_BYTES = BN * BK * 2;
-constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int BM = 128, BN = 256, BK = 64;
 constexpr int THREADS = 192;
 constexpr int TMEM_COLS = 512;
+constexpr int MAX_STAGES = 6;
+
+// Per-CTA staging for CTA groups of CG = 1 or 2 SMs.
+template <int CG> struct Cfg {
+  static constexpr int TILE_M = BM * CG;                   // rows of C per work unit (128 per CTA)
+  static constexpr int B_COLS = BN / CG;                   // columns of the B tile this CTA stages
+  static constexpr int A_STAGE_BYTES = BM * BK * 2, B_STAGE_BYTES = B_COLS * BK * 2;
+  static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+  static constexpr int STAGES = (CG == 1) ? 4 : 6;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
 
 enum { EPI_STORE_F32 = 0, EPI_STATS = 1, EPI_GRAD = 2 };
 
@@ -98,6 +114,41 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+// ---- CTA pairs (cluster of two) -------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void bar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+// Load of one CTA of a pair; the completion bytes go to `cluster_bar`, which may live in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t cluster_bar) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void mma_bf16_pair(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(tmem_c), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far are done.
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+
 // Shared-memory matrix descriptor: K-major tile with rows of 128 bytes, 128-byte swizzle (8-row groups 1024 bytes apart).
 __device__ __forceinline__ uint64_t make_desc_k_sw128(uint32_t saddr) {
   uint64_t d = 0;
@@ -120,9 +171,12 @@ __device__ __forceinline__ uint64_t make_desc_mn_sw128(uint32_t saddr, uint32_t 
   d |= (uint64_t)2 << 61;                          // layout type: 128-byte swizzle
   return d;
 }
-// Instruction descriptor: D = f32, A = B = bf16, A K-major, B K-major or MN-major (bit 16), N = 256, M = 128.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-constexpr uint32_t kIdescBmn = kIdesc | (1u << 16);
+// Instruction descriptor: D = f32, A = B = bf16, A K-major, B K-major or MN-major (bit 16), N = 256, M = 128 per CTA of
+// the group (M = 256 for a pair).
+__host__ __device__ constexpr uint32_t make_idesc(int cg, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn ? (1u << 16) : 0u) | ((uint32_t)(BN >> 3) << 17) |
+         ((uint32_t)((BM * cg) >> 4) << 24);
+}
 
 __device__ __forceinline__ void mma_bf16(uint32_t tmem_c, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -150,12 +204,14 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // B_MN = false: B given as [N, K] (K contiguous).  B_MN = true: B given as [K, N] (N contiguous, "NN" product); its tile is
-// then loaded as four boxes of 64 columns x 64 k-rows.
-template <int EPI, bool B_MN>
+// then loaded as boxes of 64 columns x 64 k-rows.  CG = 2: launched as clusters of two CTAs (see the top of the file).
+template <int EPI, bool B_MN, int CG>
 __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a,
                                                              const __grid_constant__ CUtensorMap map_b, Params p) {
+  using C = Cfg<CG>;
+  constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, A_STAGE_BYTES = C::A_STAGE_BYTES;
   extern __shared__ unsigned char smem_raw[];
-  // 1024-byte alignment for the 128-byte swizzle atoms
+  // 1024-byte alignment for the 128-byte swizzle atoms (the same offset in both CTAs of a pair)
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + STAGES * STAGE_BYTES);
   const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + STAGES);
@@ -163,27 +219,36 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = (CG == 2) ? cluster_ctarank() : 0u;       // 0: leader of the pair
+  const int group = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int ngroups = (CG == 2) ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
   if (tid == 0) {
     for (int i = 0; i < STAGES; ++i) { bar_init(full0 + 8 * i, 1); bar_init(empty0 + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) { bar_init(tfull0 + 8 * i, 1); bar_init(tempty0 + 8 * i, 4); }
+    for (int i = 0; i < 2; ++i) { bar_init(tfull0 + 8 * i, 1); bar_init(tempty0 + 8 * i, 4 * CG); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {   // the MMA warp owns the tensor memory
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (warp == 1) {   // the MMA warp owns the tensor memory (in a pair: the same warp of both CTAs, together)
+    if (CG == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  if (CG == 2) cluster_sync_all();      // the peer's barriers exist before anything is sent to them
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
   int m_lim = p.M, k_lim = p.K;
   if (p.m_live) { const int v = *p.m_live; m_lim = v < 0 ? 0 : (v < p.M ? v : p.M); }
   if (p.k_live) { const int v = *p.k_live; k_lim = v < 0 ? 0 : (v < p.K ? v : p.K); }
-  const int tiles_m = m_lim > 0 ? (m_lim + BM - 1) / BM : 1, tiles_n = (p.N + BN - 1) / BN;
+  const int tiles_m = m_lim > 0 ? (m_lim + C::TILE_M - 1) / C::TILE_M : 1, tiles_n = (p.N + BN - 1) / BN;
   const int ntiles = tiles_m * tiles_n;
   const int kblocks = k_lim > 0 ? (k_lim + BK - 1) / BK : 1;
   // work unit u = part * ntiles + tile: all tiles of one K part are in flight together and share operand strips
@@ -191,9 +256,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   if (EPI == EPI_STORE_F32) {
     if (p.splits > 1) splits = p.splits;
     else if (p.splits < 0 && p.sms > 0 && kblocks >= 8) {
-      // few output tiles, very long K: cut K in two when the halves fill whole waves of CTAs better
-      const float w1 = (float)ntiles / (float)(((ntiles + p.sms - 1) / p.sms) * p.sms);
-      const float w2 = (float)(2 * ntiles) / (float)(((2 * ntiles + p.sms - 1) / p.sms) * p.sms);
+      // few output tiles, very long K: cut K in two when the halves fill whole waves of CTA groups better
+      const int slots = p.sms / CG;
+      const float w1 = (float)ntiles / (float)(((ntiles + slots - 1) / slots) * slots);
+      const float w2 = (float)(2 * ntiles) / (float)(((2 * ntiles + slots - 1) / slots) * slots);
       if (w2 > w1 + 0.05f) splits = 2;
     }
   }
@@ -202,42 +268,61 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   const uint32_t smem_base = smem_addr(smem);
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer (of this CTA's operand slices)
     if (lane == 0) {
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < nunits && ok; u += gridDim.x) {
+      for (int u = group; u < nunits && ok; u += ngroups) {
         const int tile = u % ntiles, part = u / ntiles;
-        const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+        const int m0 = (tile % tiles_m) * C::TILE_M + (int)rank * BM, n0 = (tile / tiles_m) * BN + (int)rank * C::B_COLS;
         const int kb0 = part * kper, kb1 = (kb0 + kper < kblocks) ? kb0 + kper : kblocks;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!bar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = smem_base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
-          bar_expect_tx(full0 + 8 * s, STAGE_BYTES);
-          tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
-          if (B_MN) {
+          if (CG == 2) {
+            // both CTAs' bytes are counted on the leader's barrier (the leader may post its expectation after the
+            // peer's bytes have begun to land: the phase cannot complete before the leader's own arrival)
+            const uint32_t bar = map_to_cta(full0 + 8 * s, 0);
+            if (rank == 0) bar_expect_tx(full0 + 8 * s, 2 * STAGE_BYTES);
+            tma_load_2d_pair(a_dst, &map_a, kb * BK, m0, bar);
+            if (B_MN) {
 #pragma unroll
-            for (int i = 0; i < BN / 64; ++i) tma_load_2d(b_dst + i * (64 * BK * 2), &map_b, n0 + i * 64, kb * BK, full0 + 8 * s);
+              for (int i = 0; i < C::B_COLS / 64; ++i) tma_load_2d_pair(b_dst + i * (64 * BK * 2), &map_b, n0 + i * 64, kb * BK, bar);
+            } else {
+              tma_load_2d_pair(b_dst, &map_b, kb * BK, n0, bar);
+            }
           } else {
-            tma_load_2d(b_dst, &map_b, kb * BK, n0, full0 + 8 * s);
+            bar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+            tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
+            if (B_MN) {
+#pragma unroll
+              for (int i = 0; i < C::B_COLS / 64; ++i) tma_load_2d(b_dst + i * (64 * BK * 2), &map_b, n0 + i * 64, kb * BK, full0 + 8 * s);
+            } else {
+              tma_load_2d(b_dst, &map_b, kb * BK, n0, full0 + 8 * s);
+            }
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
       }
+      if (!ok) {      // gave up: let the copies still in flight land before this CTA's shared memory goes away
+        const unsigned long long t0 = timer_ns();
+        while (timer_ns() - t0 < 100000ull) { }
+      }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer (in a pair: the leader's only)
+    if (lane == 0 && rank == 0) {
       int s = 0;
       uint32_t ph = 0;
       uint32_t it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < nunits && ok; u += gridDim.x, ++it) {
+      constexpr uint32_t idesc = make_idesc(CG, B_MN);
+      for (int u = group; u < nunits && ok; u += ngroups, ++it) {
         const int part = u / ntiles;
         const int kb0 = part * kper, kb1 = (kb0 + kper < kblocks) ? kb0 + kper : kblocks;
         const uint32_t b = it & 1u, use = it >> 1;
-        if (!bar_wait(tempty0 + 8 * b, (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }   // epilogue drained this buffer
+        if (!bar_wait(tempty0 + 8 * b, (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }   // epilogues drained this buffer
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t tmem_c = tmem_base + b * BN;
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -249,21 +334,24 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
           // per step of 16 along K: K-major operands move 32 bytes inside the swizzle atom, an MN-major one 16 k-rows (2048 bytes)
           constexpr uint64_t kStepB = B_MN ? (uint64_t)(16 * 128 >> 4) : 2ull;
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)
-            mma_bf16(tmem_c, adesc + (uint64_t)(k * 2), bdesc + kStepB * k, B_MN ? kIdescBmn : kIdesc, (kb != kb0 || k != 0) ? 1u : 0u);
-          mma_commit(empty0 + 8 * s);            // stage free once these MMAs have read it
+          for (int k = 0; k < BK / 16; ++k) {
+            if (CG == 2) mma_bf16_pair(tmem_c, adesc + (uint64_t)(k * 2), bdesc + kStepB * k, idesc, (kb != kb0 || k != 0) ? 1u : 0u);
+            else mma_bf16(tmem_c, adesc + (uint64_t)(k * 2), bdesc + kStepB * k, idesc, (kb != kb0 || k != 0) ? 1u : 0u);
+          }
+          // stage free (in both CTAs of a pair) once these MMAs have read it
+          if (CG == 2) mma_commit_pair(empty0 + 8 * s); else mma_commit(empty0 + 8 * s);
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
-        if (ok) mma_commit(tfull0 + 8 * b);      // accumulator complete
+        if (ok) { if (CG == 2) mma_commit_pair(tfull0 + 8 * b); else mma_commit(tfull0 + 8 * b); }   // accumulator complete
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps (TMEM lane quarter = warp % 4)
     const int q = warp & 3;
     uint32_t it = 0;
-    for (int u = blockIdx.x; u < nunits; u += gridDim.x, ++it) {
+    for (int u = group; u < nunits; u += ngroups, ++it) {
       const int tile = u % ntiles;
-      const int m0 = (tile % tiles_m) * BM, nb = tile / tiles_m, n0 = nb * BN;
+      const int m0 = (tile % tiles_m) * C::TILE_M + (int)rank * BM, nb = tile / tiles_m, n0 = nb * BN;
       const uint32_t b = it & 1u, use = it >> 1;
       const bool ok = __all_sync(0xffffffffu, bar_wait(tfull0 + 8 * b, use & 1u, abort_flag));
       if (!ok) break;
@@ -360,16 +448,23 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
-      if (lane == 0) bar_arrive(tempty0 + 8 * b);
+      if (lane == 0) {       // buffer drained: tell the MMA issuer (the leader's, in a pair)
+        if (CG == 2 && rank != 0) bar_arrive_cluster(map_to_cta(tempty0 + 8 * b, 0));
+        else bar_arrive(tempty0 + 8 * b);
+      }
     }
   }
 
+  __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  // a pair leaves together: neither CTA's shared or tensor memory may go away while the other can still reach it
+  if (CG == 2) cluster_sync_all();
   if (*abort_flag && tid == 0 && p.status) atomicOr(p.status, DPPO_STATUS_WAIT_LIMIT);
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (CG == 2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 

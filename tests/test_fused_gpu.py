@@ -13,8 +13,16 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
+@pytest.fixture(params=[2, 1], ids=["cta_pair", "single_cta"])
+def cta_group(request):
+    """Both modes of the tensor-core GEMM: pairs of SMs (the default) and single SMs."""
+    prev = dppo.dppo_gemm_cta_group(request.param)
+    yield request.param
+    dppo.dppo_gemm_cta_group(prev)
+
+
 @pytest.mark.parametrize("M,N,K", [(128, 256, 64), (128, 256, 256), (300, 520, 200), (256, 1024, 1024), (1000, 264, 4104)])
-def test_gemm_tn_bf16_matches_fp64_product(M, N, K):
+def test_gemm_tn_bf16_matches_fp64_product(M, N, K, cta_group):
     g = torch.Generator(device=DEV).manual_seed(M * 7 + N * 3 + K)
     A = torch.randn((M, K), generator=g, device=DEV).to(torch.bfloat16)
     B = torch.randn((N, K), generator=g, device=DEV).to(torch.bfloat16)
@@ -34,7 +42,7 @@ def test_gemm_tn_bf16_matches_fp64_product(M, N, K):
 
 
 @pytest.mark.parametrize("M,N,K", [(128, 256, 64), (128, 256, 256), (300, 520, 200), (256, 1024, 1024), (264, 4104, 1000)])
-def test_gemm_nn_bf16_matches_fp64_product(M, N, K):
+def test_gemm_nn_bf16_matches_fp64_product(M, N, K, cta_group):
     """B given as [K, N]: the MN-major operand path of the tensor-core GEMM."""
     g = torch.Generator(device=DEV).manual_seed(M * 5 + N * 11 + K)
     A = torch.randn((M, K), generator=g, device=DEV).to(torch.bfloat16)
@@ -83,7 +91,7 @@ def _check_fused(b, variant, delta, tok=None, K=0, is_cap=0.0):
 
 
 @pytest.mark.parametrize("T,d,V", [(256, 128, 1024), (200, 72, 1000), (384, 256, 2304)])
-def test_fused_matches_oracle_small(T, d, V):
+def test_fused_matches_oracle_small(T, d, V, cta_group):
     b = _fused_case(T, d, V, seed=41, resp_len=8)
     out, ora = _check_fused(b, dppo.BINARY_TV, 0.2)
     # mask stress near the median divergence, KL variant, ragged mask
@@ -122,7 +130,7 @@ def test_fused_topk_variants_match_oracle(variant):
     assert int(o3["status"].item()) == dppo.binding.STATUS_BAD_TOPK_ID and not o3["dHidden"][7].any()
 
 
-def test_fused_backward_skips_rows_without_gradient():
+def test_fused_backward_skips_rows_without_gradient(cta_group):
     """Rows with zero advantage, rows blocked by the mask and invalid rows drop out of the backward GEMMs (the kept rows are
     packed on the device); the outputs must not change: zeros in dHidden for those rows, the same dW."""
     T, d, V = 600, 128, 1536
