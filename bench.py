@@ -107,14 +107,13 @@ def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
     ms_sparse = e0.elapsed_time(e1) / max(1, steps // 2)
     b.advantages = adv_full
     peak, src = measured_tensor_peak()
-    useful = 6.0 * T * d * V / (ms * 1e-3) / 1e12          # forward + dHidden + dW
-    executed = 8.0 * T * d * V / (ms * 1e-3) / 1e12        # + the recomputation of the logits tiles
+    useful = 6.0 * T * d * V / (ms * 1e-3) / 1e12          # forward + dHidden + dW; every logits tile is computed once
     return {"workload": ("" if T == 8192 else f"REDUCED to {T} rows (profiling case): ") + "fused_lm_head_binary_tv: hidden [8192,2048] bf16 x W [2048,151936] bf16, delta=0.2",
             "ms_per_step": ms, "tokens_per_s": T / (ms * 1e-3), "steps": steps, "warmup": warmup,
             "roofline": {"bound": "tensor", "achieved": useful, "peak": peak, "unit": "TFLOP/s", "frac": useful / peak,
-                         "executed_tflops": executed, "executed_frac": executed / peak, "traffic": None,
-                         "peak_source": "of " + src, "flop_count": "useful = 6*T*d*V (forward, dHidden, dW); executed = 8*T*d*V with the recomputed logits"},
-            "gpu_launches_per_step": 10, "loss": float(out["loss"].item()),
+                         "traffic": None, "peak_source": "of " + src,
+                         "flop_count": "6*T*d*V (forward, dHidden, dW); nothing is recomputed"},
+            "gpu_launches_per_step": 15, "loss": float(out["loss"].item()),
             "ms_per_step_quarter_of_responses_zero_advantage": ms_sparse}
 
 

@@ -1,20 +1,29 @@
 // Fused LM-head variant of the DPPO loss: logits = hidden x W are produced tile by tile on the tensor cores and
-// consumed in the accumulators' epilogue, so the [T, V] logits never exist in memory.
+// consumed in the accumulators' epilogue, so the [T, V] logits never exist in memory, and every tile is computed once.
 //
-//   1. (token mask given) the valid rows of hidden packed together; (Top-K variants) W^T for the gather
-//   2. stats GEMM     z-tile = hidden . W-tile (B = W [d, V] as an MN-major operand); epilogue: per-row (max, sum exp)
-//                     of the tile, z at the sampled id
-//   3. scalar kernel  merge the tiles' partials -> lse; ratio, divergence, mask, loss term, gradient coefficients
-//                     (Top-K variants: the K logits per row come from a small gather-dot kernel over rows of W^T)
-//   4. packing        rows with a non-zero gradient, in order, packed together (hidden rows, coefficients) and transposed;
-//                     their count stays on the device and bounds the tile loops of the three GEMMs below
-//   5. grad GEMM      the same tiles again; epilogue: P = dlogits = g (softmax - onehot) in bf16, [rows, V]
-//   6. dHidden = P . W^T   (A = P, B = W [d,V] K-major), rows scattered back        fp32
-//   7. dW = hidden^T . P   (A = packed hidden^T, B = P as MN-major)                 fp32
+// The gradient row is g (softmax(z) - onehot) = (g / S) (E - S onehot) with E_j = exp(z_j - c) and S = sum_j E_j for ANY
+// per-row reference c.  With c known before the GEMM (the logit of the sampled token, one dot product per row) the
+// exponentials can be written in the same pass that sums them; the per-row factor g / S, known only after the whole
+// vocabulary has been seen, is applied later where it is cheap: to the rows of dHidden in that GEMM's epilogue, and to
+// the rows of hidden before the dW GEMM.  bf16 has the exponent range of fp32, so E needs no row maximum.
+//
+//   1. partition      valid rows with a non-zero advantage first, then the other valid rows (they need the divergence
+//                     but no gradient), packed copies of hidden / sampled ids; (Top-K variants) W^T for the gather
+//   2. reference      c_t = z_t[a_t] by a dot product per row
+//   3. forward GEMM   z-tile = hidden . W-tile (B = W [d, V] as an MN-major operand); epilogue: E = exp(z - c) in bf16
+//                     [rows with a gradient only], per-row partial sums of E, z at the sampled id
+//   4. scalar kernel  S, lse = c + log S; ratio, divergence, mask, loss term; row factor g / S; the sampled token's entry
+//                     of E becomes E - S (Top-K variants: the K logits per row come from a gather-dot over rows of W^T)
+//   5. rescue         rows whose S left the safe range (the sampled token's probability below 2^-60, or non-finite
+//                     logits) are packed and go through the two-pass kernels (statistics GEMM with an online maximum,
+//                     scalar stage, gradient GEMM writing the finished gradient row into E, row factor 1); normally
+//                     there are none and these launches find nothing to do
+//   6. dHidden = diag(g / S) (E . W^T)   (A = E, B = W [d,V] K-major), rows scattered back        fp32
+//   7. dW = (diag(g / S) hidden)^T . E   (A = scaled packed hidden^T, B = E as MN-major)          fp32
 //
 // dHidden and dW are d = thousands of columns wide, far more than the 512 accumulator columns of tensor memory, so they
-// cannot be accumulated on chip across the vocabulary; the bf16 gradient P (not the logits) is therefore staged in the
-// caller's workspace between steps 4 and 5/6.
+// cannot be accumulated on chip across the vocabulary; the bf16 exponentials E (not the logits) are therefore staged in
+// the caller's workspace between steps 3 and 6/7.
 #include <atomic>
 #include <mutex>
 
@@ -104,22 +113,37 @@ cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, 
                                  : launch_gemm_cg<EPI, B_MN, 1>(A, lda, B, ldb, p, st);
 }
 
-// out[c, r] = in[r, c] for bf16 matrices; 64 x 64 tiles through shared memory, 16-byte global accesses when the
-// layout allows (leading dimensions multiples of 8 elements, 16-byte aligned bases), 2-byte accesses at the edges.
+// out[c, r] = scale[r] * in[r, c] for bf16 matrices (scale optional: rows at and beyond *n_live count as scale 0);
+// 64 x 64 tiles through shared memory, 16-byte global accesses when the layout allows (leading dimensions multiples of
+// 8 elements, 16-byte aligned bases), 2-byte accesses at the edges.
+__device__ __forceinline__ unsigned short scale_bf16(unsigned short v, float sc) {
+  // a zero factor gives an exact zero, whatever the element is (a dropped row may hold non-finite values)
+  return sc == 0.f ? (unsigned short)0 : __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float((uint32_t)v << 16) * sc));
+}
 __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* in, int64_t rows, int64_t cols, int64_t ld_in,
-                                                             __nv_bfloat16* out, int64_t ld_out, int vec_ok) {
+                                                             __nv_bfloat16* out, int64_t ld_out, int vec_ok,
+                                                             const float* row_scale, const int32_t* n_live) {
   __shared__ unsigned short tile[64][72];                 // [r][c], row pitch 144 bytes (16-byte aligned rows)
   const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
   const int tid = threadIdx.x;
   const unsigned short* src = reinterpret_cast<const unsigned short*>(in);
   unsigned short* dst = reinterpret_cast<unsigned short*>(out);
   const bool interior = vec_ok && r0 + 64 <= rows && c0 + 64 <= cols;
+  const int64_t live = n_live ? (int64_t)*n_live : rows;
   if (interior) {
     // 64 rows x 8 vectors of 8 elements: thread -> (row = tid / 8 + 32 * pass, vector = tid % 8)
 #pragma unroll
     for (int pass = 0; pass < 2; ++pass) {
       const int r = (tid >> 3) + 32 * pass, v = tid & 7;
-      const uint4 x = *reinterpret_cast<const uint4*>(src + (r0 + r) * ld_in + c0 + v * 8);
+      uint4 x = *reinterpret_cast<const uint4*>(src + (r0 + r) * ld_in + c0 + v * 8);
+      if (row_scale) {
+        const float sc = (r0 + r < live) ? row_scale[r0 + r] : 0.f;
+        uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          w[k] = (uint32_t)scale_bf16((unsigned short)(w[k] & 0xffffu), sc) | ((uint32_t)scale_bf16((unsigned short)(w[k] >> 16), sc) << 16);
+        x = make_uint4(w[0], w[1], w[2], w[3]);
+      }
       *reinterpret_cast<uint4*>(&tile[r][v * 8]) = x;
     }
     __syncthreads();
@@ -138,7 +162,9 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
     const int tx = tid & 63, ty = tid >> 6;
     for (int i = ty; i < 64; i += 4) {
       const int64_t r = r0 + i, c = c0 + tx;
-      tile[i][tx] = (r < rows && c < cols) ? src[r * ld_in + c] : (unsigned short)0;
+      unsigned short v = (r < rows && c < cols) ? src[r * ld_in + c] : (unsigned short)0;
+      if (row_scale) v = scale_bf16(v, (r < rows && r < live) ? row_scale[r] : 0.f);
+      tile[i][tx] = v;
     }
     __syncthreads();
     for (int i = ty; i < 64; i += 4) {
@@ -148,13 +174,42 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
   }
 }
 
-cudaError_t transpose_bf16(const void* in, int64_t rows, int64_t cols, int64_t ld_in, void* out, int64_t ld_out, cudaStream_t st) {
+cudaError_t transpose_bf16(const void* in, int64_t rows, int64_t cols, int64_t ld_in, void* out, int64_t ld_out, cudaStream_t st,
+                           const float* row_scale = nullptr, const int32_t* n_live = nullptr) {
   if (rows <= 0 || cols <= 0) return cudaSuccess;
   dim3 grid((unsigned)((cols + 63) / 64), (unsigned)((rows + 63) / 64));
   const int vec_ok = (ld_in % 8 == 0) && (ld_out % 8 == 0) && ((uintptr_t)in % 16 == 0) && ((uintptr_t)out % 16 == 0);
   transpose_bf16_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(in), rows, cols, ld_in,
-                                              reinterpret_cast<__nv_bfloat16*>(out), ld_out, vec_ok);
+                                              reinterpret_cast<__nv_bfloat16*>(out), ld_out, vec_ok, row_scale, n_live);
   return cudaGetLastError();
+}
+
+// cref2[i] = log2(e) * hidden_c[i, :] . W[:, ids[i]]: the reference exponent of packed row i (the logit of its sampled
+// token), one warp per row.  The column of W is strided (one 2-byte element per row of W).  Out-of-range ids give 0.
+__global__ void __launch_bounds__(256) fused_ref_logit_kernel(const __nv_bfloat16* hc, const __nv_bfloat16* W, int64_t T, int64_t d,
+                                                              int64_t V, const int32_t* ids, const int32_t* n_rows, float* cref2) {
+  const int lane = threadIdx.x & 31;
+  const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (i >= T) return;
+  float acc = 0.f;
+  const int id = ids[i];
+  if (i < (int64_t)*n_rows && id >= 0 && (int64_t)id < V) {
+    const unsigned short* h = reinterpret_cast<const unsigned short*>(hc + i * d);
+    const unsigned short* w = reinterpret_cast<const unsigned short*>(W) + id;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    int64_t k = lane;
+    for (; k + 96 < d; k += 128) {
+      a0 = fmaf(__uint_as_float((uint32_t)h[k] << 16), __uint_as_float((uint32_t)w[k * V] << 16), a0);
+      a1 = fmaf(__uint_as_float((uint32_t)h[k + 32] << 16), __uint_as_float((uint32_t)w[(k + 32) * V] << 16), a1);
+      a2 = fmaf(__uint_as_float((uint32_t)h[k + 64] << 16), __uint_as_float((uint32_t)w[(k + 64) * V] << 16), a2);
+      a3 = fmaf(__uint_as_float((uint32_t)h[k + 96] << 16), __uint_as_float((uint32_t)w[(k + 96) * V] << 16), a3);
+    }
+    for (; k < d; k += 32) a0 = fmaf(__uint_as_float((uint32_t)h[k] << 16), __uint_as_float((uint32_t)w[k * V] << 16), a0);
+    acc = (a0 + a1) + (a2 + a3);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) cref2[i] = isfinite(acc) ? acc * kLog2e : 0.f;
 }
 
 // z_topk[t, k] = hidden[t, :] . W^T[ids[t, k], :]: the logits at the rollout policy's top-K ids, one warp per (t, k).
@@ -185,38 +240,50 @@ __global__ void __launch_bounds__(256) fused_topk_logits_kernel(const __nv_bfloa
   if (lane == 0) z_topk[w] = acc;       // out-of-range ids give 0 here and raise the status bit in the scalar stage
 }
 
-// Stable compaction of the rows to keep (one block): idx[i] = i-th kept row, pos[t] = its place in idx or -1, *n = count.
-// A row is kept when its token_mask byte is non-zero (mask8 given) or when its gradient sign is non-zero (sgn given).
-__global__ void __launch_bounds__(1024) fused_compact_rows_kernel(const uint8_t* mask8, const float* sgn, int64_t T, int32_t* idx,
-                                                                  int32_t* pos, int32_t* n) {
-  __shared__ int warp_tot[32];
+// Stable two-class partition of the rows (one block): idx = the rows of class 0 in order, then those of class 1;
+// pos[t] = the place of row t in idx, or -1 for dropped rows; n[0] = rows of class 0, n[1] = rows of both classes.
+//   flag given:  class 0 = rows with flag[t] != 0, everything else dropped
+//   otherwise:   class 0 = valid rows (token_mask byte non-zero, or no mask) with adv[t] != 0, class 1 = the other valid rows
+__global__ void __launch_bounds__(1024) fused_partition_rows_kernel(const uint8_t* mask8, const float* adv, const int32_t* flag,
+                                                                    int64_t T, int32_t* idx, int32_t* pos, int32_t* n) {
+  __shared__ int warp_tot[2][32];
+  __shared__ int total[2];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t per = (T + 1023) / 1024;
-  const int64_t t0 = (int64_t)tid * per, t1 = (t0 + per < T) ? t0 + per : T;
-  auto keep = [&](int64_t t) { return mask8 ? (mask8[t] != 0) : (sgn[t] != 0.f); };
-  int cnt = 0;
-  for (int64_t t = t0; t < t1; ++t) cnt += keep(t) ? 1 : 0;
-  int incl = cnt;
+  const int64_t t0 = (int64_t)tid * per < T ? (int64_t)tid * per : T, t1 = (t0 + per < T) ? t0 + per : T;
+  auto cls = [&](int64_t t) -> int {
+    if (flag) return flag[t] != 0 ? 0 : -1;
+    if (mask8 && mask8[t] == 0) return -1;
+    return adv[t] != 0.f ? 0 : 1;
+  };
+  int cnt[2] = {0, 0};
+  for (int64_t t = t0; t < t1; ++t) { const int c = cls(t); if (c >= 0) ++cnt[c]; }
+  int incl[2] = {cnt[0], cnt[1]};
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
-  if (lane == 31) warp_tot[warp] = incl;
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v0 = __shfl_up_sync(0xffffffffu, incl[0], o), v1 = __shfl_up_sync(0xffffffffu, incl[1], o);
+    if (lane >= o) { incl[0] += v0; incl[1] += v1; }
+  }
+  if (lane == 31) { warp_tot[0][warp] = incl[0]; warp_tot[1][warp] = incl[1]; }
   __syncthreads();
-  if (warp == 0) {
-    int v = warp_tot[lane], w = v;
+  if (warp < 2) {
+    int v = warp_tot[warp][lane], w = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) { const int u = __shfl_up_sync(0xffffffffu, w, o); if (lane >= o) w += u; }
-    warp_tot[lane] = w - v;                     // exclusive offset of each warp
-    if (lane == 31) *n = w;
+    warp_tot[warp][lane] = w - v;                     // exclusive offset of each warp
+    if (lane == 31) total[warp] = w;
   }
   __syncthreads();
-  int at = warp_tot[warp] + incl - cnt;
+  if (tid == 0) { n[0] = total[0]; n[1] = total[0] + total[1]; }
+  int at[2] = {warp_tot[0][warp] + incl[0] - cnt[0], total[0] + warp_tot[1][warp] + incl[1] - cnt[1]};
   for (int64_t t = t0; t < t1; ++t) {
-    if (keep(t)) { idx[at] = (int32_t)t; pos[t] = at; ++at; }
+    const int c = cls(t);
+    if (c >= 0) { idx[at[c]] = (int32_t)t; pos[t] = at[c]; ++at[c]; }
     else pos[t] = -1;
   }
 }
 
-// Row i of the compact copies = row idx[i] of the sources for i < *n, zeros after that (one block per row).
+// Row i of the compact copies = row idx[i] of the sources for i < *n; after that zeros (zero_fill) or left alone.
 struct GatherArgs {
   const int32_t* idx;
   const int32_t* n;
@@ -225,67 +292,137 @@ struct GatherArgs {
   __nv_bfloat16* dst;            // [T, d]
   const int32_t* ids_in;
   int32_t* ids_out;
-  const float* f_in[3];          // optional per-row floats (null: skipped)
-  float* f_out[3];
+  int zero_fill;
 };
 __global__ void __launch_bounds__(256) fused_gather_rows_kernel(GatherArgs g) {
   const int64_t i = blockIdx.x;
   const bool live = i < (int64_t)*g.n;
+  if (!live && !g.zero_fill) return;
   const int64_t t = live ? g.idx[i] : 0;
   const uint4* src = reinterpret_cast<const uint4*>(g.src + t * g.d);
   uint4* dst = reinterpret_cast<uint4*>(g.dst + i * g.d);
   for (int64_t j = threadIdx.x; j < g.d / 8; j += blockDim.x) dst[j] = live ? src[j] : make_uint4(0, 0, 0, 0);
-  if (threadIdx.x == 0) {
-    g.ids_out[i] = live ? g.ids_in[t] : 0;
-#pragma unroll
-    for (int k = 0; k < 3; ++k)
-      if (g.f_in[k]) g.f_out[k][i] = live ? g.f_in[k][t] : 0.f;
-  }
+  if (threadIdx.x == 0) g.ids_out[i] = live ? g.ids_in[t] : 0;
 }
 
-// One warp per row: merge the stats GEMM's per-tile partials, then the same scalar stage as the streaming kernels.
-// `pos` (optional) maps a row to its row in the statistics (rows compacted by the token mask; -1: not there).
-__global__ void __launch_bounds__(256) fused_scalar_kernel(RowParams p, const float2* part, int tiles_n, const float* z_a,
-                                                           const int32_t* pos, const float* z_topk, float* c2, float* sgn, float* fix) {
+// What the single-pass scalar stage adds to RowParams.
+struct ExpArgs {
+  const float* psum;        // [rows, tiles_n] partial sums of exp(z - c), packed row order
+  int tiles_n;
+  const float* z_a;         // [rows] z at the sampled id, packed row order
+  const float* cref2;       // [rows] c in log2 units, packed row order
+  const int32_t* pos;       // [T] packed row of row t, -1: not valid
+  const int32_t* n_grad;    // packed rows below *n_grad have a row in E
+  const float* z_topk;      // [T, K] or null
+  float* row_factor;        // [rows] g / S, packed row order
+  int32_t* rescue;          // [T] 1: the row goes through the two-pass kernels
+  __nv_bfloat16* E;
+  int64_t lde;
+};
+
+// Sums of exp(z - c) above this, or not finite, or not positive, send a row to the two-pass kernels: E and the row
+// factor g / S stay far inside the range of bf16 / fp32 for every row that is handled here.
+constexpr double kMaxSafeSum = 1.152921504606846976e18;      // 2^60
+
+// One warp per row: S from the forward GEMM's partial sums, then the same scalar stage as the streaming kernels.
+__global__ void __launch_bounds__(256) fused_scalar_exp_kernel(RowParams p, ExpArgs x) {
   const int lane = threadIdx.x & 31;
   const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (t >= p.T) return;
   const double scale = p.hdr->scale;
-  bool valid = p.token_mask ? (p.token_mask[t] != 0) : true;
-  int flags = 0;
+  const int64_t ts = (int64_t)x.pos[t];                 // < 0: token_mask says invalid
+  bool valid = ts >= 0;
+  int flags = 0, resc = 0;
   const int a = p.sampled_ids[t];
   if (valid && (a < 0 || (int64_t)a >= p.V)) { valid = false; flags = DPPO_STATUS_BAD_SAMPLED_ID; }
+  float D = 0.f, r = 0.f, absdiff = 0.f, factor = 0.f;
+  int M = 0;
+  double g = 0.0;
+  if (valid) {
+    double S = 0.0;
+    for (int i = lane; i < x.tiles_n; i += 32) S += (double)x.psum[ts * x.tiles_n + i];
+    S = warp_sum(S);
+    if (!(S > 0.0) || !(S <= kMaxSafeSum)) {
+      resc = 1;                                         // outputs of this row are written by the rescue pass
+    } else {
+      const double lse = ((double)x.cref2[ts] + log2(S)) / (double)kLog2e;
+      double pi_a;
+      int f2 = 0;
+      const float za = x.z_a[ts];
+      const float* zk = x.z_topk ? x.z_topk + t * (int64_t)p.K : nullptr;
+      auto z_at = [&](int, int k) { return k < 0 ? za : zk[k]; };   // sampled id, or position k of the top-K list
+      row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
+      if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
+      else if (g != 0.0) {
+        factor = (float)(g / S);
+        // the sampled token's entry: g (pi_a - 1) = (g / S) (E_a - S)
+        if (lane == 0 && ts < (int64_t)*x.n_grad) x.E[ts * x.lde + a] = __float2bfloat16_rn((float)((pi_a - 1.0) * S));
+      }
+    }
+  }
+  if (lane == 0) {
+    x.rescue[t] = resc;
+    if (ts >= 0) x.row_factor[ts] = factor;
+    if (!resc) {
+      p.divergence[t] = D;
+      p.mask[t] = (uint8_t)M;
+      p.row_loss[t] = (float)(-g);
+      p.row_r[t] = r;
+      p.row_absdiff[t] = absdiff;
+    }
+    if (flags) atomicOr(p.status, flags);
+  }
+}
+
+// Rescue pass, one warp per flagged row: merge the statistics GEMM's per-tile (max, sum) partials, run the scalar stage
+// and leave the coefficients of the gradient epilogue at the row's place among the rescued rows.
+struct RescueArgs {
+  const int32_t* rescue;    // [T] rows to process
+  const int32_t* pos_r;     // [T] place of row t among the rescued rows
+  const int32_t* pos_e;     // [T] packed row of row t in E
+  const float2* part;       // [rescued rows, tiles_n]
+  int tiles_n;
+  const float* z_a;         // [rescued rows]
+  const float* z_topk;
+  float *c2, *sgn, *fix;    // [rescued rows]
+  int32_t* p_row_map;       // [rescued rows] row of E the finished gradient row goes to
+  float* row_factor;        // [rows of E]
+};
+__global__ void __launch_bounds__(256) fused_scalar_rescue_kernel(RowParams p, RescueArgs x) {
+  const int lane = threadIdx.x & 31;
+  const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= p.T || !x.rescue[t]) return;
+  const double scale = p.hdr->scale;
+  const int64_t ts = x.pos_r[t], te = x.pos_e[t];
+  int flags = 0;
+  const int a = p.sampled_ids[t];
   float D = 0.f, r = 0.f, absdiff = 0.f;
   int M = 0;
   double g = 0.0;
   RowCoef coef;
   coef.c2 = 0.f; coef.sgn = 0.f; coef.fix = 0.f; coef.zero_row = 1;
-  const int64_t ts = pos ? (int64_t)pos[t] : t;       // row of the statistics
-  if (ts < 0) valid = false;
-  if (valid) {
-    float mm = -INFINITY;
-    for (int i = lane; i < tiles_n; i += 32) mm = fmaxf(mm, part[ts * tiles_n + i].x);
+  float mm = -INFINITY;
+  for (int i = lane; i < x.tiles_n; i += 32) mm = fmaxf(mm, x.part[ts * x.tiles_n + i].x);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
-    double S = 0.0;
-    for (int i = lane; i < tiles_n; i += 32) {
-      const float2 pr = part[ts * tiles_n + i];
-      if (pr.y > 0.f || pr.y != pr.y) S += (double)pr.y * exp((double)pr.x - (double)mm);
-    }
-    S = warp_sum(S);
-    const double lse = (double)mm + log(S);
-    if (!isfinite(lse)) {
-      flags |= DPPO_STATUS_NONFINITE_ROW;
-    } else {
-      double pi_a;
-      int f2 = 0;
-      const float za = z_a[ts];
-      const float* zk = z_topk ? z_topk + t * (int64_t)p.K : nullptr;
-      auto z_at = [&](int, int k) { return k < 0 ? za : zk[k]; };   // sampled id, or position k of the top-K list
-      row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
-      if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
-      else coef = make_coef(g, lse, pi_a);
-    }
+  for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
+  double S = 0.0;
+  for (int i = lane; i < x.tiles_n; i += 32) {
+    const float2 pr = x.part[ts * x.tiles_n + i];
+    if (pr.y > 0.f || pr.y != pr.y) S += (double)pr.y * exp((double)pr.x - (double)mm);
+  }
+  S = warp_sum(S);
+  const double lse = (double)mm + log(S);
+  if (!isfinite(lse)) {
+    flags |= DPPO_STATUS_NONFINITE_ROW;
+  } else {
+    double pi_a;
+    int f2 = 0;
+    const float za = x.z_a[ts];
+    const float* zk = x.z_topk ? x.z_topk + t * (int64_t)p.K : nullptr;
+    auto z_at = [&](int, int k) { return k < 0 ? za : zk[k]; };
+    row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
+    if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
+    else coef = make_coef(g, lse, pi_a);
   }
   if (lane == 0) {
     p.divergence[t] = D;
@@ -293,9 +430,13 @@ __global__ void __launch_bounds__(256) fused_scalar_kernel(RowParams p, const fl
     p.row_loss[t] = (float)(-g);
     p.row_r[t] = r;
     p.row_absdiff[t] = absdiff;
-    c2[t] = coef.c2;
-    sgn[t] = coef.zero_row ? 0.f : coef.sgn;
-    fix[t] = coef.fix;
+    x.c2[ts] = coef.c2;
+    x.sgn[ts] = coef.zero_row ? 0.f : coef.sgn;
+    x.fix[ts] = coef.fix;
+    // the gradient epilogue writes the finished row over the row's exponentials (zeros if g = 0: whatever overflowed
+    // there must not meet a later GEMM, not even multiplied by zero)
+    x.p_row_map[ts] = (int32_t)te;
+    x.row_factor[te] = coef.zero_row ? 0.f : 1.f;
     if (flags) atomicOr(p.status, flags);
   }
 }
@@ -304,35 +445,42 @@ constexpr size_t kAlign = 256;
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct FusedLayout {
-  size_t wt, ht, hc, P, Pt, part, z_a, z_topk, c2, sgn, fix, c2c, sgnc, fixc, ids_c, idx, pos, nlive, loss_ws, total;
-  int64_t ldp, ldt;
+  size_t wt, ht, hc, hr, E, psum, part, z_a, z_ar, z_topk, cref2, factor, c2, sgn, fix, ids_c, ids_r, idx, pos, idx_r, pos_r,
+      rescue, rmap, counts, loss_ws, total;
+  int64_t lde, ldt;
   int tiles_n;
 };
 FusedLayout fused_layout(int64_t T, int64_t d, int64_t V, int K) {
   FusedLayout L;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += round_up(bytes ? bytes : 1, kAlign); return o; };
-  L.ldp = (V + 7) / 8 * 8;
+  L.lde = (V + 7) / 8 * 8;
   L.ldt = (T + 7) / 8 * 8;
   L.tiles_n = (int)((V + gemm::BN - 1) / gemm::BN);
   L.wt = take(K > 0 ? (size_t)V * d * 2 : 0);      // W^T is only needed to gather the top-K logits
-  L.ht = take((size_t)d * L.ldt * 2);
-  L.hc = take((size_t)T * d * 2);                  // hidden rows compacted (valid rows, then rows with a gradient)
-  L.P = take((size_t)T * L.ldp * 2);
-  L.Pt = 0;
+  L.ht = take((size_t)d * L.ldt * 2);              // packed hidden rows times their row factor, transposed
+  L.hc = take((size_t)T * d * 2);                  // hidden rows packed (rows with a gradient, then the other valid rows)
+  L.hr = take((size_t)T * d * 2);                  // hidden rows of the rescue pass
+  L.E = take((size_t)T * L.lde * 2);
+  L.psum = take((size_t)T * L.tiles_n * sizeof(float));
   L.part = take((size_t)T * L.tiles_n * sizeof(float2));
   L.z_a = take((size_t)T * 4);
+  L.z_ar = take((size_t)T * 4);
   L.z_topk = take((size_t)T * (K > 0 ? K : 0) * 4);
+  L.cref2 = take((size_t)T * 4);
+  L.factor = take((size_t)T * 4);
   L.c2 = take((size_t)T * 4);
   L.sgn = take((size_t)T * 4);
   L.fix = take((size_t)T * 4);
-  L.c2c = take((size_t)T * 4);                     // the same per-row values in compact row order
-  L.sgnc = take((size_t)T * 4);
-  L.fixc = take((size_t)T * 4);
   L.ids_c = take((size_t)T * 4);
+  L.ids_r = take((size_t)T * 4);
   L.idx = take((size_t)T * 4);
   L.pos = take((size_t)T * 4);
-  L.nlive = take(2 * sizeof(int32_t));
+  L.idx_r = take((size_t)T * 4);
+  L.pos_r = take((size_t)T * 4);
+  L.rescue = take((size_t)T * 4);
+  L.rmap = take((size_t)T * 4);
+  L.counts = take(4 * sizeof(int32_t));
   L.loss_ws = take(dppo_workspace_bytes(T));
   L.total = off;
   return L;
@@ -424,75 +572,88 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
     DPPO_TRY(launch_finalize(p, st));
     return DPPO_OK;
   }
-  float2* part = reinterpret_cast<float2*>(ws + L.part);
-  float *z_a = reinterpret_cast<float*>(ws + L.z_a), *c2 = reinterpret_cast<float*>(ws + L.c2);
-  float *sgn = reinterpret_cast<float*>(ws + L.sgn), *fix = reinterpret_cast<float*>(ws + L.fix);
-  int32_t *idx = reinterpret_cast<int32_t*>(ws + L.idx), *pos = reinterpret_cast<int32_t*>(ws + L.pos);
-  int32_t *nlive = reinterpret_cast<int32_t*>(ws + L.nlive), *ids_c = reinterpret_cast<int32_t*>(ws + L.ids_c);
+  auto F = [&](size_t off) { return reinterpret_cast<float*>(ws + off); };
+  auto I = [&](size_t off) { return reinterpret_cast<int32_t*>(ws + off); };
   const __nv_bfloat16* hid = reinterpret_cast<const __nv_bfloat16*>(hidden);
+  const __nv_bfloat16* Wb = reinterpret_cast<const __nv_bfloat16*>(W);
   __nv_bfloat16* hc = reinterpret_cast<__nv_bfloat16*>(ws + L.hc);
-  auto gather = [&](const int32_t* n, bool coefs) {
-    GatherArgs ga = {};
-    ga.idx = idx; ga.n = n; ga.d = d; ga.src = hid; ga.dst = hc; ga.ids_in = sampled_ids; ga.ids_out = ids_c;
-    if (coefs) {
-      ga.f_in[0] = c2; ga.f_in[1] = sgn; ga.f_in[2] = fix;
-      ga.f_out[0] = reinterpret_cast<float*>(ws + L.c2c); ga.f_out[1] = reinterpret_cast<float*>(ws + L.sgnc);
-      ga.f_out[2] = reinterpret_cast<float*>(ws + L.fixc);
-    }
-    fused_gather_rows_kernel<<<(unsigned)T, 256, 0, st>>>(ga);
-    return cudaGetLastError();
-  };
-  // 1. W^T for the Top-K gather; with a token mask, the valid rows of hidden packed together for the statistics
+  __nv_bfloat16* E = reinterpret_cast<__nv_bfloat16*>(ws + L.E);
+  int32_t* counts = I(L.counts);
+  const int32_t *n_grad = counts, *n_valid = counts + 1, *n_resc = counts + 2;
+  const unsigned row_warps = (unsigned)((T + 7) / 8);
+  // 1. rows with a gradient to come (valid, advantage not zero) first, then the other valid rows; W^T for the Top-K gather
   if (K > 0) DPPO_TRY(transpose_bf16(W, d, V, V, ws + L.wt, d, st));
-  const void* a_stats = hidden;
-  const int32_t* ids_stats = sampled_ids;
-  const int32_t *m_stats = nullptr, *pos_stats = nullptr;
-  if (token_mask) {
-    fused_compact_rows_kernel<<<1, 1024, 0, st>>>(token_mask, nullptr, T, idx, pos, nlive);
+  fused_partition_rows_kernel<<<1, 1024, 0, st>>>(token_mask, advantages, nullptr, T, I(L.idx), I(L.pos), counts);
+  DPPO_TRY(cudaGetLastError());
+  {
+    GatherArgs ga = {};
+    ga.idx = I(L.idx); ga.n = n_valid; ga.d = d; ga.src = hid; ga.dst = hc; ga.ids_in = sampled_ids; ga.ids_out = I(L.ids_c);
+    ga.zero_fill = 1;
+    fused_gather_rows_kernel<<<(unsigned)T, 256, 0, st>>>(ga);
     DPPO_TRY(cudaGetLastError());
-    DPPO_TRY(gather(nlive, false));
-    a_stats = hc; ids_stats = ids_c; m_stats = nlive; pos_stats = pos;
   }
-  // 2. statistics of the logits
-  DPPO_TRY(cudaMemsetAsync(z_a, 0, (size_t)T * 4, st));
+  // 2. reference exponent of every packed row
+  fused_ref_logit_kernel<<<row_warps, 256, 0, st>>>(hc, Wb, T, d, V, I(L.ids_c), n_valid, F(L.cref2));
+  DPPO_TRY(cudaGetLastError());
+  // 3. forward GEMM: exponentials, their sums, z at the sampled id
+  DPPO_TRY(cudaMemsetAsync(F(L.z_a), 0, (size_t)T * 4, st));
   gemm::Params g1 = {};
-  g1.M = (int)T; g1.N = (int)V; g1.K = (int)d; g1.part = part; g1.z_a = z_a; g1.ids = ids_stats; g1.status = status;
-  g1.m_live = m_stats;
-  DPPO_TRY((launch_gemm<gemm::EPI_STATS, true>(a_stats, d, W, V, g1, st)));      // B = W [d, V], MN-major
-  // 3. per-row scalars, loss
+  g1.M = (int)T; g1.N = (int)V; g1.K = (int)d; g1.psum = F(L.psum); g1.z_a = F(L.z_a); g1.ids = I(L.ids_c); g1.cref2 = F(L.cref2);
+  g1.P = E; g1.ldp = L.lde; g1.status = status; g1.m_live = n_valid; g1.e_live = n_grad;
+  DPPO_TRY((launch_gemm<gemm::EPI_EXP, true>(hc, d, W, V, g1, st)));      // B = W [d, V], MN-major
+  // 4. per-row scalars
   float* z_topk = nullptr;
   if (K > 0) {      // logits at the rollout policy's top-K ids: T x K dot products against rows of W^T
-    z_topk = reinterpret_cast<float*>(ws + L.z_topk);
+    z_topk = F(L.z_topk);
     fused_topk_logits_kernel<<<(unsigned)((T * K + 7) / 8), 256, 0, st>>>(
         hid, reinterpret_cast<const __nv_bfloat16*>(ws + L.wt), T, d, V, mu_topk_ids, K, z_topk);
     DPPO_TRY(cudaGetLastError());
   }
-  fused_scalar_kernel<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(p, part, L.tiles_n, z_a, pos_stats, z_topk, c2, sgn, fix);
-  DPPO_TRY(cudaGetLastError());
+  {
+    ExpArgs x = {};
+    x.psum = F(L.psum); x.tiles_n = L.tiles_n; x.z_a = F(L.z_a); x.cref2 = F(L.cref2); x.pos = I(L.pos); x.n_grad = n_grad;
+    x.z_topk = z_topk; x.row_factor = F(L.factor); x.rescue = I(L.rescue); x.E = E; x.lde = L.lde;
+    fused_scalar_exp_kernel<<<row_warps, 256, 0, st>>>(p, x);
+    DPPO_TRY(cudaGetLastError());
+  }
+  // 5. rescue pass over the rows flagged by the scalar kernel (normally none: the GEMMs then have no tile to process)
+  {
+    fused_partition_rows_kernel<<<1, 1024, 0, st>>>(nullptr, nullptr, I(L.rescue), T, I(L.idx_r), I(L.pos_r), counts + 2);
+    DPPO_TRY(cudaGetLastError());
+    GatherArgs ga = {};
+    ga.idx = I(L.idx_r); ga.n = n_resc; ga.d = d; ga.src = hid; ga.dst = reinterpret_cast<__nv_bfloat16*>(ws + L.hr);
+    ga.ids_in = sampled_ids; ga.ids_out = I(L.ids_r); ga.zero_fill = 0;
+    fused_gather_rows_kernel<<<(unsigned)T, 256, 0, st>>>(ga);
+    DPPO_TRY(cudaGetLastError());
+    DPPO_TRY(cudaMemsetAsync(F(L.z_ar), 0, (size_t)T * 4, st));
+    gemm::Params gs = {};
+    gs.M = (int)T; gs.N = (int)V; gs.K = (int)d; gs.part = reinterpret_cast<float2*>(ws + L.part); gs.z_a = F(L.z_ar);
+    gs.ids = I(L.ids_r); gs.status = status; gs.m_live = n_resc; gs.allow_empty = 1;
+    DPPO_TRY((launch_gemm<gemm::EPI_STATS, true>(ws + L.hr, d, W, V, gs, st)));
+    RescueArgs x = {};
+    x.rescue = I(L.rescue); x.pos_r = I(L.pos_r); x.pos_e = I(L.pos);
+    x.part = reinterpret_cast<const float2*>(ws + L.part); x.tiles_n = L.tiles_n; x.z_a = F(L.z_ar); x.z_topk = z_topk;
+    x.c2 = F(L.c2); x.sgn = F(L.sgn); x.fix = F(L.fix); x.p_row_map = I(L.rmap); x.row_factor = F(L.factor);
+    fused_scalar_rescue_kernel<<<row_warps, 256, 0, st>>>(p, x);
+    DPPO_TRY(cudaGetLastError());
+    gemm::Params gg = {};
+    gg.M = (int)T; gg.N = (int)V; gg.K = (int)d; gg.ids = I(L.ids_r); gg.c2 = F(L.c2); gg.sgn = F(L.sgn); gg.fix = F(L.fix);
+    gg.P = E; gg.ldp = L.lde; gg.status = status; gg.m_live = n_resc; gg.allow_empty = 1; gg.p_row_map = I(L.rmap);
+    DPPO_TRY((launch_gemm<gemm::EPI_GRAD, true>(ws + L.hr, d, W, V, gg, st)));
+  }
   DPPO_TRY(launch_finalize(p, st));
-  // 4. rows whose gradient is zero (invalid, blocked by the mask, zero advantage) drop out of the backward: the rows
-  //    that remain are packed together, so the three GEMMs below run over *n_act rows instead of T
-  int32_t* n_act = nlive + 1;
-  fused_compact_rows_kernel<<<1, 1024, 0, st>>>(nullptr, sgn, T, idx, pos, n_act);
-  DPPO_TRY(cudaGetLastError());
-  DPPO_TRY(gather(n_act, true));
-  DPPO_TRY(transpose_bf16(hc, T, d, d, ws + L.ht, L.ldt, st));
-  // 5. gradient with respect to the logits of the packed rows, bf16, [T, ldp] (zero rows from *n_act to the tile's end)
-  gemm::Params g2 = {};
-  g2.M = (int)T; g2.N = (int)V; g2.K = (int)d; g2.ids = ids_c; g2.c2 = reinterpret_cast<float*>(ws + L.c2c);
-  g2.sgn = reinterpret_cast<float*>(ws + L.sgnc); g2.fix = reinterpret_cast<float*>(ws + L.fixc);
-  g2.P = reinterpret_cast<__nv_bfloat16*>(ws + L.P); g2.ldp = L.ldp; g2.status = status; g2.m_live = n_act;
-  DPPO_TRY((launch_gemm<gemm::EPI_GRAD, true>(hc, d, W, V, g2, st)));
-  // 6. dHidden[idx[i], :] = P[i, :] . W[d, V]^T; the other rows stay zero.  Few output tiles, very long K: K is cut in
-  //    two when that fills the waves better (two partial sums added into zeros, in either order the same result).
+  // 6. dHidden[idx[i], :] = factor[i] * (E[i, :] . W[d, V]^T) for the rows with a gradient; the other rows stay zero.
+  //    Few output tiles, very long K: K is cut in two when that fills the waves better (two partial sums added into
+  //    zeros, in either order the same result).
   gemm::Params g3 = {};
   g3.M = (int)T; g3.N = (int)d; g3.K = (int)V; g3.C = dHidden; g3.ldc = d; g3.status = status;
-  g3.m_live = n_act; g3.row_map = idx; g3.splits = -1;
-  DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(ws + L.P, L.ldp, W, V, g3, st));
-  // 7. dW[d, V] = packed hidden^T[d, n_act] . P[n_act, V]
+  g3.m_live = n_grad; g3.row_map = I(L.idx); g3.row_scale = F(L.factor); g3.splits = -1;
+  DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(E, L.lde, W, V, g3, st));
+  // 7. dW[d, V] = (factor * packed hidden)^T[d, n_grad] . E[n_grad, V]
+  DPPO_TRY(transpose_bf16(hc, T, d, d, ws + L.ht, L.ldt, st, F(L.factor), n_grad));
   gemm::Params g4 = {};
-  g4.M = (int)d; g4.N = (int)V; g4.K = (int)T; g4.C = dW; g4.ldc = V; g4.status = status; g4.k_live = n_act;
-  DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(ws + L.ht, L.ldt, ws + L.P, L.ldp, g4, st)));   // B = P [T, V], MN-major
+  g4.M = (int)d; g4.N = (int)V; g4.K = (int)T; g4.C = dW; g4.ldc = V; g4.status = status; g4.k_live = n_grad;
+  DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(ws + L.ht, L.ldt, E, L.lde, g4, st)));   // B = E [T, V], MN-major
 #undef DPPO_TRY
   return DPPO_OK;
 }

@@ -45,7 +45,7 @@ template <int CG> struct Cfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-enum { EPI_STORE_F32 = 0, EPI_STATS = 1, EPI_GRAD = 2 };
+enum { EPI_STORE_F32 = 0, EPI_STATS = 1, EPI_GRAD = 2, EPI_EXP = 3 };
 
 struct Params {
   int M, N, K;
@@ -61,6 +61,8 @@ struct Params {
   const int* m_live;
   const int* k_live;
   const int* row_map;    // EPI_STORE_F32: output row of tile row i (null: i); rows >= *m_live are not stored
+  const float* row_scale;  // EPI_STORE_F32: tile row i of the product is multiplied by row_scale[i] (null: 1)
+  int allow_empty;       // 1: *m_live == 0 means no tile at all (default: one row of tiles is always processed)
   // EPI_STATS: per (row, n-tile) partial (max, sum exp(z - max)); z at the sampled id
   float2* part;          // [M, tiles_n]
   float* z_a;            // [M]
@@ -73,6 +75,13 @@ struct Params {
   int64_t ldp;
   __nv_bfloat16* Pt;     // optional transposed copy [N, ldpt] (same values)
   int64_t ldpt;
+  const int* p_row_map;  // EPI_GRAD: row of P that tile row i is written to (null: i; < 0: not written); with a map only
+                         // the rows below *m_live are written
+  // EPI_EXP: E[row, col] = 2^(z*log2e - cref2[row]) in bf16 (written to P), per (row, n-tile) the fp32 sum of those
+  // exponentials before rounding, and z at the sampled id
+  const float* cref2;    // [M] per-row reference exponent, log2 units
+  float* psum;           // [M, tiles_n]
+  const int* e_live;     // rows of E that later steps read: rows below max(64, *e_live rounded up to 64) are written
   int32_t* status;
 };
 
@@ -248,7 +257,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   int m_lim = p.M, k_lim = p.K;
   if (p.m_live) { const int v = *p.m_live; m_lim = v < 0 ? 0 : (v < p.M ? v : p.M); }
   if (p.k_live) { const int v = *p.k_live; k_lim = v < 0 ? 0 : (v < p.K ? v : p.K); }
-  const int tiles_m = m_lim > 0 ? (m_lim + C::TILE_M - 1) / C::TILE_M : 1, tiles_n = (p.N + BN - 1) / BN;
+  int e_lim = p.M;
+  if (EPI == EPI_EXP && p.e_live) {
+    const int v = *p.e_live, up = v <= 64 ? 64 : (v + 63) / 64 * 64;
+    e_lim = up < p.M ? up : p.M;
+  }
+  const int tiles_m = m_lim > 0 ? (m_lim + C::TILE_M - 1) / C::TILE_M : (p.allow_empty ? 0 : 1), tiles_n = (p.N + BN - 1) / BN;
   const int ntiles = tiles_m * tiles_n;
   const int kblocks = k_lim > 0 ? (k_lim + BK - 1) / BK : 1;
   // work unit u = part * ntiles + tile: all tiles of one K part are in flight together and share operand strips
@@ -357,8 +371,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int row = m0 + q * 32 + lane;
-      // the gradient epilogue fills its whole tile (zero rows past the live extent feed the next GEMM's last K block)
-      const bool row_ok = (EPI == EPI_STORE_F32) ? row < m_lim : row < p.M;
+      // the gradient and exponential epilogues fill whole tiles (the rows past the live extent feed the last K block of
+      // a later GEMM and must hold finite values), unless the gradient rows go through a row map
+      const bool row_ok = (EPI == EPI_STORE_F32 || (EPI == EPI_GRAD && p.p_row_map)) ? row < m_lim : row < p.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * BN;
       if (EPI == EPI_STORE_F32) {
 #pragma unroll 1
@@ -367,6 +382,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
           tmem_ld32(taddr + c, r);
           if (row_ok) {
             float* dst = p.C + (int64_t)(p.row_map ? p.row_map[row] : row) * p.ldc + n0 + c;
+            if (p.row_scale) {
+              const float sc = p.row_scale[row];
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * sc);
+            }
             if (splits > 1) {              // partial sum over a K part: add into the zeroed output
 #pragma unroll
               for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) atomicAdd(dst + j, __uint_as_float(r[j]));
@@ -408,16 +428,59 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
           }
         }
         if (row_ok) p.part[(int64_t)row * tiles_n + nb] = make_float2(m, s);
-      } else {  // EPI_GRAD
+      } else if (EPI == EPI_EXP) {
         const int a = row_ok ? p.ids[row] : -1;
-        const float c2 = row_ok ? p.c2[row] : 0.f, sg = row_ok ? p.sgn[row] : 0.f, fx = row_ok ? p.fix[row] : 0.f;
-        const uint32_t sign2 = (sg < 0.f) ? 0x80008000u : 0u;
+        const float ncr = row_ok ? -p.cref2[row] : 0.f;
+        const bool store = row_ok && row < e_lim;
+        float s = 0.f;
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
           uint32_t r[32];
           tmem_ld32(taddr + c, r);
           const int col0 = n0 + c;
-          if (row_ok && col0 < p.N) {
+          if (col0 < p.N) {
+            uint32_t o[16];
+            float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              float v0 = ex2(fmaf(__uint_as_float(r[j]), 1.4426950408889634f, ncr));
+              float v1 = ex2(fmaf(__uint_as_float(r[j + 1]), 1.4426950408889634f, ncr));
+              if (col0 + j >= p.N) v0 = 0.f;
+              if (col0 + j + 1 >= p.N) v1 = 0.f;
+              acc0 += v0;
+              acc1 += v1;
+              __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+              o[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            s += acc0 + acc1;
+            if (a >= col0 && a < col0 + 32) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) if (col0 + j == a) p.z_a[row] = __uint_as_float(r[j]);
+            }
+            if (store) {
+              __nv_bfloat16* dst = p.P + (int64_t)row * p.ldp + col0;
+              if (col0 + 32 <= p.N) {
+#pragma unroll
+                for (int j = 0; j < 16; j += 4) *reinterpret_cast<uint4*>(dst + 2 * j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+              } else {
+                for (int j = 0; j < 32; ++j)
+                  if (col0 + j < p.N) dst[j] = __ushort_as_bfloat16((unsigned short)((j & 1) ? (o[j >> 1] >> 16) : (o[j >> 1] & 0xffffu)));
+              }
+            }
+          }
+        }
+        if (row_ok) p.psum[(int64_t)row * tiles_n + nb] = s;
+      } else {  // EPI_GRAD
+        const int a = row_ok ? p.ids[row] : -1;
+        const float c2 = row_ok ? p.c2[row] : 0.f, sg = row_ok ? p.sgn[row] : 0.f, fx = row_ok ? p.fix[row] : 0.f;
+        const uint32_t sign2 = (sg < 0.f) ? 0x80008000u : 0u;
+        const int prow = (row_ok && p.p_row_map) ? p.p_row_map[row] : row;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          const int col0 = n0 + c;
+          if (row_ok && prow >= 0 && col0 < p.N) {
             uint32_t o[16];
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
@@ -435,7 +498,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
               for (int j = 0; j < 32; ++j)
                 if (col0 + j < p.N) dt[(int64_t)j * p.ldpt] = (unsigned short)((j & 1) ? (o[j >> 1] >> 16) : (o[j >> 1] & 0xffffu));
             }
-            __nv_bfloat16* dst = p.P + (int64_t)row * p.ldp + col0;
+            __nv_bfloat16* dst = p.P + (int64_t)prow * p.ldp + col0;
             if (col0 + 32 <= p.N) {
 #pragma unroll
               for (int j = 0; j < 16; j += 4) *reinterpret_cast<uint4*>(dst + 2 * j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
