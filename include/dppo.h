@@ -213,17 +213,21 @@ size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V, int K);
  *  hidden   [T, d] bf16 row-major;  W  [d, V] bf16 row-major (LM head);  d and V multiples of 8, 16-byte aligned.
  *  sampled_ids, mu_logp, advantages, token_mask, delta, opts, loss, divergence, mask, stats, status: as for
  *           dppo_loss_fwd_bwd.  mu_topk_ids / mu_topk_p [T, K]: as for dppo_loss_fwd_bwd (Top-K variants; the K
- *           logits per row are recomputed as dot products, K is ignored by the other variants).
+ *           logits per row are computed as dot products, K is ignored by the other variants).
  *  dHidden  [T, d] fp32 out: d loss / d hidden = dlogits . W^T.
  *  dW       [d, V] fp32 out: d loss / d W = hidden^T . dlogits (overwritten, not accumulated).
- *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V, K) bytes; it holds a packed copy of hidden
- *           and its transpose and the bf16 gradient with respect to the logits (about 2 T V bytes; plus W^T,
- *           2 d V bytes, for Top-K variants).
- * The gradient with respect to the logits is rounded to bf16 before the two gradient GEMMs (fp32 accumulation).
- * Rows whose gradient is zero (token_mask 0, blocked by the trust-region mask, zero advantage) are left out of the three
- * backward GEMMs: the remaining rows are packed on the device, their count is never read by the host, and the call
- * stays asynchronous.  Rows with token_mask 0 are left out of the forward GEMM as well.  The outputs are the same as
- * without packing: such rows of dHidden are zero.
+ *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V, K) bytes; it holds packed copies of hidden
+ *           and the bf16 exponentials of the logits (about 2 T V bytes; plus W^T, 2 d V bytes, for Top-K variants).
+ * Every logits tile is computed once: the forward GEMM writes exp(z - c_t) in bf16 against a per-row reference known
+ * beforehand (c_t = the sampled token's logit) together with the fp32 row sums; the per-row factor g_t / S_t that turns
+ * those exponentials into the gradient with respect to the logits is applied to the rows of dHidden in fp32 and to the
+ * hidden rows (bf16) in front of the dW GEMM.  Entrywise accuracy: |error of dHidden| <= 2^-8 |dlogits| |W|^T,
+ * |error of dW| <= 2^-7 |hidden|^T |dlogits| (one resp. two bf16 roundings, fp32 accumulation).  Rows for which the
+ * reference is unusable (pi(a_t) below 2^-60, non-finite logits) are recomputed by a two-pass route inside the same
+ * call; non-finite rows raise DPPO_STATUS_NONFINITE_ROW and are dropped.
+ * Rows with token_mask 0 are left out of every GEMM, rows with zero advantage out of the two backward GEMMs: the
+ * remaining rows are packed on the device, their count is never read by the host, and the call stays asynchronous.
+ * The outputs are the same as without packing: such rows of dHidden are zero.
  */
 int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int64_t d, int64_t V,
                               const int32_t* sampled_ids, const float* mu_logp,
