@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--fused-rows", type=int, default=8192, help="token rows of the fused measurement; anything but 8192 is a reduced profiling case")
     ap.add_argument("--no-fused", action="store_true", help="skip the fused LM-head measurement (reported as an extra object at N=1)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-variants", action="store_true", help="skip the other streaming configurations and the exact-divergence monitor (extra objects at N=1)")
+    ap.add_argument("--variants-only", action="store_true", help="run only those extra measurements (profiling aid)")
     return ap.parse_args()
 
 
@@ -115,6 +117,76 @@ def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
                          "flop_count": "6*T*d*V (forward, dHidden, dW); nothing is recomputed"},
             "gpu_launches_per_step": 15, "loss": float(out["loss"].item()),
             "ms_per_step_quarter_of_responses_zero_advantage": ms_sparse}
+
+
+def _time_steps(torch, fn, steps, warmup):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def bench_other_configs(dppo, wl, dev, steps=20, warmup=3, n_resp=16):
+    """The other streaming configurations at full size (same kernel, other variant switches), and the exact
+    full-vocabulary divergence monitor.  Extra objects of the benchmark line; the headline stays Binary-TV."""
+    import torch
+    peak, src = measured_peaks()
+    out = {}
+
+    def entry(ms, rows, valid, bytes_moved, note):
+        gbs = bytes_moved / (ms * 1e-3) / 1e9
+        return {"ms_per_step": ms, "rows_per_s": rows / (ms * 1e-3), "valid_tokens_per_s": valid / (ms * 1e-3),
+                "achieved_gbs": gbs, "frac_of_hbm_peak": gbs / peak, "peak_source": "of " + src, "note": note}
+
+    # Binary-KL and Top-K TV (K = 20) on the Qwen3-vocabulary rows
+    b = wl.qwen_vocab_rows(dev, seed=1, K=20, n_resp=n_resp, group=min(16, n_resp))     # n_resp != 16: reduced profiling case
+    T = b.T
+    dl = torch.empty_like(b.logits)
+    ws = torch.empty(dppo.dppo_workspace_bytes(T), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    for name, variant, K, delta in (("binary_kl_delta0.1", dppo.BINARY_KL, 0, 0.1), ("topk_tv_k20_delta0.2", dppo.TOPK_TV, 20, 0.2)):
+        fn = lambda: dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, variant, K, delta,
+                                            b.mu_topk_ids, b.mu_topk_p, dlogits=dl, workspace=ws, status=status)
+        ms = _time_steps(torch, fn, steps, warmup)
+        out[name] = entry(ms, T, T, T * BYTES_PER_TOKEN, f"T={T}, V=151936, bf16 in/out; bytes = logits read + dlogits written")
+    # exact full-vocabulary TV / KL / entropy from the trainer's and the rollout's logits (two tensors read, nothing written)
+    zmu = torch.empty_like(b.logits)
+    g = torch.Generator(device=dev).manual_seed(77)
+    for r0 in range(0, T, 1024):
+        zmu[r0:r0 + 1024] = (b.logits[r0:r0 + 1024].float() + 0.1 * torch.randn((min(1024, T - r0), VOCAB), generator=g, device=dev)).to(torch.bfloat16)
+    ms = _time_steps(torch, lambda: dppo.dppo_exact_divergence(b.logits, zmu, status=status), steps, warmup)
+    out["exact_divergence"] = entry(ms, T, T, T * BYTES_PER_TOKEN, f"dppo_exact_divergence, T={T}, V=151936, bf16; bytes = both logits tensors read once "
+                                    "(the second sweep is served by L2); 4 exp per element pair: the special-function pipe, not HBM, bounds it")
+    assert int(status.item()) == 0
+    del b, dl, zmu
+    torch.cuda.empty_cache()
+    # Top-K KL, K = 64, ragged: two padded responses of the 64 (8192 rows each) with their token mask and the global scale
+    lengths = wl.ragged_lengths()
+    blocks = [wl.ragged_response(dev, i, lengths) for i in (0, 1)]
+    cat = lambda xs: torch.cat(xs).contiguous()
+    lg = cat([x.logits for x in blocks])
+    for x in blocks:
+        x.logits = None
+    ids, mu, adv = cat([x.sampled_ids for x in blocks]), cat([x.mu_logp for x in blocks]), cat([x.advantages for x in blocks])
+    tok, kid, kp = cat([x.token_mask for x in blocks]), cat([x.mu_topk_ids for x in blocks]), cat([x.mu_topk_p for x in blocks])
+    T2, valid = lg.shape[0], int(tok.sum().item())
+    dl = torch.empty_like(lg)
+    ws = torch.empty(dppo.dppo_workspace_bytes(T2), dtype=torch.uint8, device=dev)
+    scale = 1.0 / float(sum(lengths))
+    fn = lambda: dppo.dppo_loss_fwd_bwd(lg, ids, mu, adv, tok, dppo.TOPK_KL, 64, 0.05, kid, kp, loss_scale=scale,
+                                        dlogits=dl, workspace=ws, status=status)
+    ms = _time_steps(torch, fn, steps, warmup)
+    assert int(status.item()) == 0
+    out["topk_kl_k64_ragged_delta0.05"] = entry(ms, T2, valid, valid * BYTES_PER_TOKEN + (T2 - valid) * 2 * VOCAB,
+                                                f"responses 0 and 1 of the 64 as padded blocks of 8192 rows ({valid} valid of {T2}); "
+                                                "bytes = valid rows read + every row of dlogits written (padding rows are zero-filled)")
+    return out
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one full-size launch of the row kernel, from the ncu
@@ -262,6 +334,11 @@ def run_ours(args):
         print(json.dumps({"fused_lm_head": bench_fused(dppo, wl, dev, steps=max(1, min(args.steps, 10)), warmup=max(1, min(args.warmup, 3)), T=args.fused_rows)}))
         return
 
+    if args.variants_only:
+        print(json.dumps({"other_configs": bench_other_configs(dppo, wl, dev, steps=max(1, min(args.steps, 20)), warmup=max(1, min(args.warmup, 3)),
+                                                                 n_resp=max(1, args.rows // 1024))}))
+        return
+
     # each rank owns T rows of the global batch of world*T rows
     b = wl.qwen_vocab_rows(dev, seed=1 + rank, rows=args.rows) if args.rows != T_ROWS else wl.qwen_vocab_rows(dev, seed=1 + rank)
     T = b.T
@@ -359,6 +436,9 @@ def run_ours(args):
         b.logits = None
         torch.cuda.empty_cache()
         line["fused_lm_head"] = bench_fused(dppo, wl, dev)
+        if not args.no_variants:
+            torch.cuda.empty_cache()
+            line["other_configs"] = bench_other_configs(dppo, wl, dev)
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import dppo_oracle as O

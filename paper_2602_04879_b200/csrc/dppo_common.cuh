@@ -94,10 +94,12 @@ __device__ __forceinline__ double xlogx_over_y(double x, double y) {
 // Per-row scalar stage, run by ONE full warp (all 32 lanes call it with the same arguments).
 //   lse        log-sum-exp of the row (double, from fp32 partial sums)
 //   z_at(id, k)  fp32 value of this row's logit `id`; k is its position in the top-K list, -1 for the sampled id
+//   list_at(k, id, pm)  entry k of the row's top-K list (id and rollout probability); a caller that fetched the list
+//                earlier hands it over here, the default reads it from global memory
 // Returns on every lane the same values.  `flags` receives DPPO_STATUS_* bits found here.
-template <typename ZAt>
+template <typename ZAt, typename ListAt>
 __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, int a, double lse, double scale,
-                                                 ZAt z_at, float& D_out, int& M_out, double& g_out,
+                                                 ZAt z_at, ListAt list_at, float& D_out, int& M_out, double& g_out,
                                                  float& r_out, float& absdiff_out, double& pi_a_out, int& flags) {
   const int lane = threadIdx.x & 31;
   const double mu_logp = (double)p.mu_logp[t];
@@ -122,26 +124,24 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
     D = first + xlogx_over_y(-expm1(mu_logp), -expm1(lpa));
   } else {
     // Reduced categorical over set(top-K ids) u {a} u {other}  (Sec. 4.4, Eq. topk_tv / topk_kl)
-    double sum_mu = 0.0, sum_pi = 0.0, tv = 0.0, kl = 0.0;
+    // per list entry in fp32 (log pi from the double lse, then expf / logf: relative error ~1e-7, two orders below the
+    // tolerance of D); the lane's partial sums go to double for the reduction across the warp
+    float l_mu = 0.f, l_pi = 0.f, l_tv = 0.f, l_kl = 0.f;
     int in_list = 0, bad = 0;
-    const int32_t* ids = p.topk_ids + t * (int64_t)p.K;
-    const float* ps = p.topk_p + t * (int64_t)p.K;
     for (int k = lane; k < p.K; k += 32) {
-      int id = ids[k];
+      int id;
+      float pm;
+      list_at(k, id, pm);
       if (id < 0 || (int64_t)id >= p.V) { bad = 1; continue; }
-      double pm = (double)ps[k];
-      double lpk = (double)z_at(id, k) - lse;
-      double pk = exp(lpk);
-      sum_mu += pm;
-      sum_pi += pk;
-      tv += fabs(pm - pk);
-      if (pm > 0.0) kl += pm * (log(pm) - lpk);
+      const float lpk = (float)((double)z_at(id, k) - lse);
+      const float pk = expf(lpk);
+      l_mu += pm;
+      l_pi += pk;
+      l_tv += fabsf(pm - pk);
+      if (pm > 0.f) l_kl += pm * (logf(pm) - lpk);
       in_list |= (id == a);
     }
-    sum_mu = warp_sum(sum_mu);
-    sum_pi = warp_sum(sum_pi);
-    tv = warp_sum(tv);
-    kl = warp_sum(kl);
+    double sum_mu = warp_sum((double)l_mu), sum_pi = warp_sum((double)l_pi), tv = warp_sum((double)l_tv), kl = warp_sum((double)l_kl);
     in_list = __any_sync(0xffffffffu, in_list);
     bad = __any_sync(0xffffffffu, bad);
     if (bad) flags |= DPPO_STATUS_BAD_TOPK_ID;
@@ -169,6 +169,16 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
   r_out = (float)r;
   absdiff_out = (float)fabs(mu_a - pi_a);
   pi_a_out = pi_a;
+}
+
+template <typename ZAt>
+__device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, int a, double lse, double scale,
+                                                 ZAt z_at, float& D_out, int& M_out, double& g_out,
+                                                 float& r_out, float& absdiff_out, double& pi_a_out, int& flags) {
+  const int32_t* ids = p.topk_ids + t * (int64_t)p.K;
+  const float* ps = p.topk_p + t * (int64_t)p.K;
+  auto list_at = [&](int k, int& id, float& pm) { id = ids[k]; pm = ps[k]; };
+  row_scalars_warp(p, t, a, lse, scale, z_at, list_at, D_out, M_out, g_out, r_out, absdiff_out, pi_a_out, flags);
 }
 
 // Turns g, lse into the coefficients of the gradient sweep.

@@ -5,12 +5,18 @@
 //   sweep 1  online sums of both rows: (m, S, A = sum e^(z-m) z) for pi and (m', S', B = sum e^(z'-m') (z' - z)) for mu
 //            -> lse, entropy = lse - A/S, KL = B/S' - lse' + lse
 //   sweep 2  TV = 1/2 sum |e^(z'-lse') - e^(z-lse)|   (second read of both rows, normally from L2)
+// One CTA of 512 threads per SM: the row pairs in flight (148 x 608 KB at V = 151936 bf16) then fit in L2 for the
+// second read.  With 16-byte aligned rows the sweeps run on whole 8-element vectors, two vectors of each row in flight
+// per thread while a third is computed on, and the per-thread reference of the sums only moves when a vector would
+// otherwise grow past 2^23.
 #include "dppo_common.cuh"
+#include "dppo_pipe.cuh"
 
 namespace dppo {
 namespace {
 
 constexpr int kThreads = 512;
+constexpr float kRefMargin = 16.f;      // a vector may exceed the running reference by this much before it moves
 
 struct ExactParams {
   const void* z; const void* zmu;
@@ -34,6 +40,28 @@ struct Acc3 {
       a = fmaf(e, (e > 0.f) ? w : 0.f, a);              // e = 0 (x = -inf): contributes nothing even if w is inf/nan
     }
   }
+  // N values at once against a reference that moves rarely: m stays put while the vector's maximum is within
+  // kRefMargin above it (the sums are relative to m, whatever m is)
+  template <int N>
+  __device__ __forceinline__ void addN(const float* x, const float* w) {
+    float vm = x[0];
+#pragma unroll
+    for (int i = 1; i < N; ++i) asm("max.NaN.f32 %0, %0, %1;" : "+f"(vm) : "f"(x[i]));
+    if (!(vm <= m + kRefMargin)) {                      // above the margin, the first finite vector, or NaN
+      const float f = ex2_approx((m - vm) * kLog2e);    // m = -inf gives 0
+      s *= f; a *= f; m = vm;
+    }
+    if (m != -INFINITY) {
+      const float c = -m * kLog2e;
+#pragma unroll
+      for (int i = 0; i < N; ++i) {
+        const float e = ex2_approx(fmaf(x[i], kLog2e, c));
+        s += e;
+        a = fmaf(e, (e > 0.f) ? w[i] : 0.f, a);
+      }
+    }
+  }
+  __device__ __forceinline__ void add8(const float* x, const float* w) { addN<8>(x, w); }
   __device__ __forceinline__ void merge(const Acc3& o) {
     const float mn = fmaxf(m, o.m);
     if (mn == -INFINITY) return;
@@ -72,8 +100,55 @@ __device__ __forceinline__ void load8<float>(const float* p, int64_t j, int64_t 
   }
 }
 
+// Whole 8-element vectors of an aligned row: raw 16-byte loads first (several in flight), unpacked when used.
+template <typename InT> struct Raw8;
+template <> struct Raw8<__nv_bfloat16> {
+  uint4 v;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = *reinterpret_cast<const uint4*>(p); }
+  __device__ __forceinline__ void unpack(float* o) const {
+    o[0] = __uint_as_float(v.x << 16); o[1] = __uint_as_float(v.x & 0xffff0000u);
+    o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
+    o[4] = __uint_as_float(v.z << 16); o[5] = __uint_as_float(v.z & 0xffff0000u);
+    o[6] = __uint_as_float(v.w << 16); o[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+};
+template <> struct Raw8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load(const float* p) {
+    a = *reinterpret_cast<const float4*>(p);
+    b = *reinterpret_cast<const float4*>(p + 4);
+  }
+  __device__ __forceinline__ void unpack(float* o) const {
+    o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+  }
+};
+
+// Walks the whole 8-element vectors j = tid*8, +kStep, ... of an aligned row pair and hands them to f8(a[8], b[8]) as
+// floats; two vector pairs are kept in flight: a buffer is unpacked, refilled with the pair two steps ahead, and only
+// then computed on, so that the loads overlap the arithmetic.  Returns the first j that was not processed.
+template <typename InT, typename F8>
+__device__ __forceinline__ int64_t sweep_vectors(const InT* z, const InT* zm, int64_t V, int64_t j, int64_t step, F8&& f8) {
+  Raw8<InT> a0, b0, a1, b1;
+  if (j + 8 <= V) { a0.load(z + j); b0.load(zm + j); }
+  if (j + step + 8 <= V) { a1.load(z + j + step); b1.load(zm + j + step); }
+  for (;;) {
+    float a[8], b[8];
+    if (j + 8 > V) break;
+    a0.unpack(a); b0.unpack(b);
+    if (j + 2 * step + 8 <= V) { a0.load(z + j + 2 * step); b0.load(zm + j + 2 * step); }
+    f8(a, b);
+    j += step;
+    if (j + 8 > V) break;
+    a1.unpack(a); b1.unpack(b);
+    if (j + 2 * step + 8 <= V) { a1.load(z + j + 2 * step); b1.load(zm + j + 2 * step); }
+    f8(a, b);
+    j += step;
+  }
+  return j;
+}
+
 template <typename InT>
-__global__ void __launch_bounds__(kThreads) dppo_exact_kernel(ExactParams p, int vec_ok) {
+__global__ void __launch_bounds__(kThreads, 1) dppo_exact_kernel(ExactParams p, int vec_ok) {
   __shared__ Acc3 s_pi[kThreads / 32], s_mu[kThreads / 32];
   __shared__ double s_tv[kThreads / 32];
   __shared__ float s_lse[2];
@@ -90,7 +165,16 @@ __global__ void __launch_bounds__(kThreads) dppo_exact_kernel(ExactParams p, int
     const InT* zm = ZM + t * p.ld_mu;
     // ---- sweep 1
     Acc3 api{-INFINITY, 0.f, 0.f}, amu{-INFINITY, 0.f, 0.f};
-    for (int64_t j = (int64_t)tid * 8; j < p.V; j += (int64_t)kThreads * 8) {
+    constexpr int64_t kStep = (int64_t)kThreads * 8;
+    int64_t j = (int64_t)tid * 8;
+    if (vec_ok)
+      j = sweep_vectors<InT>(z, zm, p.V, j, kStep, [&](float* a, const float* b) {
+        api.add8(a, a);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a[i] = b[i] - a[i];
+        amu.add8(b, a);
+      });
+    for (; j < p.V; j += kStep) {
       float a[8], b[8];
       int n, n2;
       load8<InT>(z, j, p.V, vec_ok, a, n);
@@ -106,26 +190,33 @@ __global__ void __launch_bounds__(kThreads) dppo_exact_kernel(ExactParams p, int
     }
     if (lane == 0) { s_pi[warp] = api; s_mu[warp] = amu; }
     __syncthreads();
-    if (tid == 0) {
-      // fixed order, double precision
-      float mp = -INFINITY, mq = -INFINITY;
-      for (int w = 0; w < kThreads / 32; ++w) { mp = fmaxf(mp, s_pi[w].m); mq = fmaxf(mq, s_mu[w].m); }
-      double Sp = 0, Ap = 0, Sq = 0, Bq = 0;
-      for (int w = 0; w < kThreads / 32; ++w) {
-        if (s_pi[w].s > 0.f || s_pi[w].s != s_pi[w].s) { const double f = exp((double)s_pi[w].m - (double)mp); Sp += f * s_pi[w].s; Ap += f * s_pi[w].a; }
-        if (s_mu[w].s > 0.f || s_mu[w].s != s_mu[w].s) { const double f = exp((double)s_mu[w].m - (double)mq); Sq += f * s_mu[w].s; Bq += f * s_mu[w].a; }
+    if (warp == 0) {
+      // the warps' partials, one per lane, merged by the same fp32 rule as inside a warp; the last step in double
+      constexpr int kWarps = kThreads / 32;
+      static_assert(kWarps <= 32, "one lane per warp");
+      Acc3 xp{-INFINITY, 0.f, 0.f}, xq{-INFINITY, 0.f, 0.f};
+      if (lane < kWarps) { xp = s_pi[lane]; xq = s_mu[lane]; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        Acc3 x{__shfl_xor_sync(0xffffffffu, xp.m, o), __shfl_xor_sync(0xffffffffu, xp.s, o), __shfl_xor_sync(0xffffffffu, xp.a, o)};
+        Acc3 y{__shfl_xor_sync(0xffffffffu, xq.m, o), __shfl_xor_sync(0xffffffffu, xq.s, o), __shfl_xor_sync(0xffffffffu, xq.a, o)};
+        xp.merge(x);
+        xq.merge(y);
       }
-      const double lse_p = (double)mp + log(Sp), lse_q = (double)mq + log(Sq);
-      const bool ok = isfinite(lse_p) && isfinite(lse_q);
-      s_bad = ok ? 0 : 1;
-      s_lse[0] = (float)lse_p;
-      s_lse[1] = (float)lse_q;
-      if (ok) {
-        p.entropy[t] = (float)(lse_p - Ap / Sp);
-        p.kl[t] = (float)(Bq / Sq - lse_q + lse_p);
-      } else {
-        p.entropy[t] = 0.f; p.kl[t] = 0.f; p.tv[t] = 0.f;
-        atomicOr(p.status, DPPO_STATUS_NONFINITE_ROW);
+      if (lane == 0) {
+        const double Sp = xp.s, Ap = xp.a, Sq = xq.s, Bq = xq.a;
+        const double lse_p = (double)xp.m + log(Sp), lse_q = (double)xq.m + log(Sq);
+        const bool ok = isfinite(lse_p) && isfinite(lse_q);
+        s_bad = ok ? 0 : 1;
+        s_lse[0] = (float)lse_p;
+        s_lse[1] = (float)lse_q;
+        if (ok) {
+          p.entropy[t] = (float)(lse_p - Ap / Sp);
+          p.kl[t] = (float)(Bq / Sq - lse_q + lse_p);
+        } else {
+          p.entropy[t] = 0.f; p.kl[t] = 0.f; p.tv[t] = 0.f;
+          atomicOr(p.status, DPPO_STATUS_NONFINITE_ROW);
+        }
       }
     }
     __syncthreads();
@@ -133,7 +224,15 @@ __global__ void __launch_bounds__(kThreads) dppo_exact_kernel(ExactParams p, int
     // ---- sweep 2: total variation with both normalisers known
     const float cp = -s_lse[0] * kLog2e, cq = -s_lse[1] * kLog2e;
     float acc = 0.f;
-    for (int64_t j = (int64_t)tid * 8; j < p.V; j += (int64_t)kThreads * 8) {
+    j = (int64_t)tid * 8;
+    if (vec_ok)
+      j = sweep_vectors<InT>(z, zm, p.V, j, kStep, [&](const float* a, const float* b) {
+        float part = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) part += fabsf(ex2_approx(fmaf(b[i], kLog2e, cq)) - ex2_approx(fmaf(a[i], kLog2e, cp)));
+        acc += part;
+      });
+    for (; j < p.V; j += kStep) {
       float a[8], b[8];
       int n, n2;
       load8<InT>(z, j, p.V, vec_ok, a, n);
@@ -151,6 +250,221 @@ __global__ void __launch_bounds__(kThreads) dppo_exact_kernel(ExactParams p, int
     }
     __syncthreads();
   }
+}
+
+// ---- 16-byte aligned rows: the same two sweeps fed through a shared-memory ring ------------------------------------
+// One producer lane streams the chunks of the row pair (16 KB of each tensor per slot) with bulk asynchronous copies,
+// first for sweep 1 (from HBM, kept in L2), then again for sweep 2 (normally from L2), and simply runs ahead as far as
+// the ring allows: the consumer warps never wait on global memory, and the copies for sweep 2 are already in flight
+// while the row's normalisers are being reduced.  Consumers synchronise among themselves through mbarriers only, so
+// every wait in the kernel is bounded (about 2 s; then DPPO_STATUS_WAIT_LIMIT is raised and the CTA leaves).
+constexpr int kXChunk = 16384;                       // bytes per tensor per slot
+constexpr int kXSlots = 6;
+constexpr int kXConsumers = 512;
+constexpr int kXWarps = kXConsumers / 32;
+constexpr int kXThreads = kXConsumers + 32;          // + producer warp
+constexpr int kXVec = kXChunk / 16 / kXConsumers;    // 16-byte vectors per thread per chunk and tensor
+constexpr int kXMiscBytes = 1024;
+static_assert(kXVec * kXConsumers * 16 == kXChunk, "chunk geometry");
+
+struct XMisc {
+  unsigned long long full[kXSlots], empty[kXSlots];
+  unsigned long long red[2];             // all consumer warps have posted their partials (sweep 1 / sweep 2)
+  Acc3 pi[kXWarps], mu[kXWarps];
+  double tv[kXWarps];
+  int abort_flag;
+};
+static_assert(sizeof(XMisc) <= kXMiscBytes, "misc area");
+
+template <typename InT> struct XVecOf;
+template <> struct XVecOf<__nv_bfloat16> {
+  static constexpr int N = 8;
+  static __device__ __forceinline__ void unpack(const uint4& v, float* z) {
+    z[0] = __uint_as_float(v.x << 16); z[1] = __uint_as_float(v.x & 0xffff0000u);
+    z[2] = __uint_as_float(v.y << 16); z[3] = __uint_as_float(v.y & 0xffff0000u);
+    z[4] = __uint_as_float(v.z << 16); z[5] = __uint_as_float(v.z & 0xffff0000u);
+    z[6] = __uint_as_float(v.w << 16); z[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+};
+template <> struct XVecOf<float> {
+  static constexpr int N = 4;
+  static __device__ __forceinline__ void unpack(const uint4& v, float* z) {
+    z[0] = __uint_as_float(v.x); z[1] = __uint_as_float(v.y); z[2] = __uint_as_float(v.z); z[3] = __uint_as_float(v.w);
+  }
+};
+
+template <typename InT>
+__global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  constexpr int N = XVecOf<InT>::N;
+  XMisc* misc = reinterpret_cast<XMisc*>(smem + (size_t)kXSlots * 2 * kXChunk);
+  const uint32_t slots_base = smem_u32(smem);
+  const uint32_t full_base = smem_u32(&misc->full[0]), empty_base = smem_u32(&misc->empty[0]), red_base = smem_u32(&misc->red[0]);
+  volatile int* abort_flag = &misc->abort_flag;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    for (int i = 0; i < kXSlots; ++i) { mbar_init(full_base + 8u * i, 1); mbar_init(empty_base + 8u * i, kXWarps); }
+    mbar_init(red_base, kXWarps);
+    mbar_init(red_base + 8u, kXWarps);
+    misc->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  const uint32_t row_bytes = (uint32_t)(p.V * (int64_t)sizeof(InT));     // launcher guarantees < 2^31
+  const int C = (int)((row_bytes + kXChunk - 1) / kXChunk);
+  const InT* Z = reinterpret_cast<const InT*>(p.z);
+  const InT* ZM = reinterpret_cast<const InT*>(p.zmu);
+
+  if (warp == kXWarps) {
+    // ------------------------------------------------------------------ producer (one lane)
+    if (lane == 0) {
+      uint64_t keep, drop;
+      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(drop));
+      uint32_t it = 0;
+      bool ok = true;
+      for (int64_t t = blockIdx.x; t < p.T && ok; t += gridDim.x) {
+        if (p.token_mask && p.token_mask[t] == 0) continue;
+        const char* z = reinterpret_cast<const char*>(Z + t * p.ld_z);
+        const char* zm = reinterpret_cast<const char*>(ZM + t * p.ld_mu);
+        for (int pass = 0; pass < 2 && ok; ++pass) {
+          for (int c = 0; c < C; ++c, ++it) {
+            const uint32_t slot = it % kXSlots, use = it / kXSlots;
+            if (use > 0 && !mbar_wait(empty_base + 8u * slot, (use - 1u) & 1u, abort_flag)) { ok = false; break; }
+            const uint32_t off = (uint32_t)c * kXChunk;
+            const uint32_t bytes = (row_bytes - off) < (uint32_t)kXChunk ? (row_bytes - off) : (uint32_t)kXChunk;
+            const uint32_t bar = full_base + 8u * slot, dst = slots_base + slot * (2u * kXChunk);
+            mbar_arrive_expect_tx(bar, 2u * bytes);
+            bulk_load(dst, z + off, bytes, bar, pass == 0 ? keep : drop);
+            bulk_load(dst + kXChunk, zm + off, bytes, bar, pass == 0 ? keep : drop);
+          }
+        }
+      }
+      if (!ok) {      // gave up: let the copies still in flight land before this CTA's shared memory goes away
+        const unsigned long long t_exit = globaltimer_ns();
+        while (globaltimer_ns() - t_exit < 1000000ull) __nanosleep(1000);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers
+    uint32_t it = 0, nrow = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < p.T && ok; t += gridDim.x) {
+      if (p.token_mask && p.token_mask[t] == 0) {
+        if (tid == 0) { p.tv[t] = 0.f; p.kl[t] = 0.f; p.entropy[t] = 0.f; }
+        continue;
+      }
+      // ---- sweep 1
+      Acc3 api{-INFINITY, 0.f, 0.f}, amu{-INFINITY, 0.f, 0.f};
+      for (int c = 0; c < C && ok; ++c, ++it) {
+        const uint32_t slot = it % kXSlots, use = it / kXSlots;
+        ok = mbar_wait_warp(full_base + 8u * slot, use & 1u, abort_flag);
+        if (!ok) break;
+        const uint32_t off = (uint32_t)c * kXChunk;
+        const uint32_t nvec = ((row_bytes - off) < (uint32_t)kXChunk ? (row_bytes - off) : (uint32_t)kXChunk) / 16u;
+        const uint32_t sa = slots_base + slot * (2u * kXChunk), sb = sa + kXChunk;
+        uint4 va[kXVec], vb[kXVec];
+#pragma unroll
+        for (int k = 0; k < kXVec; ++k) {
+          const uint32_t v = (uint32_t)k * kXConsumers + (uint32_t)tid;
+          if (v < nvec) { va[k] = lds128(sa + v * 16u); vb[k] = lds128(sb + v * 16u); }
+        }
+#pragma unroll
+        for (int k = 0; k < kXVec; ++k) {
+          if ((uint32_t)k * kXConsumers + (uint32_t)tid < nvec) {
+            float a[N], b[N];
+            XVecOf<InT>::unpack(va[k], a);
+            XVecOf<InT>::unpack(vb[k], b);
+            api.addN<N>(a, a);
+#pragma unroll
+            for (int i = 0; i < N; ++i) a[i] = b[i] - a[i];
+            amu.addN<N>(b, a);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_base + 8u * slot);
+      }
+      if (!ok) break;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        Acc3 x{__shfl_xor_sync(0xffffffffu, api.m, o), __shfl_xor_sync(0xffffffffu, api.s, o), __shfl_xor_sync(0xffffffffu, api.a, o)};
+        Acc3 y{__shfl_xor_sync(0xffffffffu, amu.m, o), __shfl_xor_sync(0xffffffffu, amu.s, o), __shfl_xor_sync(0xffffffffu, amu.a, o)};
+        api.merge(x);
+        amu.merge(y);
+      }
+      if (lane == 0) { misc->pi[warp] = api; misc->mu[warp] = amu; mbar_arrive(red_base); }
+      ok = mbar_wait_warp(red_base, nrow & 1u, abort_flag);
+      if (!ok) break;
+      // every warp merges the warps' partials for itself (the same fp32 rule, the same order: identical results)
+      Acc3 xp{-INFINITY, 0.f, 0.f}, xq{-INFINITY, 0.f, 0.f};
+      if (lane < kXWarps) { xp = misc->pi[lane]; xq = misc->mu[lane]; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        Acc3 x{__shfl_xor_sync(0xffffffffu, xp.m, o), __shfl_xor_sync(0xffffffffu, xp.s, o), __shfl_xor_sync(0xffffffffu, xp.a, o)};
+        Acc3 y{__shfl_xor_sync(0xffffffffu, xq.m, o), __shfl_xor_sync(0xffffffffu, xq.s, o), __shfl_xor_sync(0xffffffffu, xq.a, o)};
+        xp.merge(x);
+        xq.merge(y);
+      }
+      const double lse_p = (double)xp.m + log((double)xp.s), lse_q = (double)xq.m + log((double)xq.s);
+      const bool finite = isfinite(lse_p) && isfinite(lse_q);
+      if (tid == 0) {
+        if (finite) {
+          p.entropy[t] = (float)(lse_p - (double)xp.a / (double)xp.s);
+          p.kl[t] = (float)((double)xq.a / (double)xq.s - lse_q + lse_p);
+        } else {
+          p.entropy[t] = 0.f; p.kl[t] = 0.f;
+          atomicOr(p.status, DPPO_STATUS_NONFINITE_ROW);
+        }
+      }
+      // ---- sweep 2 (a non-finite row still drains its chunks: the producer does not know)
+      const float cp = -(float)lse_p * kLog2e, cq = -(float)lse_q * kLog2e;
+      float acc = 0.f;
+      for (int c = 0; c < C && ok; ++c, ++it) {
+        const uint32_t slot = it % kXSlots, use = it / kXSlots;
+        ok = mbar_wait_warp(full_base + 8u * slot, use & 1u, abort_flag);
+        if (!ok) break;
+        const uint32_t off = (uint32_t)c * kXChunk;
+        const uint32_t nvec = ((row_bytes - off) < (uint32_t)kXChunk ? (row_bytes - off) : (uint32_t)kXChunk) / 16u;
+        const uint32_t sa = slots_base + slot * (2u * kXChunk), sb = sa + kXChunk;
+        if (finite) {
+          uint4 va[kXVec], vb[kXVec];
+#pragma unroll
+          for (int k = 0; k < kXVec; ++k) {
+            const uint32_t v = (uint32_t)k * kXConsumers + (uint32_t)tid;
+            if (v < nvec) { va[k] = lds128(sa + v * 16u); vb[k] = lds128(sb + v * 16u); }
+          }
+#pragma unroll
+          for (int k = 0; k < kXVec; ++k) {
+            if ((uint32_t)k * kXConsumers + (uint32_t)tid < nvec) {
+              float a[N], b[N];
+              XVecOf<InT>::unpack(va[k], a);
+              XVecOf<InT>::unpack(vb[k], b);
+              float part = 0.f;
+#pragma unroll
+              for (int i = 0; i < N; ++i) part += fabsf(ex2_approx(fmaf(b[i], kLog2e, cq)) - ex2_approx(fmaf(a[i], kLog2e, cp)));
+              acc += part;
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_base + 8u * slot);
+      }
+      if (!ok) break;
+      const double d = warp_sum((double)acc);
+      if (lane == 0) { misc->tv[warp] = d; mbar_arrive(red_base + 8u); }
+      ok = mbar_wait_warp(red_base + 8u, nrow & 1u, abort_flag);
+      if (!ok) break;
+      if (tid == 0) {
+        double tot = 0;
+        for (int w = 0; w < kXWarps; ++w) tot += misc->tv[w];
+        p.tv[t] = finite ? (float)(0.5 * tot) : 0.f;
+      }
+      ++nrow;
+    }
+  }
+  __syncwarp();
+  if (*abort_flag && lane == 0) atomicOr(p.status, DPPO_STATUS_WAIT_LIMIT);
 }
 
 }  // namespace
@@ -175,9 +489,20 @@ extern "C" int dppo_exact_divergence(const void* logits, const void* mu_logits, 
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int64_t want = (int64_t)sms * 4;
+  const int64_t want = (int64_t)sms;                 // one CTA per SM
   const int grid = (int)(T < want ? T : want);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  // aligned rows whose byte length is a multiple of 16 go through the shared-memory ring
+  if (vec_ok && (V * (int64_t)esz) % 16 == 0 && V * (int64_t)esz < ((int64_t)1 << 31)) {
+    const int smem = kXSlots * 2 * kXChunk + kXMiscBytes;
+    cudaError_t e = (dtype == DPPO_BF16)
+        ? cudaFuncSetAttribute(dppo_exact_ring_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+        : cudaFuncSetAttribute(dppo_exact_ring_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return DPPO_ERR_CUDA;
+    if (dtype == DPPO_BF16) dppo_exact_ring_kernel<__nv_bfloat16><<<grid, kXThreads, smem, st>>>(p);
+    else dppo_exact_ring_kernel<float><<<grid, kXThreads, smem, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? DPPO_OK : DPPO_ERR_CUDA;
+  }
   if (dtype == DPPO_BF16) dppo_exact_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(p, vec_ok);
   else dppo_exact_kernel<float><<<grid, kThreads, 0, st>>>(p, vec_ok);
   return cudaGetLastError() == cudaSuccess ? DPPO_OK : DPPO_ERR_CUDA;

@@ -20,6 +20,7 @@
 // Every wait is bounded: a wait that runs out sets a shared abort flag and the status bit
 // DPPO_STATUS_WAIT_LIMIT; from then on every warp skips its remaining work and returns.
 #include "dppo_common.cuh"
+#include "dppo_pipe.cuh"
 
 namespace dppo {
 
@@ -46,60 +47,6 @@ struct RingMisc {
 };
 static_assert(sizeof(RingMisc) <= kMiscBytes, "misc area");
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait: gives up after ~2 s (or when another thread already gave up) and returns false.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 0xff) == 0) {
-      if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > 2000000000ull) { *abort_flag = 1; return false; }
-    }
-  }
-}
-// All lanes of a warp wait; the warp proceeds only if every lane saw the phase complete.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  const bool ok = mbar_wait(bar, parity, abort_flag);
-  return __all_sync(0xffffffffu, ok);
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
-      : "memory");
-}
-
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-  return v;
-}
 __device__ __forceinline__ void stg128_cs(void* p, uint4 v) {
   asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
@@ -459,6 +406,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
   } else {
     // ------------------------------------------------------------------ scalar warp
     const double scale = p.hdr->scale;
+    const bool topk = (p.variant == DPPO_TOPK_TV || p.variant == DPPO_TOPK_KL) && p.K > 0;
     uint32_t vrow = 0;
     int meta = load_meta(p, t0);
     for (int64_t t = t0; t < p.T; t += G) {
@@ -473,6 +421,24 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         const uint32_t b = vrow & 1u;
         const InT* zrow = reinterpret_cast<const InT*>(p.logits) + t * p.ld_in;
         const float z_a = to_f32<InT>(zrow[a]);                       // in flight while we wait for the partials
+        // Top-K variants: this lane's list entries (positions lane, lane + 32, ...) and their logits are fetched now
+        // too, so that the two dependent memory latencies (id, then z[id]) do not sit between the row's sums and
+        // its gradient; positions beyond 32 * kPre are loaded when the scalar stage asks for them
+        constexpr int kPre = 4;
+        float zk_pre[kPre] = {0.f, 0.f, 0.f, 0.f}, pm_pre[kPre] = {0.f, 0.f, 0.f, 0.f};
+        int id_pre[kPre] = {-1, -1, -1, -1};
+        if (topk) {
+          const int32_t* ids = p.topk_ids + t * (int64_t)p.K;
+          const float* ps = p.topk_p + t * (int64_t)p.K;
+#pragma unroll
+          for (int i = 0; i < kPre; ++i) {
+            const int k = lane + 32 * i;
+            if (k < p.K) { id_pre[i] = ids[k]; pm_pre[i] = ps[k]; }
+          }
+#pragma unroll
+          for (int i = 0; i < kPre; ++i)
+            if (id_pre[i] >= 0 && (int64_t)id_pre[i] < p.V) zk_pre[i] = to_f32<InT>(zrow[id_pre[i]]);
+        }
         const bool have = mbar_wait_warp(part_full + 8u * b, (vrow >> 1) & 1u, abort_flag);
         float2 pr = make_float2(-INFINITY, 0.f);
         if (lane < kGroupWarps) pr = misc->part[b][lane];
@@ -493,8 +459,18 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           } else {
             double pi_a;
             int f2 = 0;
-            auto z_at = [&](int id, int) { return id == a ? z_a : to_f32<InT>(zrow[id]); };
-            row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
+            // this lane only ever asks for its own list positions k = lane + 32 i
+            auto pick = [&](const auto* v, int i) { return i == 0 ? v[0] : (i == 1 ? v[1] : (i == 2 ? v[2] : v[3])); };
+            auto z_at = [&](int id, int k) {
+              if (id == a) return z_a;
+              if (k >= 0 && k < 32 * kPre) return pick(zk_pre, k >> 5);
+              return to_f32<InT>(zrow[id]);
+            };
+            auto list_at = [&](int k, int& id, float& pm) {
+              if (k < 32 * kPre) { id = pick(id_pre, k >> 5); pm = pick(pm_pre, k >> 5); }
+              else { id = p.topk_ids[t * (int64_t)p.K + k]; pm = p.topk_p[t * (int64_t)p.K + k]; }
+            };
+            row_scalars_warp(p, t, a, lse, scale, z_at, list_at, D, M, g, r, absdiff, pi_a, f2);
             if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
             else coef = make_coef(g, lse, pi_a);
           }
