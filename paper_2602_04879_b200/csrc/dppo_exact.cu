@@ -8,7 +8,7 @@
 // One CTA of 512 threads per SM: the row pairs in flight (148 x 608 KB at V = 151936 bf16) then fit in L2 for the
 // second read.  With 16-byte aligned rows the sweeps run on whole 8-element vectors, two vectors of each row in flight
 // per thread while a third is computed on, and the per-thread reference of the sums only moves when a vector would
-// otherwise grow past 2^23.
+// otherwise grow past 2^24.
 #include "dppo_common.cuh"
 #include "dppo_pipe.cuh"
 
@@ -16,7 +16,7 @@ namespace dppo {
 namespace {
 
 constexpr int kThreads = 512;
-constexpr float kRefMargin = 16.f;      // a vector may exceed the running reference by this much before it moves
+constexpr float kRefLimit = 1.6e7f;      // a vector's sum of exp(x - reference) may reach this (about 2^24) before the reference moves
 
 struct ExactParams {
   const void* z; const void* zmu;
@@ -40,28 +40,73 @@ struct Acc3 {
       a = fmaf(e, (e > 0.f) ? w : 0.f, a);              // e = 0 (x = -inf): contributes nothing even if w is inf/nan
     }
   }
-  // N values at once against a reference that moves rarely: m stays put while the vector's maximum is within
-  // kRefMargin above it (the sums are relative to m, whatever m is)
+  // N values at once against a reference that moves rarely.  The sums are relative to m, whatever m is: the values are
+  // first added against the current m; only if that overflows the margin (a partial sum above 2^kRefBits, infinite or
+  // NaN) or m is still -inf are they redone against the vector's own maximum.  Weights of entries with e = 0 must not
+  // turn 0 * inf into NaN, so they are clamped to the finite range instead of being tested one by one.
   template <int N>
   __device__ __forceinline__ void addN(const float* x, const float* w) {
+    const float c = -m * kLog2e;                        // m = -inf: c = +inf, every e below is inf or NaN -> redone
+    float ds = 0.f, da = 0.f;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      const float e = ex2_approx(fmaf(x[i], kLog2e, c));
+      ds += e;
+      da = fmaf(e, fminf(fmaxf(w[i], -3.0e38f), 3.0e38f), da);
+    }
+    if (ds <= kRefLimit) { s += ds; a += da; return; }  // the common case; false for inf and NaN
     float vm = x[0];
 #pragma unroll
     for (int i = 1; i < N; ++i) asm("max.NaN.f32 %0, %0, %1;" : "+f"(vm) : "f"(x[i]));
-    if (!(vm <= m + kRefMargin)) {                      // above the margin, the first finite vector, or NaN
+    if (!(vm <= m)) {                                   // a larger maximum, the first finite vector, or NaN
       const float f = ex2_approx((m - vm) * kLog2e);    // m = -inf gives 0
       s *= f; a *= f; m = vm;
     }
     if (m != -INFINITY) {
-      const float c = -m * kLog2e;
+      const float c2 = -m * kLog2e;
 #pragma unroll
       for (int i = 0; i < N; ++i) {
-        const float e = ex2_approx(fmaf(x[i], kLog2e, c));
+        const float e = ex2_approx(fmaf(x[i], kLog2e, c2));
         s += e;
         a = fmaf(e, (e > 0.f) ? w[i] : 0.f, a);
       }
     }
   }
   __device__ __forceinline__ void add8(const float* x, const float* w) { addN<8>(x, w); }
+  // The same on pairs (two fp32 lanes per instruction for the multiply-adds); x and w must be finite or x = +inf / NaN
+  // (callers clamp -inf to a large negative number, which gives e = 0 and finite weights).
+  template <int N>
+  __device__ __forceinline__ void addN2(const float2* x, const float2* w) {
+    const float c = -m * kLog2e;                        // m = -inf: c = +inf, every e below is inf or NaN -> redone
+    const float2 l2 = make_float2(kLog2e, kLog2e), c2 = make_float2(c, c);
+    float2 ds = make_float2(0.f, 0.f), da = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) {
+      const float2 arg = __ffma2_rn(x[i], l2, c2);
+      const float2 e = make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
+      ds = __fadd2_rn(ds, e);
+      da = __ffma2_rn(e, w[i], da);
+    }
+    const float dsum = ds.x + ds.y;
+    if (dsum <= kRefLimit) { s += dsum; a += da.x + da.y; return; }
+    float xs[N], ws[N];
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) { xs[2 * i] = x[i].x; xs[2 * i + 1] = x[i].y; ws[2 * i] = w[i].x; ws[2 * i + 1] = w[i].y; }
+    float vm = xs[0];
+#pragma unroll
+    for (int i = 1; i < N; ++i) asm("max.NaN.f32 %0, %0, %1;" : "+f"(vm) : "f"(xs[i]));
+    if (!(vm <= m)) {
+      const float f = ex2_approx((m - vm) * kLog2e);
+      s *= f; a *= f; m = vm;
+    }
+    const float c3 = -m * kLog2e;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      const float e = ex2_approx(fmaf(xs[i], kLog2e, c3));
+      s += e;
+      a = fmaf(e, ws[i], a);
+    }
+  }
   __device__ __forceinline__ void merge(const Acc3& o) {
     const float mn = fmaxf(m, o.m);
     if (mn == -INFINITY) return;
@@ -71,6 +116,10 @@ struct Acc3 {
     m = mn;
   }
 };
+
+// The weights z' - z are clamped to +-3e38 inside the sums (see addN), so a rollout probability that meets a trainer
+// probability of zero shows up as an astronomically large sum, not as inf: report it as the +inf it stands for.
+__device__ __forceinline__ float kl_out(double kl) { return kl > 1e30 ? INFINITY : (float)kl; }
 
 template <typename InT>
 __device__ __forceinline__ void load8(const InT* p, int64_t j, int64_t V, bool vec, float* out, int& n);
@@ -212,7 +261,7 @@ __global__ void __launch_bounds__(kThreads, 1) dppo_exact_kernel(ExactParams p, 
         s_lse[1] = (float)lse_q;
         if (ok) {
           p.entropy[t] = (float)(lse_p - Ap / Sp);
-          p.kl[t] = (float)(Bq / Sq - lse_q + lse_p);
+          p.kl[t] = kl_out(Bq / Sq - lse_q + lse_p);
         } else {
           p.entropy[t] = 0.f; p.kl[t] = 0.f; p.tv[t] = 0.f;
           atomicOr(p.status, DPPO_STATUS_NONFINITE_ROW);
@@ -292,6 +341,18 @@ template <> struct XVecOf<float> {
     z[0] = __uint_as_float(v.x); z[1] = __uint_as_float(v.y); z[2] = __uint_as_float(v.z); z[3] = __uint_as_float(v.w);
   }
 };
+
+// -inf (probability zero) becomes a large finite negative number: its exponential is still exactly 0 and differences
+// of two clamped values stay finite; +inf and NaN pass through and poison the row's sums, as they must.
+__device__ __forceinline__ float clamp_low(float x) {
+  asm("max.NaN.f32 %0, %0, %1;" : "+f"(x) : "f"(-1.0e38f));
+  return x;
+}
+template <int N>
+__device__ __forceinline__ void to_pairs(const float* z, float2* z2) {
+#pragma unroll
+  for (int i = 0; i < N / 2; ++i) z2[i] = make_float2(clamp_low(z[2 * i]), clamp_low(z[2 * i + 1]));
+}
 
 template <typename InT>
 __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactParams p) {
@@ -376,10 +437,14 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
             float a[N], b[N];
             XVecOf<InT>::unpack(va[k], a);
             XVecOf<InT>::unpack(vb[k], b);
-            api.addN<N>(a, a);
+            float2 a2[N / 2], b2[N / 2];
+            to_pairs<N>(a, a2);
+            to_pairs<N>(b, b2);
+            api.addN2<N>(a2, a2);
+            const float2 neg1 = make_float2(-1.f, -1.f);
 #pragma unroll
-            for (int i = 0; i < N; ++i) a[i] = b[i] - a[i];
-            amu.addN<N>(b, a);
+            for (int i = 0; i < N / 2; ++i) a2[i] = __ffma2_rn(a2[i], neg1, b2[i]);      // z' - z
+            amu.addN2<N>(b2, a2);
           }
         }
         __syncwarp();
@@ -411,7 +476,7 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
       if (tid == 0) {
         if (finite) {
           p.entropy[t] = (float)(lse_p - (double)xp.a / (double)xp.s);
-          p.kl[t] = (float)((double)xq.a / (double)xq.s - lse_q + lse_p);
+          p.kl[t] = kl_out((double)xq.a / (double)xq.s - lse_q + lse_p);
         } else {
           p.entropy[t] = 0.f; p.kl[t] = 0.f;
           atomicOr(p.status, DPPO_STATUS_NONFINITE_ROW);
@@ -440,9 +505,17 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
               float a[N], b[N];
               XVecOf<InT>::unpack(va[k], a);
               XVecOf<InT>::unpack(vb[k], b);
+              const float2 l2 = make_float2(kLog2e, kLog2e), cp2 = make_float2(cp, cp), cq2 = make_float2(cq, cq);
+              const float2 neg1 = make_float2(-1.f, -1.f);
               float part = 0.f;
 #pragma unroll
-              for (int i = 0; i < N; ++i) part += fabsf(ex2_approx(fmaf(b[i], kLog2e, cq)) - ex2_approx(fmaf(a[i], kLog2e, cp)));
+              for (int i = 0; i < N / 2; ++i) {
+                const float2 ea = __ffma2_rn(make_float2(a[2 * i], a[2 * i + 1]), l2, cp2);
+                const float2 eb = __ffma2_rn(make_float2(b[2 * i], b[2 * i + 1]), l2, cq2);
+                const float2 pa = make_float2(ex2_approx(ea.x), ex2_approx(ea.y)), pb = make_float2(ex2_approx(eb.x), ex2_approx(eb.y));
+                const float2 d = __ffma2_rn(pa, neg1, pb);
+                part += fabsf(d.x) + fabsf(d.y);
+              }
               acc += part;
             }
           }
