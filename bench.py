@@ -163,6 +163,11 @@ def bench_other_configs(dppo, wl, dev, steps=20, warmup=3, n_resp=16):
     ms = _time_steps(torch, lambda: dppo.dppo_exact_divergence(b.logits, zmu, status=status), steps, warmup)
     out["exact_divergence"] = entry(ms, T, T, T * BYTES_PER_TOKEN, f"dppo_exact_divergence, T={T}, V=151936, bf16; bytes = both logits tensors read once "
                                     "(the second sweep is served by L2); 4 exp per element pair: the special-function pipe, not HBM, bounds it")
+    # 4 ex2 per element pair on the special-function pipe (16 per clock and SM, 148 SMs, 1965 MHz maximum clock)
+    sfu_peak = 148 * 16 * 1.965
+    sfu = T * 4 * VOCAB / (ms * 1e-3) / 1e9
+    out["exact_divergence"]["roofline"] = {"bound": "alu", "achieved": sfu, "peak": sfu_peak, "unit": "Gex2/s", "frac": sfu / sfu_peak,
+                                           "peak_source": "148 SMs x 16 ex2/clk x 1.965 GHz (maximum SM clock)"}
     assert int(status.item()) == 0
     del b, dl, zmu
     torch.cuda.empty_cache()
@@ -192,14 +197,14 @@ def bench_other_configs(dppo, wl, dev, steps=20, warmup=3, n_resp=16):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one full-size launch of the row kernel, from the ncu
 # capture summarised under profiles/ (row ring kernel, V = 151936), and the hash of the kernel sources it was
 # taken with: once the kernel changes the figure no longer applies and None is reported.
-TRAFFIC_BYTES_PER_LAUNCH = 5521499819 + 4917211648
-TRAFFIC_KERNEL_SHA = "4f41c1ae413adf92"
+TRAFFIC_BYTES_PER_LAUNCH = 5522199637 + 4917825792
+TRAFFIC_KERNEL_SHA = "af7c3a10c875a4f4"
 
 
 def measured_traffic():
     import hashlib
     h = hashlib.sha256()
-    for f in ("dppo_ring.cu", "dppo_common.cuh"):
+    for f in ("dppo_ring.cu", "dppo_common.cuh", "dppo_pipe.cuh"):
         with open(os.path.join(ROOT, "paper_2602_04879_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return TRAFFIC_BYTES_PER_LAUNCH if h.hexdigest()[:16] == TRAFFIC_KERNEL_SHA else None
