@@ -648,6 +648,7 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   gemm::Params g3 = {};
   g3.M = (int)T; g3.N = (int)d; g3.K = (int)V; g3.C = dHidden; g3.ldc = d; g3.status = status;
   g3.m_live = n_grad; g3.row_map = I(L.idx); g3.row_scale = F(L.factor); g3.splits = -1;
+  g3.n_fastest = 1;      // d / 256 tiles along N: the CTAs of a wave then share each 2 V-byte row block of E instead of re-reading it
   DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(E, L.lde, W, V, g3, st));
   // 7. dW[d, V] = (factor * packed hidden)^T[d, n_grad] . E[n_grad, V]
   DPPO_TRY(transpose_bf16(hc, T, d, d, ws + L.ht, L.ldt, st, F(L.factor), n_grad));

@@ -8,7 +8,9 @@
 //               K=16 per instruction); tcgen05.commit releases smem stages and publishes finished accumulators
 //   warps 2-5   epilogue: tcgen05.ld of the accumulator (one row per thread, 32 columns at a time) while the MMA warp
 //               already fills the other 256-column accumulator buffer
-// Tiles are walked M-fastest so that CTAs running at the same time share B strips through L2.
+// Tiles are walked M-fastest so that CTAs running at the same time share B strips through L2 (or N-fastest, on request,
+// to share A strips).  Epilogues: fp32 store with an optional row factor; exponentials against a per-row reference with
+// their row sums; per-tile softmax statistics with an online maximum; finished gradient rows.
 // Every mbarrier wait is bounded; on expiry the CTA raises DPPO_STATUS_WAIT_LIMIT, skips the rest and frees its TMEM.
 //
 // CG = 2 runs the same roles on pairs of CTAs (a cluster of two SMs) with tcgen05.mma.cta_group::2: one work unit is a
@@ -63,6 +65,8 @@ struct Params {
   const int* row_map;    // EPI_STORE_F32: output row of tile row i (null: i); rows >= *m_live are not stored
   const float* row_scale;  // EPI_STORE_F32: tile row i of the product is multiplied by row_scale[i] (null: 1)
   int allow_empty;       // 1: *m_live == 0 means no tile at all (default: one row of tiles is always processed)
+  int n_fastest;         // order of the tiles: 0 = M-fastest (CTAs running together share strips of B through L2),
+                         // 1 = N-fastest (they share strips of A: for few tiles along N and a large A)
   // EPI_STATS: per (row, n-tile) partial (max, sum exp(z - max)); z at the sampled id
   float2* part;          // [M, tiles_n]
   float* z_a;            // [M]
@@ -289,7 +293,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       bool ok = true;
       for (int u = group; u < nunits && ok; u += ngroups) {
         const int tile = u % ntiles, part = u / ntiles;
-        const int m0 = (tile % tiles_m) * C::TILE_M + (int)rank * BM, n0 = (tile / tiles_m) * BN + (int)rank * C::B_COLS;
+        const int tm = p.n_fastest ? tile / tiles_n : tile % tiles_m, tn = p.n_fastest ? tile % tiles_n : tile / tiles_m;
+        const int m0 = tm * C::TILE_M + (int)rank * BM, n0 = tn * BN + (int)rank * C::B_COLS;
         const int kb0 = part * kper, kb1 = (kb0 + kper < kblocks) ? kb0 + kper : kblocks;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!bar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -365,7 +370,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
     uint32_t it = 0;
     for (int u = group; u < nunits; u += ngroups, ++it) {
       const int tile = u % ntiles;
-      const int m0 = (tile % tiles_m) * C::TILE_M + (int)rank * BM, nb = tile / tiles_m, n0 = nb * BN;
+      const int tm = p.n_fastest ? tile / tiles_n : tile % tiles_m, nb = p.n_fastest ? tile % tiles_n : tile / tiles_m;
+      const int m0 = tm * C::TILE_M + (int)rank * BM, n0 = nb * BN;
       const uint32_t b = it & 1u, use = it >> 1;
       const bool ok = __all_sync(0xffffffffu, bar_wait(tfull0 + 8 * b, use & 1u, abort_flag));
       if (!ok) break;
