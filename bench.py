@@ -108,6 +108,17 @@ def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
     torch.cuda.synchronize()
     ms_sparse = e0.elapsed_time(e1) / max(1, steps // 2)
     b.advantages = adv_full
+    # the same step with the Top-K TV divergence (K = 20): adds W^T and T x K gather dot products to the forward
+    ms_topk = None
+    if T == 8192:
+        bk = wl.lm_head_workload(dev, seed=5, T=T, d=d, V=V, K=20)
+        wsk = torch.empty(dppo.dppo_fused_workspace_bytes(T, d, V, 20), dtype=torch.uint8, device=dev)
+        fn = lambda: dppo.dppo_fused_lmhead_fwd_bwd(bk.hidden, bk.lm_head, bk.sampled_ids, bk.mu_logp, bk.advantages, None,
+                                                    dppo.TOPK_TV, DELTA, K=20, mu_topk_ids=bk.mu_topk_ids, mu_topk_p=bk.mu_topk_p,
+                                                    workspace=wsk, dHidden=dH, dW=dW, status=status)
+        ms_topk = _time_steps(torch, fn, max(1, steps // 2), 2)
+        assert int(status.item()) == 0
+        del bk, wsk
     peak, src = measured_tensor_peak()
     useful = 6.0 * T * d * V / (ms * 1e-3) / 1e12          # forward + dHidden + dW; every logits tile is computed once
     return {"workload": ("" if T == 8192 else f"REDUCED to {T} rows (profiling case): ") + "fused_lm_head_binary_tv: hidden [8192,2048] bf16 x W [2048,151936] bf16, delta=0.2",
@@ -116,7 +127,7 @@ def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
                          "traffic": None, "peak_source": "of " + src,
                          "flop_count": "6*T*d*V (forward, dHidden, dW); nothing is recomputed"},
             "gpu_launches_per_step": 15, "loss": float(out["loss"].item()),
-            "ms_per_step_quarter_of_responses_zero_advantage": ms_sparse}
+            "ms_per_step_quarter_of_responses_zero_advantage": ms_sparse, "ms_per_step_topk_tv_k20": ms_topk}
 
 
 def _time_steps(torch, fn, steps, warmup):
