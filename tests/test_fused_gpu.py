@@ -169,7 +169,7 @@ def test_fused_rows_with_a_vanishing_sampled_token_take_the_two_pass_route():
     probability below 2^-60 under the trainer policy (sum of exponentials out of the safe range, or beyond fp32
     altogether) are recomputed by the two-pass kernels; the results must match the oracle like any other row."""
     T, d, V = 300, 128, 1536
-    b = _fused_case(T, d, V, seed=53, resp_len=4, sigma_w=0.35)           # logits ~ N(0, 4^2)
+    b = _fused_case(T, d, V, seed=53, resp_len=4, sigma_w=0.35, K=8)      # logits ~ N(0, 4^2)
     rows = torch.tensor([3, 64, 65, 130, 255, 299], device=DEV)
     hid = b.hidden.clone()
     hid[rows] = hid[rows] * torch.tensor([4, 4, 8, 8, 8, 4], device=DEV, dtype=hid.dtype)[:, None]   # spreads of +-50 / +-100
@@ -194,6 +194,9 @@ def test_fused_rows_with_a_vanishing_sampled_token_take_the_two_pass_route():
         assert g_rows.min() > 1e-2 * np.abs(ora["dlogits"]).max()        # the recomputed rows matter in dW and dHidden
     tok = (torch.arange(T, device=DEV) % 9 != 2).to(torch.uint8)         # row 65 invalid, 299 invalid
     _check_fused(b, dppo.BINARY_TV, 0.2, tok)
+    # the two-pass route with a Top-K divergence (TV: on these extremely peaked rows the "other" mass of pi is ~1e-12,
+    # below what an fp32-accurate normaliser resolves, so the KL form's log of it is not a fair comparison)
+    _check_fused(b, dppo.TOPK_TV, 0.05, tok, K=8)
     # a non-finite hidden row is reported, dropped, and does not leak into dW
     hid = b.hidden.clone()
     hid[10, 5] = float("inf")
@@ -202,6 +205,20 @@ def test_fused_rows_with_a_vanishing_sampled_token_take_the_two_pass_route():
     assert int(o["status"].item()) == dppo.binding.STATUS_NONFINITE_ROW
     assert not o["dHidden"][10].any() and int(o["mask"][10].item()) == 0
     assert torch.isfinite(o["dW"]).all() and torch.isfinite(o["dHidden"]).all()
+
+
+@pytest.mark.parametrize("T,d,V", [(1, 8, 8), (7, 16, 264), (65, 8, 520)])
+def test_fused_tiny_shapes(T, d, V):
+    """Fewer rows than one K block of the dW GEMM, one row, one tile: the padded parts of the staged operands must not leak."""
+    b = _fused_case(T, d, V, seed=59, resp_len=1, sigma_w=0.5)
+    poison = torch.full((dppo.dppo_fused_workspace_bytes(T, d, V),), 0xFF, dtype=torch.uint8, device=DEV)   # NaN patterns
+    out = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.BINARY_TV, 0.2,
+                                         workspace=poison)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    assert torch.isfinite(out["dW"]).all() and torch.isfinite(out["dHidden"]).all()
+    _check_fused(b, dppo.BINARY_TV, 0.2)
+    _check_fused(b, dppo.BINARY_KL, 0.0)
 
 
 def test_fused_rejects_misuse():
