@@ -56,7 +56,10 @@ enum { DPPO_BINARY_TV = 0, DPPO_BINARY_KL = 1, DPPO_TOPK_TV = 2, DPPO_TOPK_KL = 
 enum { DPPO_F32 = 0, DPPO_BF16 = 1 };
 /* opts->dlogits_dtype */
 enum { DPPO_DLOGITS_SAME = 0, DPPO_DLOGITS_F32 = 1 };
-/* opts->kernel */
+/* opts->kernel.  RING: the bulk-copy (TMA) streaming kernel; it takes logits / dlogits whose bases are 16-byte aligned
+ * and whose rows either all start on 16-byte boundaries with V * element size a multiple of 16, or are shifted alike
+ * (same element size, row strides in bytes equal modulo 16: e.g. both contiguous with an odd V).  GENERIC: element-wise
+ * kernel for any layout (several times slower).  AUTO picks RING whenever it can take the layout. */
 enum { DPPO_KERNEL_AUTO = 0, DPPO_KERNEL_GENERIC = 1, DPPO_KERNEL_RING = 2 };
 
 /* Host-visible error codes. */

@@ -118,11 +118,33 @@ __device__ __forceinline__ int load_meta(const RowParams& p, int64_t t) {
   return (a < 0 || (int64_t)a >= p.V) ? -2 : a;
 }
 
+// Where a row lies in the image the ring holds of it.  SH = false: rows start on 16-byte boundaries and their byte
+// length is a multiple of 16, the image is the row.  SH = true ("shifted" rows: row starts that are only element
+// aligned): the image starts at the 16-byte boundary below the row's first element, `head` bytes early, and the bulk
+// copies cover it up to the last boundary inside the row; the few bytes after that are fetched with plain loads.
+struct RowGeom {
+  uint32_t head;      // bytes in front of the row's first element
+  uint32_t xend;      // head + bytes of the row
+  uint32_t xa;        // bytes of the image that bulk copies deliver (xend rounded down to 16)
+  int C;              // chunks
+};
+template <typename InT, bool SH>
+__device__ __forceinline__ RowGeom row_geom(const RowParams& p, int64_t t, uint32_t row_bytes, int C_static) {
+  RowGeom g;
+  if (!SH) { g.head = 0; g.xend = row_bytes; g.xa = row_bytes; g.C = C_static; return g; }
+  const uintptr_t addr = reinterpret_cast<uintptr_t>(p.logits) + (uintptr_t)(t * p.ld_in) * sizeof(InT);
+  g.head = (uint32_t)(addr & 15u);
+  g.xend = g.head + row_bytes;
+  g.xa = g.xend & ~15u;
+  g.C = (int)((g.xend + kChunkBytes - 1) / kChunkBytes);
+  return g;
+}
+
 // One producer lane: copies every chunk of every valid row of this CTA into the ring
 // [first_slot, first_slot + nslots), in order, as slots are released.
-template <typename InT>
-__device__ __forceinline__ void produce_stream(const RowParams& p, uint32_t slots_base, uint32_t full_base, uint32_t empty_base,
-                                               int first_slot, int nslots, uint32_t row_bytes, int C, uint64_t policy,
+template <typename InT, bool SH>
+__device__ __forceinline__ void produce_stream(const RowParams& p, uint32_t slots_base, unsigned char* slots_ptr, uint32_t full_base,
+                                               uint32_t empty_base, int first_slot, int nslots, uint32_t row_bytes, int C, uint64_t policy,
                                                volatile int* abort_flag, volatile unsigned int* follow, unsigned int lead) {
   const char* logits = reinterpret_cast<const char*>(p.logits);
   const int64_t t0 = blockIdx.x, G = gridDim.x;
@@ -133,8 +155,9 @@ __device__ __forceinline__ void produce_stream(const RowParams& p, uint32_t slot
   for (int64_t t = t0; t < p.T; t += G) {
     const int meta_next = load_meta(p, t + G);
     if (meta >= 0) {
-      const char* row = logits + t * p.ld_in * (int64_t)sizeof(InT);
-      for (int c = 0; c < C; ++c) {
+      const RowGeom gm = row_geom<InT, SH>(p, t, row_bytes, C);
+      const char* row = logits + t * p.ld_in * (int64_t)sizeof(InT) - gm.head;      // start of the image
+      for (int c = 0; c < gm.C; ++c) {
         const int slot = first_slot + pos.slot;
         if (follow) {                      // stay at most `lead` chunks ahead of the stream we feed L2 for
           if (issued - *follow >= lead) {
@@ -150,10 +173,27 @@ __device__ __forceinline__ void produce_stream(const RowParams& p, uint32_t slot
         // lap u >= 1 of a slot needs its (u-1)-th release: parity (u-1)&1 = phase^1
         if (!first_lap && !mbar_wait(empty_base + 8u * slot, pos.phase ^ 1u, abort_flag)) return;
         const uint32_t off = (uint32_t)c * kChunkBytes;
-        const uint32_t bytes = (row_bytes - off) < (uint32_t)kChunkBytes ? (row_bytes - off) : (uint32_t)kChunkBytes;
         const uint32_t bar = full_base + 8u * slot;
-        mbar_arrive_expect_tx(bar, bytes);
-        bulk_load(slots_base + (uint32_t)slot * kChunkBytes, row + off, bytes, bar, policy);
+        if (!SH) {
+          const uint32_t bytes = (row_bytes - off) < (uint32_t)kChunkBytes ? (row_bytes - off) : (uint32_t)kChunkBytes;
+          mbar_arrive_expect_tx(bar, bytes);
+          bulk_load(slots_base + (uint32_t)slot * kChunkBytes, row + off, bytes, bar, policy);
+        } else {
+          const uint32_t bytes = off < gm.xa ? ((gm.xa - off) < (uint32_t)kChunkBytes ? (gm.xa - off) : (uint32_t)kChunkBytes) : 0u;
+          // the row's last bytes, past the last 16-byte boundary inside it, belong to this chunk when that boundary
+          // does: plain loads (nothing beyond the row is read), stored before the arrival that publishes the chunk
+          if (gm.xend > gm.xa && gm.xa >= off && gm.xa < off + (uint32_t)kChunkBytes) {
+            const InT* src = reinterpret_cast<const InT*>(row + gm.xa);
+            InT* dst = reinterpret_cast<InT*>(slots_ptr + (size_t)slot * kChunkBytes + (gm.xa - off));
+            for (uint32_t i = 0; i < (gm.xend - gm.xa) / (uint32_t)sizeof(InT); ++i) dst[i] = src[i];
+          }
+          if (bytes) {
+            mbar_arrive_expect_tx(bar, bytes);
+            bulk_load(slots_base + (uint32_t)slot * kChunkBytes, row + off, bytes, bar, policy);
+          } else {
+            mbar_arrive(bar);
+          }
+        }
         if (++pos.slot == nslots) { pos.slot = 0; pos.phase ^= 1u; first_lap = false; }
       }
     }
@@ -161,7 +201,18 @@ __device__ __forceinline__ void produce_stream(const RowParams& p, uint32_t slot
   }
 }
 
-template <typename InT, typename OutT>
+// Element-wise store of the valid part of a vector at the edge of a shifted row: element i of the vector sits at byte
+// xo + i * sizeof(OutT) of the row's image and is written iff that lies in [head, xend).
+template <typename OutT, int N>
+__device__ __forceinline__ void store_edge(OutT* row_image, uint32_t xo, const float* v, uint32_t sign2, uint32_t head, uint32_t xend) {
+#pragma unroll
+  for (int i = 0; i < N; ++i) {
+    const uint32_t pos = xo + (uint32_t)i * (uint32_t)sizeof(OutT);
+    if (pos >= head && pos < xend) row_image[pos / (uint32_t)sizeof(OutT)] = from_f32<OutT>(sign2 ? -v[i] : v[i]);
+  }
+}
+
+template <typename InT, typename OutT, bool SH>
 __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParams p, int nslots) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int N = Vec<InT>::N;
@@ -196,7 +247,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
   __syncthreads();
 
   const uint32_t row_bytes = (uint32_t)(p.V * (int64_t)sizeof(InT));     // launcher guarantees < 2^31
-  const int C = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);      // chunks per row
+  const int C = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);      // chunks per row (shifted rows: of most rows)
   const int64_t t0 = blockIdx.x, G = gridDim.x;
 
   if (warp >= 2 * kGroupWarps + 1) {
@@ -210,11 +261,11 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         // occupy about #SMs x lead chunks of L2 (61 MB at V = 151936 bf16); a longer lead makes the second
         // read miss L2, a shorter one leaves the sum warps idle.  Measured optimum on B200: C + 7.
         const int lead = (C + 7 <= 26 || C + 2 > 26) ? ((C + 7 <= 26) ? C + 7 : C + 2) : 26;
-        produce_stream<InT>(p, slots_base, full_base, empty_base, 0, ns_sum, row_bytes, C, policy, abort_flag,
-                            &misc->grad_chunks, (unsigned int)lead);
+        produce_stream<InT, SH>(p, slots_base, smem, full_base, empty_base, 0, ns_sum, row_bytes, C, policy, abort_flag,
+                                &misc->grad_chunks, (unsigned int)lead);
       } else {
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-        produce_stream<InT>(p, slots_base, full_base, empty_base, ns_sum, ns_grad, row_bytes, C, policy, abort_flag, nullptr, 0u);
+        produce_stream<InT, SH>(p, slots_base, smem, full_base, empty_base, ns_sum, ns_grad, row_bytes, C, policy, abort_flag, nullptr, 0u);
       }
     }
   } else if (warp < kGroupWarps) {
@@ -230,12 +281,15 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         // per-thread partial: s = sum exp(z - ref); ref is the maximum of the thread's first entries
         // and moves up only when a chunk's sum shows that an entry exceeds it by > 44
         float ref = -INFINITY, nm = 0.f, s = 0.f;
-        for (int c = 0; c < C; ++c) {
+        const RowGeom gm = row_geom<InT, SH>(p, t, row_bytes, C);
+        for (int c = 0; c < gm.C; ++c) {
           const bool ok = mbar_wait_warp(full_base + 8u * pos.slot, pos.phase, abort_flag);
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
           const uint32_t sbase = slots_base + (uint32_t)pos.slot * kChunkBytes;
           if (ok) {
-            const bool full_chunk = cbase + (uint32_t)kChunkBytes <= row_bytes;
+            // whole chunks of whole vectors take the straight-line path (a shifted row's first chunk starts with a
+            // partial vector)
+            const bool full_chunk = cbase + (uint32_t)kChunkBytes <= gm.xa && !(SH && c == 0 && gm.head != 0);
             bool done = false;
             if (full_chunk) {
               // straight-line path: all loads first, then 4 x N independent exponentials
@@ -276,10 +330,17 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
 #pragma unroll 1
               for (int k = 0; k < kVecPerThread; ++k) {
                 const uint32_t off = ((uint32_t)k * kGroupThreads + gtid) * 16u;
-                if (cbase + off < row_bytes) {
+                if (cbase + off < gm.xend) {
                   const uint4 v = lds128(sbase + off);
                   float z[N];
                   Vec<InT>::unpack(v, z);
+                  if (SH) {                         // entries of the image outside the row count as probability zero
+#pragma unroll
+                    for (int i = 0; i < N; ++i) {
+                      const uint32_t pos_b = cbase + off + (uint32_t)i * (uint32_t)sizeof(InT);
+                      if (pos_b < gm.head || pos_b >= gm.xend) z[i] = -INFINITY;
+                    }
+                  }
                   float vm = z[0];
 #pragma unroll
                   for (int i = 1; i < N; ++i) vm = fmaxf(vm, z[i]);
@@ -332,9 +393,21 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
       const int meta_next = load_meta(p, t + G);
       if (__shfl_sync(0xffffffffu, *abort_flag, 0)) break;
       OutT* drow = dlogits + t * p.ld_out;
+      const RowGeom gm = row_geom<InT, SH>(p, t, row_bytes, C);
+      // shifted rows: the output row is shifted by the same number of bytes (same element size, same misalignment, the
+      // launcher checks), so whole vectors of the image are whole, aligned vectors of the output
+      if (SH) drow = reinterpret_cast<OutT*>(reinterpret_cast<char*>(drow) - gm.head);
+      const uint32_t head_e = gm.head / (uint32_t)sizeof(InT);         // elements of the image in front of the row
       if (meta < 0) {
         const float zero[N] = {};
-        for (uint32_t j0 = gtid * N; j0 < (uint32_t)p.V; j0 += kGroupThreads * N) Store<OutT, N>::run(drow, j0, zero);
+        if (!SH) {
+          for (uint32_t j0 = gtid * N; j0 < (uint32_t)p.V; j0 += kGroupThreads * N) Store<OutT, N>::run(drow, j0, zero);
+        } else {
+          for (uint32_t xo = gtid * 16u; xo < gm.xend; xo += kGroupThreads * 16u) {
+            if (xo >= gm.head && xo + 16u <= gm.xend) Store<OutT, N>::run(drow, xo / (uint32_t)sizeof(InT), zero);
+            else store_edge<OutT, N>(drow, xo, zero, 0u, gm.head, gm.xend);
+          }
+        }
       } else {
         const uint32_t b = vrow & 1u;
         const bool have = mbar_wait_warp(coef_full + 8u * b, (vrow >> 1) & 1u, abort_flag);
@@ -343,14 +416,14 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         if (lane == 0 && have) mbar_arrive(coef_empty + 8u * b);
         if (!have) coef.zero_row = 1;
         const uint32_t sign2 = (coef.sgn < 0.f) ? 0x80008000u : 0u;
-        const uint32_t a = (uint32_t)meta;
-        for (int c = 0; c < C; ++c) {
+        const uint32_t a = (uint32_t)meta + head_e;                    // the sampled token's place in the image
+        for (int c = 0; c < gm.C; ++c) {
           const int slot = ns_sum + pos.slot;
           const bool ok = mbar_wait_warp(full_base + 8u * slot, pos.phase, abort_flag);
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
           const uint32_t sbase = slots_base + (uint32_t)slot * kChunkBytes;
           if (ok) {
-            const bool full_chunk = cbase + (uint32_t)kChunkBytes <= row_bytes;
+            const bool full_chunk = cbase + (uint32_t)kChunkBytes <= gm.xa && !(SH && c == 0 && gm.head != 0);
             const uint32_t e0 = cbase / (uint32_t)sizeof(InT);                       // first element of the chunk
             const bool has_a = (a - e0) < (uint32_t)(kChunkBytes / sizeof(InT));     // warp-uniform
             if (full_chunk && !coef.zero_row && !has_a) {
@@ -370,7 +443,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
 #pragma unroll 1
               for (int k = 0; k < kVecPerThread; ++k) {
                 const uint32_t off = ((uint32_t)k * kGroupThreads + gtid) * 16u;
-                if (cbase + off < row_bytes) {
+                if (cbase + off < gm.xend) {
                   const uint32_t j0 = (cbase + off) / (uint32_t)sizeof(InT);
                   float v[N];
                   if (coef.zero_row) {
@@ -388,7 +461,8 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
                         if (j0 + i == a) v[i] = coef.fix * coef.sgn;   // the store flips it back
                     }
                   }
-                  Store<OutT, N>::run(drow, j0, v, sign2);
+                  if (!SH || (cbase + off >= gm.head && cbase + off + 16u <= gm.xend)) Store<OutT, N>::run(drow, j0, v, sign2);
+                  else store_edge<OutT, N>(drow, cbase + off, v, sign2, gm.head, gm.xend);
                 }
               }
             }
@@ -513,16 +587,22 @@ static int ring_slots(int dev) {
   return n > kMaxSlots ? kMaxSlots : n;
 }
 
-bool ring_layout_ok(const RowParams& p, int in_dtype, int out_dtype) {
+// 1: rows start on 16-byte boundaries and are whole 16-byte vectors long; 2: "shifted" rows (16-byte aligned tensors of
+// equal element size whose rows start at the same offset from a 16-byte boundary in logits and dlogits, e.g. contiguous
+// tensors with a vocabulary that is not a multiple of 8); 0: neither, the generic kernel takes the call.
+static int ring_mode(const RowParams& p, int in_dtype, int out_dtype) {
   const int64_t in_sz = (in_dtype == DPPO_BF16) ? 2 : 4, out_sz = (out_dtype == DPPO_BF16) ? 2 : 4;
-  if (in_dtype == DPPO_F32 && out_dtype != DPPO_F32) return false;
-  if ((p.V * in_sz) % 16 != 0 || p.V * in_sz >= ((int64_t)1 << 31)) return false;
-  if (((uintptr_t)p.logits) % 16 != 0 || (p.ld_in * in_sz) % 16 != 0) return false;
-  if (((uintptr_t)p.dlogits) % 16 != 0 || (p.ld_out * out_sz) % 16 != 0) return false;
-  return true;
+  if (in_dtype == DPPO_F32 && out_dtype != DPPO_F32) return 0;
+  if (p.V * in_sz + 16 >= ((int64_t)1 << 31)) return 0;
+  if (((uintptr_t)p.logits) % 16 != 0 || ((uintptr_t)p.dlogits) % 16 != 0) return 0;
+  if ((p.V * in_sz) % 16 == 0 && (p.ld_in * in_sz) % 16 == 0 && (p.ld_out * out_sz) % 16 == 0) return 1;
+  if (in_sz == out_sz && (p.ld_in * in_sz) % 16 == (p.ld_out * out_sz) % 16) return 2;
+  return 0;
 }
 
-template <typename InT, typename OutT>
+bool ring_layout_ok(const RowParams& p, int in_dtype, int out_dtype) { return ring_mode(p, in_dtype, out_dtype) != 0; }
+
+template <typename InT, typename OutT, bool SH>
 static cudaError_t launch_ring_t(const RowParams& p, cudaStream_t st) {
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
@@ -530,18 +610,25 @@ static cudaError_t launch_ring_t(const RowParams& p, cudaStream_t st) {
   const int nslots = ring_slots(dev);
   if (nslots < 2) return cudaErrorInvalidConfiguration;
   const size_t smem = (size_t)nslots * kChunkBytes + kMiscBytes;
-  cudaError_t e = cudaFuncSetAttribute(dppo_row_ring_kernel<InT, OutT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(dppo_row_ring_kernel<InT, OutT, SH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int grid = (int)(p.T < sms ? p.T : sms);
-  dppo_row_ring_kernel<InT, OutT><<<grid, kRingThreads, smem, st>>>(p, nslots);
+  dppo_row_ring_kernel<InT, OutT, SH><<<grid, kRingThreads, smem, st>>>(p, nslots);
   return cudaGetLastError();
 }
 
 cudaError_t launch_ring(const RowParams& p, int in_dtype, int out_dtype, cudaStream_t st) {
   if (p.T == 0) return cudaSuccess;
-  if (in_dtype == DPPO_F32 && out_dtype == DPPO_F32) return launch_ring_t<float, float>(p, st);
-  if (in_dtype == DPPO_BF16 && out_dtype == DPPO_BF16) return launch_ring_t<__nv_bfloat16, __nv_bfloat16>(p, st);
-  if (in_dtype == DPPO_BF16 && out_dtype == DPPO_F32) return launch_ring_t<__nv_bfloat16, float>(p, st);
+  const int mode = ring_mode(p, in_dtype, out_dtype);
+  if (mode == 2) {
+    if (in_dtype == DPPO_F32 && out_dtype == DPPO_F32) return launch_ring_t<float, float, true>(p, st);
+    if (in_dtype == DPPO_BF16 && out_dtype == DPPO_BF16) return launch_ring_t<__nv_bfloat16, __nv_bfloat16, true>(p, st);
+    return cudaErrorInvalidValue;
+  }
+  if (mode != 1) return cudaErrorInvalidValue;
+  if (in_dtype == DPPO_F32 && out_dtype == DPPO_F32) return launch_ring_t<float, float, false>(p, st);
+  if (in_dtype == DPPO_BF16 && out_dtype == DPPO_BF16) return launch_ring_t<__nv_bfloat16, __nv_bfloat16, false>(p, st);
+  if (in_dtype == DPPO_BF16 && out_dtype == DPPO_F32) return launch_ring_t<__nv_bfloat16, float, false>(p, st);
   return cudaErrorInvalidValue;
 }
 

@@ -98,7 +98,7 @@ def test_misuse_is_rejected_before_launch(binding):
     assert _call(B, dl=0x10000, opts=B.DppoOpts(0.0, B.DLOGITS_F32, 0, 0.0, 0.0)) == -9
     assert _call(B, dl=0x10000, ld_out=128) == -9
     # forcing the bulk-copy kernel on a layout it cannot take
-    assert _call(B, V=63, ld=63, ld_out=63, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0.0, 0.0)) == -7
+    assert _call(B, V=63, ld=63, ld_out=64, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0.0, 0.0)) == -7     # rows shifted differently
     assert _call(B, logits=0x10002, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0.0, 0.0)) == -7
 
 

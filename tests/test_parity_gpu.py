@@ -187,20 +187,53 @@ def test_small_vocab_topk_full(kernel, V, dtype):
         assert torch.allclose(o_top0["divergence"], o_bin["divergence"], atol=1e-6)
 
 
-def test_odd_vocab_falls_back_to_scalar_kernel():
+def test_odd_vocab_and_strided_rows():
     T, V = 19, 1001
     logits, a, mu_logp, ids, ps = wl.logits_rows(0, T, V, torch.bfloat16, 12, DEV, sigma=2.0, zipf=1.1, sigma_mu=0.5, K=7)
     adv = torch.linspace(-1, 1, T, device=DEV)
     b = wl.Batch(logits, a, mu_logp, adv, None, ids, ps)
-    _full_check(b, dppo.TOPK_KL, 7, 0.01, dppo.KERNEL_AUTO)
+    # contiguous rows of an odd length: row starts are only element aligned; the bulk-copy kernel takes them as
+    # "shifted" rows when logits and dlogits are shifted alike, the scalar kernel takes everything
+    for kernel in (dppo.KERNEL_AUTO, dppo.KERNEL_RING, dppo.KERNEL_GENERIC):
+        _full_check(b, dppo.TOPK_KL, 7, 0.01, kernel)
+    # fp32 gradient of bf16 logits of odd length: the two tensors cannot be shifted alike
     with pytest.raises(dppo.DppoError) as e:
-        _run(b, dppo.TOPK_KL, 7, 0.01, dppo.KERNEL_RING)
+        _run(b, dppo.TOPK_KL, 7, 0.01, dppo.KERNEL_RING, dlogits_f32=True)
     assert "alignment" in str(e.value)
+    _full_check(b, dppo.TOPK_KL, 7, 0.01, dppo.KERNEL_AUTO, dlogits_f32=True)
     # strided rows (a view into a wider buffer)
     wide = torch.zeros((T, V + 23), dtype=torch.bfloat16, device=DEV)
     wide[:, :V] = logits
     b2 = wl.Batch(wide[:, :V], a, mu_logp, adv, None, ids, ps)
     _full_check(b2, dppo.TOPK_TV, 7, 0.01, dppo.KERNEL_AUTO)
+
+
+@pytest.mark.parametrize("T,V,dtype", [(333, 20011, torch.bfloat16), (200, 5003, torch.float32), (40, 8193, torch.bfloat16),
+                                       (7, 3, torch.float32), (150, 16385, torch.bfloat16)])
+def test_shifted_rows_through_the_bulk_copy_kernel(T, V, dtype):
+    """Vocabularies that are not a multiple of 8 (bf16) / 4 (fp32) elements, contiguous: every row starts at another offset
+    from a 16-byte boundary.  Several chunks per row, several rows per CTA, invalid rows (zero fill), Top-K, in place."""
+    K = min(5, V)
+    logits, a, mu_logp, ids, ps = wl.logits_rows(0, T, V, dtype, 21, DEV, sigma=2.0, zipf=1.1, sigma_mu=0.5, K=K)
+    adv = torch.where(torch.arange(T, device=DEV) % 3 == 0, -1.0, 0.7).to(torch.float32)
+    tok = (torch.arange(T, device=DEV) % 7 != 2).to(torch.uint8)
+    b = wl.Batch(logits, a, mu_logp, adv, tok, ids, ps)
+    out, ora, _ = _full_check(b, dppo.BINARY_TV, 0, 0.05, dppo.KERNEL_RING)
+    _full_check(b, dppo.TOPK_TV, K, 0.01, dppo.KERNEL_RING)
+    gen = _run(b, dppo.BINARY_TV, 0, 0.05, dppo.KERNEL_GENERIC)
+    assert torch.equal(gen["mask"], out["mask"])
+    # in place: the gradient overwrites the logits
+    z = logits.clone()
+    bi = wl.Batch(z, a, mu_logp, adv, tok, ids, ps)
+    inpl = _run(bi, dppo.BINARY_TV, 0, 0.05, dppo.KERNEL_RING, dlogits=z)
+    torch.cuda.synchronize()
+    assert torch.equal(inpl["dlogits"], out["dlogits"]) and inpl["dlogits"].data_ptr() == z.data_ptr()
+    # guard bytes around the output stay untouched (edge vectors are written element by element)
+    pad = torch.full((T * V + 64,), 7.0, dtype=dtype, device=DEV)
+    view = pad[32:32 + T * V].view(T, V)          # 32 elements in: 16-byte aligned base for both element sizes
+    _run(b, dppo.BINARY_TV, 0, 0.05, dppo.KERNEL_RING, dlogits=view)
+    torch.cuda.synchronize()
+    assert torch.equal(view, out["dlogits"]) and torch.all(pad[:32] == 7.0) and torch.all(pad[32 + T * V:] == 7.0)
 
 
 def test_empty_and_fully_masked():
