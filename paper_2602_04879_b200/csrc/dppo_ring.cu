@@ -287,9 +287,8 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
           const uint32_t sbase = slots_base + (uint32_t)pos.slot * kChunkBytes;
           if (ok) {
-            // whole chunks of whole vectors take the straight-line path (a shifted row's first chunk starts with a
-            // partial vector)
-            const bool full_chunk = cbase + (uint32_t)kChunkBytes <= gm.xa && !(SH && c == 0 && gm.head != 0);
+            // chunks that the bulk copy filled completely take the straight-line path
+            const bool full_chunk = cbase + (uint32_t)kChunkBytes <= gm.xa;
             bool done = false;
             if (full_chunk) {
               // straight-line path: all loads first, then 4 x N independent exponentials
@@ -299,6 +298,11 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
               float z[kVecPerThread][N];
 #pragma unroll
               for (int k = 0; k < kVecPerThread; ++k) Vec<InT>::unpack(v[k], z[k]);
+              if (SH && c == 0 && gtid == 0) {    // a shifted row's image starts with entries that are not the row's
+#pragma unroll
+                for (int i = 0; i < N; ++i)
+                  if ((uint32_t)i * (uint32_t)sizeof(InT) < gm.head) z[0][i] = -INFINITY;
+              }
               if (ref == -INFINITY) {            // first chunk of the row: reference = maximum of the first entries
                 float vm = z[0][0];
 #pragma unroll
@@ -423,7 +427,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
           const uint32_t sbase = slots_base + (uint32_t)slot * kChunkBytes;
           if (ok) {
-            const bool full_chunk = cbase + (uint32_t)kChunkBytes <= gm.xa && !(SH && c == 0 && gm.head != 0);
+            const bool full_chunk = cbase + (uint32_t)kChunkBytes <= gm.xa;
             const uint32_t e0 = cbase / (uint32_t)sizeof(InT);                       // first element of the chunk
             const bool has_a = (a - e0) < (uint32_t)(kChunkBytes / sizeof(InT));     // warp-uniform
             if (full_chunk && !coef.zero_row && !has_a) {
@@ -437,7 +441,8 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
                 Vec<InT>::unpack(raw[k], z);
 #pragma unroll
                 for (int i = 0; i < N; ++i) v[i] = ex2_approx(fmaf(z[i], kLog2e, coef.c2));
-                Store<OutT, N>::run(drow, e0 + ((uint32_t)k * kGroupThreads + gtid) * N, v, sign2);
+                if (SH && c == 0 && k == 0 && gtid == 0 && gm.head != 0) store_edge<OutT, N>(drow, 0u, v, sign2, gm.head, gm.xend);
+                else Store<OutT, N>::run(drow, e0 + ((uint32_t)k * kGroupThreads + gtid) * N, v, sign2);
               }
             } else {
 #pragma unroll 1
