@@ -392,3 +392,21 @@ def test_full_size_ragged_topk_kl_k64_one_response():
     mx = float(out["dlogits"][:L].abs().max().item())
     P.check_dlogits(out["dlogits"][torch.as_tensor(rows, device=DEV)], ora["dlogits"], out_is_bf16=True, max_abs=mx)
     assert not out["dlogits"][L:].any() and not out["mask"][L:].any() and not out["divergence"][L:].any()
+
+
+def test_host_buffer_entry_with_an_odd_vocabulary():
+    """Host buffers whose rows are only element aligned: the staged chunks are contiguous, so they take the shifted-row path."""
+    T, V = 230, 20011
+    logits, a, mu_logp, ids, ps = wl.logits_rows(0, T, V, torch.bfloat16, 31, DEV, sigma=2.0, zipf=1.1, sigma_mu=0.5, K=0)
+    adv = torch.where(torch.arange(T, device=DEV) % 2 == 0, -1.0, 1.0).to(torch.float32)
+    b = wl.Batch(logits, a, mu_logp, adv, None, None, None)
+    dev = _run(b, dppo.BINARY_KL, 0, 0.01, dppo.KERNEL_AUTO)
+    pin = lambda x: x.cpu().pin_memory()
+    out = dppo.dppo_loss_fwd_bwd_host(pin(logits), pin(a), pin(mu_logp), pin(adv), None, dppo.BINARY_KL, 0, 0.01,
+                                      rows_per_chunk=64, want_dlogits=True, device=DEV)
+    assert out["status"] == 0
+    assert torch.equal(out["divergence"], dev["divergence"].cpu()) and torch.equal(out["mask"], dev["mask"].cpu())
+    a_, b_ = out["dlogits"].float(), dev["dlogits"].cpu().float()
+    assert torch.all((a_ - b_).abs() <= 2.0 ** -7 * b_.abs())
+    assert abs(out["loss"] - float(dev["loss"].item())) <= 1e-4 * abs(out["loss"]) + 1e-12
+
