@@ -134,8 +134,9 @@ def test_fused_topk_variants_match_oracle(variant):
 
 
 def test_fused_backward_skips_rows_without_gradient(cta_group):
-    """Rows with zero advantage, rows blocked by the mask and invalid rows drop out of the backward GEMMs (the kept rows are
-    packed on the device); the outputs must not change: zeros in dHidden for those rows, the same dW."""
+    """Invalid rows drop out of every GEMM and rows with zero advantage out of the backward GEMMs (the kept rows are packed
+    on the device); rows blocked by the mask stay in with a zero factor.  The outputs must not show any of this: zeros in
+    dHidden for all those rows, the same dW."""
     T, d, V = 600, 128, 1536
     b = _fused_case(T, d, V, seed=47, resp_len=8)
     adv = b.advantages.clone()
