@@ -291,3 +291,26 @@ def test_fused_full_size_masked_subset_and_properties():
     scale_w = float(dW.abs().sum(dim=1).max().item())
     assert float(dW.sum(dim=1).abs().max().item()) <= 5e-3 * scale_w
     assert torch.isfinite(out["dHidden"]).all() and torch.isfinite(dW).all()
+
+
+def test_fused_full_size_topk_sampled_rows():
+    """The fused configuration at full size with the Top-K TV divergence (K = 20): sampled rows against the oracle."""
+    T, d, V, K = 8192, 2048, 151936, 20
+    b = wl.lm_head_workload(DEV, seed=5, K=K)
+    out = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.TOPK_TV, 0.2,
+                                         K=K, mu_topk_ids=b.mu_topk_ids, mu_topk_p=b.mu_topk_p)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    g = torch.Generator().manual_seed(10)
+    rows = torch.sort(torch.randperm(T, generator=g)[:16]).values
+    ridx = rows.numpy()
+    W64 = b.lm_head.float().cpu().numpy().astype(np.float64)
+    Hr = b.hidden[rows.to(DEV)].float().cpu().numpy().astype(np.float64)
+    orr = O.dppo_fused_lmhead_fwd_bwd(Hr, W64, b.sampled_ids.cpu().numpy()[ridx], b.mu_logp.cpu().numpy().astype(np.float64)[ridx],
+                                      b.advantages.cpu().numpy().astype(np.float64)[ridx], None, O.TOPK_TV, 0.2, 1.0 / T, K,
+                                      b.mu_topk_ids.cpu().numpy()[ridx], b.mu_topk_p.cpu().numpy().astype(np.float64)[ridx])
+    P.check_scalars(out["divergence"].cpu().numpy()[ridx], out["mask"].cpu().numpy()[ridx], orr, dict(token_mask=None), 0.2)
+    eh = np.abs(out["dHidden"][rows.to(DEV)].cpu().numpy() - orr["dHidden"])
+    assert np.all(eh <= 2.0 ** -8 * (np.abs(orr["dlogits"]) @ np.abs(W64).T) + 1e-7 * np.abs(orr["dHidden"]).max())
+    assert torch.isfinite(out["dW"]).all()
+
