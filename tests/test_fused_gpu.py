@@ -222,6 +222,21 @@ def test_fused_tiny_shapes(T, d, V):
     _check_fused(b, dppo.BINARY_KL, 0.0)
 
 
+def test_fused_is_deterministic(cta_group):
+    """Same inputs, same bits: the only atomics of the path add two partial sums into zeros, which commutes."""
+    b = _fused_case(520, 136, 2056, seed=61, resp_len=8, K=4)
+    tok = (torch.arange(520, device=DEV) % 6 != 1).to(torch.uint8)
+    runs = []
+    for _ in range(3):
+        o = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, tok, dppo.TOPK_KL, 0.001,
+                                           K=4, mu_topk_ids=b.mu_topk_ids, mu_topk_p=b.mu_topk_p)
+        torch.cuda.synchronize()
+        runs.append(o)
+    for o in runs[1:]:
+        for key in ("loss", "divergence", "mask", "dHidden", "dW"):
+            assert torch.equal(o[key], runs[0][key]), key
+
+
 def test_fused_rejects_misuse():
     b = _fused_case(128, 64, 512, seed=42, resp_len=8)
     with pytest.raises(dppo.DppoError) as e:
