@@ -20,6 +20,9 @@ Reinforcement Learning", DPPO):
 * ``dppo_row`` / ``dppo_loss_fwd_bwd``  surrogate and its logits-gradient   (Eq. dppo_obj, Eq. unified_grad; C = inf unless is_cap is given).
 * ``ppo_clip_mask``             ratio-clipping mask of the PPO / GRPO baseline (App. C.1 mask definitions; Eq. ppo-clip).
 * ``minimal_mask``              the ablation mask of Sec. 5.3: negative samples whose probability dropped by >= delta.
+* variant ``GIVEN_D``           Eq. dppo_obj with the per-token divergence handed in by the caller (e.g. the exact
+                                full-vocabulary TV or KL of ``exact_divergence_row``, which the Binary / Top-K forms
+                                approximate, Sec. 4.4): the mask rule and everything after it are unchanged.
 * ``dppo_fused_lmhead_fwd_bwd`` the same applied to logits = H W with the chain rule into H and W.
 
 Readings of points the paper leaves open (each is listed in the design notes):
@@ -38,8 +41,9 @@ from __future__ import annotations
 
 import numpy as np
 
-BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL, PPO_CLIP, MINIMAL_MASK = 0, 1, 2, 3, 4, 5
-VARIANT_NAMES = {BINARY_TV: "binary_tv", BINARY_KL: "binary_kl", TOPK_TV: "topk_tv", TOPK_KL: "topk_kl", PPO_CLIP: "ppo_clip", MINIMAL_MASK: "minimal_mask"}
+BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL, PPO_CLIP, MINIMAL_MASK, GIVEN_D = 0, 1, 2, 3, 4, 5, 6
+VARIANT_NAMES = {BINARY_TV: "binary_tv", BINARY_KL: "binary_kl", TOPK_TV: "topk_tv", TOPK_KL: "topk_kl", PPO_CLIP: "ppo_clip", MINIMAL_MASK: "minimal_mask",
+                 GIVEN_D: "given_d"}
 
 
 def _f64(x):
@@ -193,7 +197,7 @@ def divergence(variant, pi, a, mu_logp, topk_ids=None, topk_p=None):
 
 
 def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=None, want_grad=True,
-             is_cap=None, eps_low=None):
+             is_cap=None, eps_low=None, given_D=None):
     """All per-token quantities of one valid row.
 
     Returns a dict: lse, log_pi_a, r, D, M, loss (= -s*M*w*A), g (= s*M*w*A) with the weight
@@ -202,7 +206,8 @@ def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=No
     loss term with M and the truncated weight held constant (d log pi(a)/dz_j = 1[j=a] - pi_j).
     variant PPO_CLIP: D = |r - 1| and the mask is ppo_clip_mask with eps_high = delta and eps_low
     (default: delta), the baseline the paper compares against.  variant MINIMAL_MASK: D = mu(a) - pi(a)
-    (signed) and the mask of Sec. 5.3.
+    (signed) and the mask of Sec. 5.3.  variant GIVEN_D: D = given_D (the caller's divergence of this token), mask
+    of Eq. dppo_obj.
     """
     log_pi, lse = log_softmax_row(z)
     pi = np.exp(log_pi)
@@ -216,6 +221,9 @@ def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=No
         mu_a = float(np.exp(float(mu_logp)))
         D = mu_a - float(pi[a])                      # signed drop of the sampled token's probability
         M = minimal_mask(adv, mu_a, pi[a], delta)
+    elif variant == GIVEN_D:
+        D = float(given_D)
+        M = dppo_mask(adv, log_pi_a, mu_logp, D, delta)
     else:
         D = divergence(variant, pi, a, mu_logp, topk_ids, topk_p)
         M = dppo_mask(adv, log_pi_a, mu_logp, D, delta)
@@ -237,11 +245,11 @@ def default_scale(T, token_mask):
 
 def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV,
                       K=0, delta=0.2, loss_scale=None, mu_topk_ids=None, mu_topk_p=None, want_grad=True,
-                      is_cap=None, eps_low=None):
+                      is_cap=None, eps_low=None, given_D=None):
     """The whole path over T rows (Eq. dppo_obj summed over tokens, as a loss to minimise).
 
     logits [T,V]; sampled_ids, mu_logp, advantages [T]; token_mask [T] or None;
-    mu_topk_ids / mu_topk_p [T,K] for the Top-K variants.  loss_scale None means
+    mu_topk_ids / mu_topk_p [T,K] for the Top-K variants; given_D [T] for GIVEN_D.  loss_scale None means
     1/N_valid.  Rows with token_mask == 0 contribute nothing: D = 0, M = 0, zero
     gradient row.  Returns dict(loss, D[T], M[T], r[T], row_loss[T], dlogits[T,V] or None).
     """
@@ -260,7 +268,7 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
         if variant in (TOPK_TV, TOPK_KL) and K > 0:
             ids, ps = mu_topk_ids[t][:K], mu_topk_p[t][:K]
         o = dppo_row(logits[t], sampled_ids[t], mu_logp[t], advantages[t], variant, delta, s, ids, ps, want_grad,
-                     is_cap, eps_low)
+                     is_cap, eps_low, None if given_D is None else given_D[t])
         D[t], M[t], r[t], row_loss[t] = o["D"], o["M"], o["r"], o["loss"]
         if want_grad:
             dl[t] = o["dlogits"]
@@ -269,7 +277,7 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
 
 def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None,
                               variant=BINARY_TV, delta=0.2, loss_scale=None, K=0, mu_topk_ids=None, mu_topk_p=None,
-                              is_cap=None, eps_low=None):
+                              is_cap=None, eps_low=None, given_D=None):
     """LM-head variant: logits = hidden @ W in float64 (never rounded), then the path above,
     then the chain rule: dHidden = dlogits @ W^T, dW = hidden^T @ dlogits.
     """
@@ -277,7 +285,7 @@ def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token
     Wm = _f64(W)
     z = H @ Wm
     o = dppo_loss_fwd_bwd(z, sampled_ids, mu_logp, advantages, token_mask, variant, K, delta, loss_scale,
-                          mu_topk_ids, mu_topk_p, True, is_cap, eps_low)
+                          mu_topk_ids, mu_topk_p, True, is_cap, eps_low, given_D)
     o["dHidden"] = o["dlogits"] @ Wm.T
     o["dW"] = H.T @ o["dlogits"]
     return o

@@ -483,7 +483,45 @@ def check_exact_divergence(O):
     assert np.isfinite(tv) and np.isfinite(ent) and np.isfinite(kl)
 
 
-CHECKS = [check_exact_divergence, check_minimal_mask, check_is_cap_and_baselines, check_ppo_clip_variant, check_worked_example, check_log_softmax, check_binary, check_topk_full_and_bounds,
+def check_given_divergence(O):
+    """Variant GIVEN_D: Eq. dppo_obj with the caller's per-token divergence.  Feeding the Binary-TV values back reproduces
+    the Binary-TV variant; with the exact full-vocabulary TV (App. B: D_bin <= D_full) every token the Binary form blocks
+    stays blocked; D = 0 never blocks, D = +inf blocks exactly the tokens that moved away from r = 1."""
+    rng = np.random.default_rng(77)
+    c = _case(rng, T=40, V=13, K=3, noise=0.9)
+    z, a, ml, adv = c["z"], c["a"], c["mu_logp"], c["adv"]
+    T = len(a)
+    zm = np.log(c["mu"])
+    delta = 0.08
+    ref = O.dppo_loss_fwd_bwd(z, a, ml, adv, None, O.BINARY_TV, 0, delta)
+    same = O.dppo_loss_fwd_bwd(z, a, ml, adv, None, O.GIVEN_D, 0, delta, given_D=ref["D"])
+    assert np.array_equal(same["M"], ref["M"]) and same["loss"] == ref["loss"] and np.array_equal(same["dlogits"], ref["dlogits"])
+    assert np.array_equal(same["D"], ref["D"])
+    full = np.array([O.exact_divergence_row(z[t], zm[t])[0] for t in range(T)])
+    assert np.all(full >= ref["D"] - 1e-15)
+    ex = O.dppo_loss_fwd_bwd(z, a, ml, adv, None, O.GIVEN_D, 0, delta, given_D=full)
+    lp = scipy.special.log_softmax(z, axis=1)[np.arange(T), a]
+    away = ((adv > 0) & (lp > ml)) | ((adv < 0) & (lp < ml))
+    assert np.array_equal(ex["M"], np.where(away & (full > delta), 0, 1).astype(np.uint8))
+    assert np.all(ex["M"] <= ref["M"]) and 0 < int((ex["M"] == 0).sum()) < T and int((ex["M"] != ref["M"]).sum()) > 0
+    assert np.array_equal(ex["D"], full)
+    tok = (np.arange(T) % 4 != 1).astype(np.uint8)
+    zero = O.dppo_loss_fwd_bwd(z, a, ml, adv, tok, O.GIVEN_D, 0, delta, given_D=np.zeros(T))
+    r = np.exp(lp - ml)
+    assert np.array_equal(zero["M"], tok) and abs(zero["loss"] + np.sum((r * adv)[tok != 0]) / tok.sum()) < 1e-12
+    inf = O.dppo_loss_fwd_bwd(z, a, ml, adv, tok, O.GIVEN_D, 0, delta, given_D=np.full(T, np.inf))
+    assert np.array_equal(inf["M"], np.where(away | (tok == 0), 0, 1).astype(np.uint8))
+    assert not inf["dlogits"][inf["M"] == 0].any()
+    # the LM-head form passes it through
+    H = rng.standard_normal((T, 5))
+    W = rng.standard_normal((5, 13))
+    zz = H @ W
+    f1 = O.dppo_fused_lmhead_fwd_bwd(H, W, a, ml, adv, None, O.GIVEN_D, delta, given_D=full)
+    f2 = O.dppo_loss_fwd_bwd(zz, a, ml, adv, None, O.GIVEN_D, 0, delta, given_D=full)
+    assert np.array_equal(f1["M"], f2["M"]) and np.allclose(f1["dW"], H.T @ f2["dlogits"])
+
+
+CHECKS = [check_given_divergence, check_exact_divergence, check_minimal_mask, check_is_cap_and_baselines, check_ppo_clip_variant, check_worked_example, check_log_softmax, check_binary, check_topk_full_and_bounds,
           check_topk_other_bucket, check_topk_equality_conditions, check_edge_conventions,
           check_mask_truth_table, check_on_policy, check_gradient, check_brute_force_tiny, check_fused]
 
@@ -569,8 +607,9 @@ def _fused_transposed(m):
 def _cap_as_max(m):
     orig = m.dppo_row
 
-    def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=None, want_grad=True, is_cap=None, eps_low=None):
-        o = orig(z, a, mu_logp, adv, variant, delta, scale, topk_ids, topk_p, want_grad, None, eps_low)
+    def dppo_row(z, a, mu_logp, adv, variant, delta, scale, topk_ids=None, topk_p=None, want_grad=True, is_cap=None, eps_low=None,
+                 given_D=None):
+        o = orig(z, a, mu_logp, adv, variant, delta, scale, topk_ids, topk_p, want_grad, None, eps_low, given_D)
         if is_cap is not None and np.isfinite(is_cap):
             f = max(o["r"], is_cap) / o["r"]
             o["g"] *= f
@@ -581,11 +620,27 @@ def _cap_as_max(m):
     return dppo_row
 
 
-MUTANTS.update({"minimal_mask_positive_side": lambda m: (lambda adv, mu, pi, delta: 0 if (adv > 0 and mu - pi >= delta) else 1),
+def _given_d_ignored(m):
+    orig = m.dppo_row
+
+    def dppo_row(z, a, mu_logp, adv, variant, *rest, **k):       # uses the Binary-TV value instead of the caller's
+        if variant == m.GIVEN_D:
+            rest = list(rest)
+            if "given_D" in k:
+                k["given_D"] = None
+            elif len(rest) >= 8:
+                rest[7] = None
+            o = orig(z, a, mu_logp, adv, m.BINARY_TV, *rest, **k)
+            return o
+        return orig(z, a, mu_logp, adv, variant, *rest, **k)
+    return dppo_row
+
+
+MUTANTS.update({"given_d_ignored": _given_d_ignored, "minimal_mask_positive_side": lambda m: (lambda adv, mu, pi, delta: 0 if (adv > 0 and mu - pi >= delta) else 1),
                 "cap_as_max": _cap_as_max, "ppo_eps_swapped": lambda m: (lambda adv, r, el, eh: 0 if ((adv > 0 and r - 1 > el) or (adv < 0 and 1 - r > eh)) else 1),
                 "topk_no_dedupe": _no_dedupe, "grad_sign": _grad_sign, "grad_no_onehot": _grad_no_onehot,
                 "fused_scaled": _fused_transposed})
-MUTANT_TARGET.update({"minimal_mask_positive_side": "minimal_mask", "cap_as_max": "dppo_row", "ppo_eps_swapped": "ppo_clip_mask", "topk_no_dedupe": "topk_reduced", "grad_sign": "dppo_row", "grad_no_onehot": "dppo_row",
+MUTANT_TARGET.update({"given_d_ignored": "dppo_row", "minimal_mask_positive_side": "minimal_mask", "cap_as_max": "dppo_row", "ppo_eps_swapped": "ppo_clip_mask", "topk_no_dedupe": "topk_reduced", "grad_sign": "dppo_row", "grad_no_onehot": "dppo_row",
                       "fused_scaled": "dppo_fused_lmhead_fwd_bwd"})
 
 
