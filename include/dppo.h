@@ -51,7 +51,11 @@ enum { DPPO_BINARY_TV = 0, DPPO_BINARY_KL = 1, DPPO_TOPK_TV = 2, DPPO_TOPK_KL = 
           M_t = 0 iff (A > 0 and r - 1 > delta) or (A < 0 and 1 - r > eps_low); delta plays eps_high */
        DPPO_PPO_CLIP = 4,
        /* ablation of Sec. 5.3: D_t = mu(a_t) - pi(a_t) (signed), M_t = 0 iff A_t < 0 and D_t >= delta */
-       DPPO_MINIMAL_MASK = 5 };
+       DPPO_MINIMAL_MASK = 5,
+       /* Eq. dppo_obj with a per-token divergence computed elsewhere, e.g. the exact full-vocabulary TV or KL that the
+          forms of Sec. 4.4 approximate (dppo_exact_divergence): the caller fills `divergence` with D_t before the call;
+          mask, loss and gradient follow as for the other variants.  Device entry points only. */
+       DPPO_GIVEN_D = 6 };
 /* Element types of the logits / dlogits tensors. */
 enum { DPPO_F32 = 0, DPPO_BF16 = 1 };
 /* opts->dlogits_dtype */
@@ -125,7 +129,8 @@ size_t dppo_workspace_bytes(int64_t T);
  *  opts            NULL = defaults.
  *  loss            [1]  out: -s * sum_t M_t r_t A_t.
  *  divergence      [T]  out: D_t (0 for invalid rows; +inf possible for KL when pi puts zero mass
- *                  where mu does not).
+ *                  where mu does not).  With DPPO_GIVEN_D it is also an input: D_t of every row on entry; on
+ *                  return the values of valid rows are unchanged, rows that were dropped read 0.
  *  mask            [T]  out: M_t as bytes (0 for invalid rows).
  *  dlogits         [T, V] out, row stride `dlogits_row_stride` (>= V), dtype per opts; may be the
  *                  same buffer as logits (in place) when the element sizes match and the strides

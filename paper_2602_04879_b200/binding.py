@@ -13,12 +13,12 @@ from ctypes import POINTER, c_char_p, c_float, c_int, c_int32, c_int64, c_size_t
 
 import torch
 
-BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL, PPO_CLIP, MINIMAL_MASK = 0, 1, 2, 3, 4, 5
+BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL, PPO_CLIP, MINIMAL_MASK, GIVEN_D = 0, 1, 2, 3, 4, 5, 6
 F32, BF16 = 0, 1
 DLOGITS_SAME, DLOGITS_F32 = 0, 1
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_RING = 0, 1, 2
 STATUS_BAD_SAMPLED_ID, STATUS_BAD_TOPK_ID, STATUS_NONFINITE_ROW, STATUS_WAIT_LIMIT = 1, 2, 4, 8
-VARIANTS = {"binary_tv": BINARY_TV, "binary_kl": BINARY_KL, "topk_tv": TOPK_TV, "topk_kl": TOPK_KL, "ppo_clip": PPO_CLIP, "minimal_mask": MINIMAL_MASK}
+VARIANTS = {"binary_tv": BINARY_TV, "binary_kl": BINARY_KL, "topk_tv": TOPK_TV, "topk_kl": TOPK_KL, "ppo_clip": PPO_CLIP, "minimal_mask": MINIMAL_MASK, "given_d": GIVEN_D}
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdppo.so")
 _lib = None
@@ -105,12 +105,22 @@ def dppo_workspace_bytes(T):
     return int(lib().dppo_workspace_bytes(int(T)))
 
 
+def _divergence_buffer(T, dev, variant, given):
+    """The call's divergence buffer: an output, and for GIVEN_D also the input (a copy of the caller's values)."""
+    if int(variant) == GIVEN_D:
+        assert given is not None and given.is_cuda and given.dtype == torch.float32 and given.shape == (T,), "given_divergence"
+        return given.contiguous().clone()
+    return torch.empty(T, dtype=torch.float32, device=dev)
+
+
 def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, K=0, delta=0.2,
                       mu_topk_ids=None, mu_topk_p=None, loss_scale=0.0, dlogits_f32=False, kernel=KERNEL_AUTO,
-                      dlogits=None, want_stats=False, workspace=None, status=None, stream=None, is_cap=0.0, eps_low=0.0):
+                      dlogits=None, want_stats=False, workspace=None, status=None, stream=None, is_cap=0.0, eps_low=0.0,
+                      given_divergence=None):
     """Calls ``dppo_loss_fwd_bwd`` on CUDA tensors.  Output tensors are allocated with torch unless
     given.  Returns dict(loss[1], divergence[T], mask[T], dlogits[T,V], stats[8] or None, status[1]);
-    nothing is synchronised."""
+    nothing is synchronised.  ``given_divergence`` [T] fp32: the per-token divergence for variant GIVEN_D (copied into
+    the in/out divergence buffer of the call)."""
     assert logits.is_cuda and logits.dim() == 2 and logits.stride(1) == 1
     T, V = logits.shape
     dev = logits.device
@@ -119,7 +129,7 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
         dlogits = torch.empty((T, V), dtype=out_dtype, device=dev)
     assert dlogits.dtype == out_dtype and dlogits.stride(1) == 1
     loss = torch.empty(1, dtype=torch.float32, device=dev)
-    D = torch.empty(T, dtype=torch.float32, device=dev)
+    D = _divergence_buffer(T, dev, variant, given_divergence)
     M = torch.empty(T, dtype=torch.uint8, device=dev)
     stats = torch.empty(8, dtype=torch.float32, device=dev) if want_stats else None
     if status is None:
@@ -152,16 +162,17 @@ def dppo_fused_workspace_bytes(T, d, V, K=0):
 
 def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, delta=0.2,
                               loss_scale=0.0, want_stats=False, workspace=None, dHidden=None, dW=None, status=None, stream=None,
-                              is_cap=0.0, eps_low=0.0, K=0, mu_topk_ids=None, mu_topk_p=None):
+                              is_cap=0.0, eps_low=0.0, K=0, mu_topk_ids=None, mu_topk_p=None, given_divergence=None):
     """Calls ``dppo_fused_lmhead_fwd_bwd`` on CUDA tensors: hidden [T,d] bf16, W [d,V] bf16.  Returns
-    dict(loss[1], divergence[T], mask[T], dHidden[T,d] fp32, dW[d,V] fp32, stats, status); nothing is synchronised."""
+    dict(loss[1], divergence[T], mask[T], dHidden[T,d] fp32, dW[d,V] fp32, stats, status); nothing is synchronised.
+    ``given_divergence``: as for ``dppo_loss_fwd_bwd`` (variant GIVEN_D)."""
     assert hidden.is_cuda and W.is_cuda and hidden.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
     assert hidden.is_contiguous() and W.is_contiguous() and hidden.shape[1] == W.shape[0]
     T, d = hidden.shape
     V = W.shape[1]
     dev = hidden.device
     loss = torch.empty(1, dtype=torch.float32, device=dev)
-    D = torch.empty(T, dtype=torch.float32, device=dev)
+    D = _divergence_buffer(T, dev, variant, given_divergence)
     M = torch.empty(T, dtype=torch.uint8, device=dev)
     if dHidden is None:
         dHidden = torch.empty((T, d), dtype=torch.float32, device=dev)

@@ -54,7 +54,7 @@ int dppo_loss_fwd_bwd(const void* logits, int64_t T, int64_t V, int64_t logits_r
   if (T < 0 || V < 1 || K < 0 || (int64_t)K > V) return DPPO_ERR_SHAPE;
   if (logits_dtype != DPPO_F32 && logits_dtype != DPPO_BF16) return DPPO_ERR_DTYPE;
   if (o.dlogits_dtype != DPPO_DLOGITS_SAME && o.dlogits_dtype != DPPO_DLOGITS_F32) return DPPO_ERR_DTYPE;
-  if (variant < DPPO_BINARY_TV || variant > DPPO_MINIMAL_MASK) return DPPO_ERR_VARIANT;
+  if (variant < DPPO_BINARY_TV || variant > DPPO_GIVEN_D) return DPPO_ERR_VARIANT;
   if (o.kernel < DPPO_KERNEL_AUTO || o.kernel > DPPO_KERNEL_RING) return DPPO_ERR_UNSUPPORTED;
   if (!loss || !status) return DPPO_ERR_NULL;
   if (T > 0 && (!logits || !sampled_ids || !mu_logp || !advantages || !divergence || !mask || !dlogits)) return DPPO_ERR_NULL;

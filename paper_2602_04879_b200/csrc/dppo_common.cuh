@@ -117,6 +117,8 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
   } else if (p.variant == DPPO_MINIMAL_MASK) {        // ablation of Sec. 5.3: signed drop of the sampled token's probability
     D = mu_a - pi_a;
     ppo_blocked = (adv < 0.0 && D >= (double)p.delta);
+  } else if (p.variant == DPPO_GIVEN_D) {             // the caller's divergence of this token (read before it is written back)
+    D = (double)p.divergence[t];
   } else if (p.variant == DPPO_BINARY_TV) {
     D = fabs(mu_a - pi_a);                            // Eq. binary_tv
   } else if (p.variant == DPPO_BINARY_KL) {           // Eq. binary_kl

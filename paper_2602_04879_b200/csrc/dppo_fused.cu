@@ -538,7 +538,7 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   dppo_opts o = {};
   if (opts) o = *opts;
   if (T < 0 || d < 1 || V < 1 || T > (int64_t)1 << 30 || V > (int64_t)1 << 30 || d > (int64_t)1 << 30) return DPPO_ERR_SHAPE;
-  if (variant < DPPO_BINARY_TV || variant > DPPO_MINIMAL_MASK) return DPPO_ERR_VARIANT;
+  if (variant < DPPO_BINARY_TV || variant > DPPO_GIVEN_D) return DPPO_ERR_VARIANT;
   const bool topk = (variant == DPPO_TOPK_TV || variant == DPPO_TOPK_KL);
   if (!topk) K = 0;
   if (K < 0 || (int64_t)K > V) return DPPO_ERR_SHAPE;

@@ -45,9 +45,9 @@ def host_inputs(batch, rows=None):
     )
 
 
-def run_oracle(h, variant, K, delta, scale, want_grad=True, is_cap=None, eps_low=None):
+def run_oracle(h, variant, K, delta, scale, want_grad=True, is_cap=None, eps_low=None, given_D=None):
     return O.dppo_loss_fwd_bwd(h["logits"], h["sampled_ids"], h["mu_logp"], h["advantages"], h["token_mask"],
-                               variant, K, delta, scale, h["mu_topk_ids"], h["mu_topk_p"], want_grad, is_cap, eps_low)
+                               variant, K, delta, scale, h["mu_topk_ids"], h["mu_topk_p"], want_grad, is_cap, eps_low, given_D)
 
 
 def bf16_round(x):

@@ -80,7 +80,7 @@ def test_misuse_is_rejected_before_launch(binding):
     assert _call(B, K=-1) == -2
     assert _call(B, dt=7) == -3
     assert _call(B, opts=B.DppoOpts(0.0, 5, 0, 0.0, 0.0)) == -3
-    assert _call(B, variant=6) == -4
+    assert _call(B, variant=7) == -4
     assert _call(B, variant=-1) == -4
     assert _call(B, opts=B.DppoOpts(0.0, 0, 9, 0.0, 0.0)) == -11
     assert _call(B, logits=None) == -1

@@ -69,3 +69,39 @@ def test_exact_divergence_edge_cases():
     wide = torch.zeros((8, 600), device=DEV)
     wide[:, :512] = z
     _check(wide[:, :512], zm)
+
+
+@pytest.mark.parametrize("kernel", ["ring", "generic"])
+@pytest.mark.parametrize("which,delta", [("tv", 0.1), ("kl", 0.03)])
+def test_exact_divergence_as_the_trust_region(which, delta, kernel):
+    """Variant GIVEN_D fed with the monitor's exact TV / KL: Eq. dppo_obj with the quantity the Sec. 4.4 forms
+    approximate.  Against the oracle given the oracle's own exact values; the blocked set contains the Binary form's."""
+    import parity_util as P
+    from paper_2602_04879_b200 import workloads as wl
+    T, V = 300, 4104
+    z, zm = _pair(T, V, torch.bfloat16, seed=5, noise=0.6)
+    g = torch.Generator(device=DEV).manual_seed(9)
+    a = torch.multinomial(torch.softmax(zm.float(), 1), 1, generator=g)[:, 0].to(torch.int32)
+    mu_logp = torch.log_softmax(zm.float(), 1).gather(1, a.long()[:, None])[:, 0].contiguous()
+    adv = torch.where(torch.arange(T, device=DEV) % 2 == 0, 1.0, -0.5).to(torch.float32)
+    tok = (torch.arange(T, device=DEV) % 6 != 4).to(torch.uint8)
+    ex = dppo.dppo_exact_divergence(z, zm, tok)
+    code = dppo.KERNEL_RING if kernel == "ring" else dppo.KERNEL_GENERIC
+    out = dppo.dppo_loss_fwd_bwd(z, a, mu_logp, adv, tok, dppo.GIVEN_D, 0, delta, kernel=code, given_divergence=ex[which],
+                                 dlogits_f32=True)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    b = wl.Batch(z, a, mu_logp, adv, tok, None, None)
+    h = P.host_inputs(b)
+    zh, zmh = h["logits"], zm.float().cpu().numpy().astype(np.float64)
+    full = np.array([O.exact_divergence_row(zh[t], zmh[t])[0 if which == "tv" else 1] if h["token_mask"][t] else 0.0 for t in range(T)])
+    ora = P.run_oracle(h, O.GIVEN_D, 0, delta, None, given_D=full)
+    P.check_scalars(out["divergence"].cpu().numpy(), out["mask"].cpu().numpy(), ora, h, delta)
+    P.check_loss(float(out["loss"].item()), ora["loss"], True, ora["row_loss"])
+    P.check_dlogits(out["dlogits"], ora["dlogits"], out_is_bf16=False)
+    valid = h["token_mask"] != 0
+    blocked = int(((ora["M"] == 0) & valid).sum())
+    assert 0 < blocked < int(valid.sum())
+    binary = dppo.dppo_loss_fwd_bwd(z, a, mu_logp, adv, tok, dppo.BINARY_TV if which == "tv" else dppo.BINARY_KL, 0, delta, kernel=code)
+    assert torch.all(out["mask"] <= binary["mask"])          # App. B: D_bin <= D_full, so the exact region blocks a superset
+

@@ -222,6 +222,30 @@ def test_fused_tiny_shapes(T, d, V):
     _check_fused(b, dppo.BINARY_KL, 0.0)
 
 
+def test_fused_with_a_given_divergence():
+    """Variant GIVEN_D through the LM-head path: the caller's per-token divergence decides the mask."""
+    T, d, V = 260, 128, 1032
+    b = _fused_case(T, d, V, seed=67, resp_len=4, sigma_w=0.3)
+    g = torch.Generator(device=DEV).manual_seed(3)
+    Dg = torch.rand(T, generator=g, device=DEV) * 0.2
+    tok = (torch.arange(T, device=DEV) % 5 != 3).to(torch.uint8)
+    out = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, tok, dppo.GIVEN_D, 0.1,
+                                         given_divergence=Dg)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    H = b.hidden.float().cpu().numpy().astype(np.float64)
+    W = b.lm_head.float().cpu().numpy().astype(np.float64)
+    tokh = tok.cpu().numpy()
+    ora = O.dppo_fused_lmhead_fwd_bwd(H, W, b.sampled_ids.cpu().numpy(), b.mu_logp.cpu().numpy().astype(np.float64),
+                                      b.advantages.cpu().numpy().astype(np.float64), tokh, O.GIVEN_D, 0.1,
+                                      given_D=Dg.cpu().numpy().astype(np.float64))
+    P.check_scalars(out["divergence"].cpu().numpy(), out["mask"].cpu().numpy(), ora, dict(token_mask=tokh), 0.1)
+    P.check_loss(float(out["loss"].item()), ora["loss"], True, ora["row_loss"])
+    assert 0 < int(((ora["M"] == 0) & (tokh != 0)).sum()) < int((tokh != 0).sum())
+    ew = np.abs(out["dW"].cpu().numpy() - ora["dW"])
+    assert np.all(ew <= DW_ROUNDING * (np.abs(H).T @ np.abs(ora["dlogits"])) + 1e-7 * np.abs(ora["dW"]).max())
+
+
 def test_fused_is_deterministic(cta_group):
     """Same inputs, same bits: the only atomics of the path add two partial sums into zeros, which commutes."""
     b = _fused_case(520, 136, 2056, seed=61, resp_len=8, K=4)
