@@ -174,6 +174,14 @@ def bench_other_configs(dppo, wl, dev, steps=20, warmup=3, n_resp=16):
     ms = _time_steps(torch, lambda: dppo.dppo_exact_divergence(b.logits, zmu, status=status), steps, warmup)
     out["exact_divergence"] = entry(ms, T, T, T * BYTES_PER_TOKEN, f"dppo_exact_divergence, T={T}, V=151936, bf16; bytes = both logits tensors read once "
                                     "(the second sweep is served by L2); 4 exp per element pair: the special-function pipe, not HBM, bounds it")
+    # DPPO with the exact TV as its trust region: the monitor, then the loss kernel on the divergence it produced
+    def exact_then_loss():
+        ex = dppo.dppo_exact_divergence(b.logits, zmu, status=status)
+        return dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.GIVEN_D, 0, 0.2,
+                                      dlogits=dl, workspace=ws, status=status, given_divergence=ex["tv"])
+    ms2 = _time_steps(torch, exact_then_loss, steps, warmup)
+    out["exact_tv_trust_region"] = entry(ms2, T, T, T * (BYTES_PER_TOKEN + 2 * VOCAB),
+                                         f"dppo_exact_divergence + dppo_loss_fwd_bwd(GIVEN_D), T={T}; bytes = both logits tensors read once + dlogits written")
     # 4 ex2 per element pair on the special-function pipe (16 per clock and SM, 148 SMs, 1965 MHz maximum clock)
     sfu_peak = 148 * 16 * 1.965
     sfu = T * 4 * VOCAB / (ms * 1e-3) / 1e9
