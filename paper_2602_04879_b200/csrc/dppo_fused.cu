@@ -215,7 +215,8 @@ __global__ void __launch_bounds__(256) fused_ref_logit_kernel(const __nv_bfloat1
 // z_topk[t, k] = hidden[t, :] . W^T[ids[t, k], :]: the logits at the rollout policy's top-K ids, one warp per (t, k).
 // W^T rows are contiguous, so each dot product reads two 2d-byte rows with 16-byte loads (d is a multiple of 8).
 __global__ void __launch_bounds__(256) fused_topk_logits_kernel(const __nv_bfloat16* hidden, const __nv_bfloat16* wt, int64_t T,
-                                                                int64_t d, int64_t V, const int32_t* ids, int K, float* z_topk) {
+                                                                int64_t d, int64_t V, const int32_t* ids, int K, float* z_topk,
+                                                                float out_scale) {
   const int lane = threadIdx.x & 31;
   const int64_t w = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (w >= T * K) return;
@@ -237,7 +238,8 @@ __global__ void __launch_bounds__(256) fused_topk_logits_kernel(const __nv_bfloa
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-  if (lane == 0) z_topk[w] = acc;       // out-of-range ids give 0 here and raise the status bit in the scalar stage
+  // out-of-range ids give 0 here and raise the status bit in the scalar stage (non-finite sums too, when used as reference)
+  if (lane == 0) z_topk[w] = (out_scale == 1.f || isfinite(acc)) ? acc * out_scale : 0.f;
 }
 
 // Stable two-class partition of the rows (one block): idx = the rows of class 0 in order, then those of class 1;
@@ -593,7 +595,11 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
     DPPO_TRY(cudaGetLastError());
   }
   // 2. reference exponent of every packed row
-  fused_ref_logit_kernel<<<row_warps, 256, 0, st>>>(hc, Wb, T, d, V, I(L.ids_c), n_valid, F(L.cref2));
+  if (K > 0)      // W^T is there: contiguous rows instead of strided columns (rows past the valid ones are zero: reference 0)
+    fused_topk_logits_kernel<<<row_warps, 256, 0, st>>>(hc, reinterpret_cast<const __nv_bfloat16*>(ws + L.wt), T, d, V, I(L.ids_c), 1,
+                                                        F(L.cref2), kLog2e);
+  else
+    fused_ref_logit_kernel<<<row_warps, 256, 0, st>>>(hc, Wb, T, d, V, I(L.ids_c), n_valid, F(L.cref2));
   DPPO_TRY(cudaGetLastError());
   // 3. forward GEMM: exponentials, their sums, z at the sampled id
   DPPO_TRY(cudaMemsetAsync(F(L.z_a), 0, (size_t)T * 4, st));
@@ -606,7 +612,7 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   if (K > 0) {      // logits at the rollout policy's top-K ids: T x K dot products against rows of W^T
     z_topk = F(L.z_topk);
     fused_topk_logits_kernel<<<(unsigned)((T * K + 7) / 8), 256, 0, st>>>(
-        hid, reinterpret_cast<const __nv_bfloat16*>(ws + L.wt), T, d, V, mu_topk_ids, K, z_topk);
+        hid, reinterpret_cast<const __nv_bfloat16*>(ws + L.wt), T, d, V, mu_topk_ids, K, z_topk, 1.f);
     DPPO_TRY(cudaGetLastError());
   }
   {
