@@ -155,6 +155,30 @@ def bench_other_configs(dppo, wl, dev, steps=20, warmup=3, n_resp=16):
         return {"ms_per_step": ms, "rows_per_s": rows / (ms * 1e-3), "valid_tokens_per_s": valid / (ms * 1e-3),
                 "achieved_gbs": gbs, "frac_of_hbm_peak": gbs / peak, "peak_source": "of " + src, "note": note}
 
+    # the tiny configuration (T = 256, V = 4096, fp32): latency of one call, L2 flushed between the timed calls
+    tb = wl.tiny_binary_tv(dev, seed=0)
+    tdl = torch.empty_like(tb.logits)
+    tws = torch.empty(dppo.dppo_workspace_bytes(tb.T), dtype=torch.uint8, device=dev)
+    tst = torch.zeros(1, dtype=torch.int32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    tiny = lambda: dppo.dppo_loss_fwd_bwd(tb.logits, tb.sampled_ids, tb.mu_logp, tb.advantages, None, dppo.BINARY_TV, 0, 0.2,
+                                          dlogits=tdl, workspace=tws, status=tst)
+    for _ in range(3):
+        tiny()
+    us = []
+    for _ in range(20):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        tiny()
+        e1.record()
+        torch.cuda.synchronize()
+        us.append(1e3 * e0.elapsed_time(e1))
+    us.sort()
+    out["tiny_binary_tv_fp32"] = {"us_per_call_median": us[len(us) // 2], "us_per_call_best": us[0], "calls": len(us),
+                                  "note": "T=256, V=4096, fp32, all valid, delta=0.2: three launches per call, 8.4 MB moved; "
+                                          "latency-bound; a 256 MB buffer is written between the timed calls (L2 flush)"}
+    del flush, tb, tdl, tws
     # Binary-KL and Top-K TV (K = 20) on the Qwen3-vocabulary rows
     b = wl.qwen_vocab_rows(dev, seed=1, K=20, n_resp=n_resp, group=min(16, n_resp))     # n_resp != 16: reduced profiling case
     T = b.T
@@ -387,9 +411,12 @@ def run_ours(args):
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler.start()
     t_host0 = time.perf_counter()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     ev0.record()
-    for _ in range(args.steps):
+    marks[0].record()
+    for i in range(args.steps):
         out = step()
+        marks[i + 1].record()
     ev1.record()
     barrier()
     t_host1 = time.perf_counter()
@@ -404,6 +431,7 @@ def run_ours(args):
         loss_val = float(out["loss"].item())
     assert int(status.item()) == 0, f"device status {int(status.item())}"
     ms_per_step = ms / args.steps
+    per_step = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))       # this rank's steps, one by one
     tokens_per_s = world * T * args.steps / (ms * 1e-3)
 
     # roofline of the row kernel: algorithmic bytes of one launch over the step's device time (the step is
@@ -424,6 +452,7 @@ def run_ours(args):
                    "variant": args.variant, "rows_per_gpu": T, "l2": "inputs_larger_than_L2 (4.98 GB read + 4.98 GB written per step)",
                    "parallelism": f"dp{world} row shards, no data-path collective", "logits_dtype": "bf16", "dlogits_dtype": "bf16"},
         "roofline": roofline, "clocks": clocks, "gpu_launches": 3 * args.steps, "loss": loss_val,
+        "ms_per_step_best": per_step[0], "ms_per_step_median": per_step[len(per_step) // 2],
     }
 
     # end to end through the host-buffer entry point: pinned host inputs -> device -> loss / D / M back on the host
