@@ -175,10 +175,16 @@ def bench_other_configs(dppo, wl, dev, steps=20, warmup=3, n_resp=16):
         torch.cuda.synchronize()
         us.append(1e3 * e0.elapsed_time(e1))
     us.sort()
+    # the same call captured in a CUDA graph and replayed back to back (no L2 flush): what launch overhead leaves
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        tiny()
+    us_replay = 1e3 * _time_steps(torch, graph.replay, 200, 5)
     out["tiny_binary_tv_fp32"] = {"us_per_call_median": us[len(us) // 2], "us_per_call_best": us[0], "calls": len(us),
+                                  "us_per_graph_replay": us_replay,
                                   "note": "T=256, V=4096, fp32, all valid, delta=0.2: three launches per call, 8.4 MB moved; "
                                           "latency-bound; a 256 MB buffer is written between the timed calls (L2 flush)"}
-    del flush, tb, tdl, tws
+    del graph, flush, tb, tdl, tws
     # Binary-KL and Top-K TV (K = 20) on the Qwen3-vocabulary rows
     b = wl.qwen_vocab_rows(dev, seed=1, K=20, n_resp=n_resp, group=min(16, n_resp))     # n_resp != 16: reduced profiling case
     T = b.T
