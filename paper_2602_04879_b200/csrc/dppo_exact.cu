@@ -73,8 +73,7 @@ struct Acc3 {
     }
   }
   __device__ __forceinline__ void add8(const float* x, const float* w) { addN<8>(x, w); }
-  // The same on pairs (two fp32 lanes per instruction for the multiply-adds); x and w must be finite or x = +inf / NaN
-  // (callers clamp -inf to a large negative number, which gives e = 0 and finite weights).
+  // The same on pairs (two fp32 lanes per instruction for the multiply-adds).
   template <int N>
   __device__ __forceinline__ void addN2(const float2* x, const float2* w) {
     const float c = -m * kLog2e;                        // m = -inf: c = +inf, every e below is inf or NaN -> redone
@@ -87,8 +86,10 @@ struct Acc3 {
       ds = __fadd2_rn(ds, e);
       da = __ffma2_rn(e, w[i], da);
     }
-    const float dsum = ds.x + ds.y;
-    if (dsum <= kRefLimit) { s += dsum; a += da.x + da.y; return; }
+    const float dsum = ds.x + ds.y, dasum = da.x + da.y;
+    // the common case; false for inf and NaN in either sum (an entry far above the reference, or a weight that is not
+    // finite: -inf logits give 0 * inf), which the slow path below sorts out entry by entry
+    if (dsum <= kRefLimit && fabsf(dasum) <= 3.0e38f) { s += dsum; a += dasum; return; }
     float xs[N], ws[N];
 #pragma unroll
     for (int i = 0; i < N / 2; ++i) { xs[2 * i] = x[i].x; xs[2 * i + 1] = x[i].y; ws[2 * i] = w[i].x; ws[2 * i + 1] = w[i].y; }
@@ -99,12 +100,13 @@ struct Acc3 {
       const float f = ex2_approx((m - vm) * kLog2e);
       s *= f; a *= f; m = vm;
     }
+    if (m == -INFINITY) return;                        // nothing but -inf so far
     const float c3 = -m * kLog2e;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
       const float e = ex2_approx(fmaf(xs[i], kLog2e, c3));
       s += e;
-      a = fmaf(e, ws[i], a);
+      a = fmaf(e, (e > 0.f) ? ws[i] : 0.f, a);      // e = 0 (a -inf logit) contributes nothing, whatever its weight
     }
   }
   __device__ __forceinline__ void merge(const Acc3& o) {
@@ -342,16 +344,10 @@ template <> struct XVecOf<float> {
   }
 };
 
-// -inf (probability zero) becomes a large finite negative number: its exponential is still exactly 0 and differences
-// of two clamped values stay finite; +inf and NaN pass through and poison the row's sums, as they must.
-__device__ __forceinline__ float clamp_low(float x) {
-  asm("max.NaN.f32 %0, %0, %1;" : "+f"(x) : "f"(-1.0e38f));
-  return x;
-}
 template <int N>
 __device__ __forceinline__ void to_pairs(const float* z, float2* z2) {
 #pragma unroll
-  for (int i = 0; i < N / 2; ++i) z2[i] = make_float2(clamp_low(z[2 * i]), clamp_low(z[2 * i + 1]));
+  for (int i = 0; i < N / 2; ++i) z2[i] = make_float2(z[2 * i], z[2 * i + 1]);
 }
 
 template <typename InT>
