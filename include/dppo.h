@@ -102,7 +102,10 @@ typedef struct dppo_opts {
                           <= 0 or +inf: no truncation (Eq. dppo_obj).  The paper's scaling runs use C = 5,
                           CISPO / PG-TIS is C = 3 with delta = +inf (no mask)                            */
   float eps_low;       /* DPPO_PPO_CLIP only: lower clip range; <= 0: same as delta                      */
+  int lm_head_layout;  /* dppo_fused_lmhead_fwd_bwd only: DPPO_LM_HEAD_DV (0) = W and dW are [d, V] row-major;
+                          DPPO_LM_HEAD_VD (1) = both are [V, d] row-major (how a linear layer stores its weight)  */
 } dppo_opts;
+enum { DPPO_LM_HEAD_DV = 0, DPPO_LM_HEAD_VD = 1 };
 
 /* Bytes of device scratch dppo_loss_fwd_bwd needs for T rows (256-byte aligned
  * pointer expected).  Contents need no initialisation and carry nothing between calls. */
@@ -219,6 +222,8 @@ size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V, int K);
  * [T, V] logits are never written to memory; the gradient is propagated to hidden and W.
  *
  *  hidden   [T, d] bf16 row-major;  W  [d, V] bf16 row-major (LM head);  d and V multiples of 8, 16-byte aligned.
+ *           With opts->lm_head_layout = DPPO_LM_HEAD_VD, W is [V, d] row-major and dW is written as [V, d] too
+ *           (no transposed copy is made: the operands are read, and dW is stored, in that layout directly).
  *  sampled_ids, mu_logp, advantages, token_mask, delta, opts, loss, divergence, mask, stats, status: as for
  *           dppo_loss_fwd_bwd.  mu_topk_ids / mu_topk_p [T, K]: as for dppo_loss_fwd_bwd (Top-K variants; the K
  *           logits per row are computed as dot products, K is ignored by the other variants).

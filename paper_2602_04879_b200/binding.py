@@ -25,7 +25,8 @@ _lib = None
 
 
 class DppoOpts(ctypes.Structure):
-    _fields_ = [("loss_scale", c_float), ("dlogits_dtype", c_int), ("kernel", c_int), ("is_cap", c_float), ("eps_low", c_float)]
+    _fields_ = [("loss_scale", c_float), ("dlogits_dtype", c_int), ("kernel", c_int), ("is_cap", c_float), ("eps_low", c_float),
+                ("lm_head_layout", c_int)]
 
 
 class DppoError(RuntimeError):
@@ -162,14 +163,15 @@ def dppo_fused_workspace_bytes(T, d, V, K=0):
 
 def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, delta=0.2,
                               loss_scale=0.0, want_stats=False, workspace=None, dHidden=None, dW=None, status=None, stream=None,
-                              is_cap=0.0, eps_low=0.0, K=0, mu_topk_ids=None, mu_topk_p=None, given_divergence=None):
+                              is_cap=0.0, eps_low=0.0, K=0, mu_topk_ids=None, mu_topk_p=None, given_divergence=None, w_is_vd=False):
     """Calls ``dppo_fused_lmhead_fwd_bwd`` on CUDA tensors: hidden [T,d] bf16, W [d,V] bf16.  Returns
     dict(loss[1], divergence[T], mask[T], dHidden[T,d] fp32, dW[d,V] fp32, stats, status); nothing is synchronised.
-    ``given_divergence``: as for ``dppo_loss_fwd_bwd`` (variant GIVEN_D)."""
+    ``given_divergence``: as for ``dppo_loss_fwd_bwd`` (variant GIVEN_D).  ``w_is_vd``: W (and dW) are [V,d], the layout
+    of a linear layer's weight, instead of [d,V]."""
     assert hidden.is_cuda and W.is_cuda and hidden.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
-    assert hidden.is_contiguous() and W.is_contiguous() and hidden.shape[1] == W.shape[0]
+    assert hidden.is_contiguous() and W.is_contiguous() and hidden.shape[1] == W.shape[1 if w_is_vd else 0]
     T, d = hidden.shape
-    V = W.shape[1]
+    V = W.shape[0 if w_is_vd else 1]
     dev = hidden.device
     loss = torch.empty(1, dtype=torch.float32, device=dev)
     D = _divergence_buffer(T, dev, variant, given_divergence)
@@ -177,13 +179,13 @@ def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token
     if dHidden is None:
         dHidden = torch.empty((T, d), dtype=torch.float32, device=dev)
     if dW is None:
-        dW = torch.empty((d, V), dtype=torch.float32, device=dev)
+        dW = torch.empty((V, d) if w_is_vd else (d, V), dtype=torch.float32, device=dev)
     stats = torch.empty(8, dtype=torch.float32, device=dev) if want_stats else None
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
     if workspace is None:
         workspace = torch.empty(dppo_fused_workspace_bytes(T, d, V, K), dtype=torch.uint8, device=dev)
-    opts = DppoOpts(float(loss_scale), 0, 0, float(is_cap), float(eps_low))
+    opts = DppoOpts(float(loss_scale), 0, 0, float(is_cap), float(eps_low), 1 if w_is_vd else 0)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     with torch.cuda.device(dev):
         rc = lib().dppo_fused_lmhead_fwd_bwd(_ptr(hidden), _ptr(W), T, d, V, _ptr(sampled_ids), _ptr(mu_logp),

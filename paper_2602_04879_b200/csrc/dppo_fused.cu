@@ -549,6 +549,8 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   if (T > 0 && (!hidden || !sampled_ids || !mu_logp || !advantages || !divergence || !mask || !dHidden)) return DPPO_ERR_NULL;
   if (((uintptr_t)hidden % 16) || ((uintptr_t)W % 16) || (d % 8) || (V % 8)) return DPPO_ERR_ALIGN;
   if (((uintptr_t)dHidden % 16) || ((uintptr_t)dW % 16)) return DPPO_ERR_ALIGN;
+  if (o.lm_head_layout != DPPO_LM_HEAD_DV && o.lm_head_layout != DPPO_LM_HEAD_VD) return DPPO_ERR_UNSUPPORTED;
+  const bool vd = (o.lm_head_layout == DPPO_LM_HEAD_VD);      // W and dW given as [V, d]
   const FusedLayout L = fused_layout(T, d, V, K);
   if (!workspace || ((uintptr_t)workspace % kAlign) || workspace_bytes < L.total) return DPPO_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -584,7 +586,9 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   const int32_t *n_grad = counts, *n_valid = counts + 1, *n_resc = counts + 2;
   const unsigned row_warps = (unsigned)((T + 7) / 8);
   // 1. rows with a gradient to come (valid, advantage not zero) first, then the other valid rows; W^T for the Top-K gather
-  if (K > 0) DPPO_TRY(transpose_bf16(W, d, V, V, ws + L.wt, d, st));
+  // rows of W^T for the gather dot products: W itself when it is stored [V, d]
+  const __nv_bfloat16* wt = vd ? Wb : reinterpret_cast<const __nv_bfloat16*>(ws + L.wt);
+  if (K > 0 && !vd) DPPO_TRY(transpose_bf16(W, d, V, V, ws + L.wt, d, st));
   fused_partition_rows_kernel<<<1, 1024, 0, st>>>(token_mask, advantages, nullptr, T, I(L.idx), I(L.pos), counts);
   DPPO_TRY(cudaGetLastError());
   {
@@ -595,9 +599,8 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
     DPPO_TRY(cudaGetLastError());
   }
   // 2. reference exponent of every packed row
-  if (K > 0)      // W^T is there: contiguous rows instead of strided columns (rows past the valid ones are zero: reference 0)
-    fused_topk_logits_kernel<<<row_warps, 256, 0, st>>>(hc, reinterpret_cast<const __nv_bfloat16*>(ws + L.wt), T, d, V, I(L.ids_c), 1,
-                                                        F(L.cref2), kLog2e);
+  if (K > 0 || vd)      // W^T is there: contiguous rows instead of strided columns (rows past the valid ones are zero: reference 0)
+    fused_topk_logits_kernel<<<row_warps, 256, 0, st>>>(hc, wt, T, d, V, I(L.ids_c), 1, F(L.cref2), kLog2e);
   else
     fused_ref_logit_kernel<<<row_warps, 256, 0, st>>>(hc, Wb, T, d, V, I(L.ids_c), n_valid, F(L.cref2));
   DPPO_TRY(cudaGetLastError());
@@ -606,13 +609,14 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   gemm::Params g1 = {};
   g1.M = (int)T; g1.N = (int)V; g1.K = (int)d; g1.psum = F(L.psum); g1.z_a = F(L.z_a); g1.ids = I(L.ids_c); g1.cref2 = F(L.cref2);
   g1.P = E; g1.ldp = L.lde; g1.status = status; g1.m_live = n_valid; g1.e_live = n_grad;
-  DPPO_TRY((launch_gemm<gemm::EPI_EXP, true>(hc, d, W, V, g1, st)));      // B = W [d, V], MN-major
+  if (vd) DPPO_TRY((launch_gemm<gemm::EPI_EXP, false>(hc, d, W, d, g1, st)));     // B = W [V, d], K-major
+  else DPPO_TRY((launch_gemm<gemm::EPI_EXP, true>(hc, d, W, V, g1, st)));         // B = W [d, V], MN-major
   // 4. per-row scalars
   float* z_topk = nullptr;
   if (K > 0) {      // logits at the rollout policy's top-K ids: T x K dot products against rows of W^T
     z_topk = F(L.z_topk);
     fused_topk_logits_kernel<<<(unsigned)((T * K + 7) / 8), 256, 0, st>>>(
-        hid, reinterpret_cast<const __nv_bfloat16*>(ws + L.wt), T, d, V, mu_topk_ids, K, z_topk, 1.f);
+        hid, wt, T, d, V, mu_topk_ids, K, z_topk, 1.f);
     DPPO_TRY(cudaGetLastError());
   }
   {
@@ -635,7 +639,8 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
     gemm::Params gs = {};
     gs.M = (int)T; gs.N = (int)V; gs.K = (int)d; gs.part = reinterpret_cast<float2*>(ws + L.part); gs.z_a = F(L.z_ar);
     gs.ids = I(L.ids_r); gs.status = status; gs.m_live = n_resc; gs.allow_empty = 1;
-    DPPO_TRY((launch_gemm<gemm::EPI_STATS, true>(ws + L.hr, d, W, V, gs, st)));
+    if (vd) DPPO_TRY((launch_gemm<gemm::EPI_STATS, false>(ws + L.hr, d, W, d, gs, st)));
+    else DPPO_TRY((launch_gemm<gemm::EPI_STATS, true>(ws + L.hr, d, W, V, gs, st)));
     RescueArgs x = {};
     x.rescue = I(L.rescue); x.pos_r = I(L.pos_r); x.pos_e = I(L.pos);
     x.part = reinterpret_cast<const float2*>(ws + L.part); x.tiles_n = L.tiles_n; x.z_a = F(L.z_ar); x.z_topk = z_topk;
@@ -645,7 +650,8 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
     gemm::Params gg = {};
     gg.M = (int)T; gg.N = (int)V; gg.K = (int)d; gg.ids = I(L.ids_r); gg.c2 = F(L.c2); gg.sgn = F(L.sgn); gg.fix = F(L.fix);
     gg.P = E; gg.ldp = L.lde; gg.status = status; gg.m_live = n_resc; gg.allow_empty = 1; gg.p_row_map = I(L.rmap);
-    DPPO_TRY((launch_gemm<gemm::EPI_GRAD, true>(ws + L.hr, d, W, V, gg, st)));
+    if (vd) DPPO_TRY((launch_gemm<gemm::EPI_GRAD, false>(ws + L.hr, d, W, d, gg, st)));
+    else DPPO_TRY((launch_gemm<gemm::EPI_GRAD, true>(ws + L.hr, d, W, V, gg, st)));
   }
   DPPO_TRY(launch_finalize(p, st));
   // 6. dHidden[idx[i], :] = factor[i] * (E[i, :] . W[d, V]^T) for the rows with a gradient; the other rows stay zero.
@@ -655,11 +661,13 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   g3.M = (int)T; g3.N = (int)d; g3.K = (int)V; g3.C = dHidden; g3.ldc = d; g3.status = status;
   g3.m_live = n_grad; g3.row_map = I(L.idx); g3.row_scale = F(L.factor); g3.splits = -1;
   g3.n_fastest = 1;      // d / 256 tiles along N: the CTAs of a wave then share each 2 V-byte row block of E instead of re-reading it
-  DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(E, L.lde, W, V, g3, st));
+  if (vd) DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(E, L.lde, W, d, g3, st)));     // B = W as [K = V, N = d], MN-major
+  else DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(E, L.lde, W, V, g3, st));                // B = W as [N = d, K = V], K-major
   // 7. dW[d, V] = (factor * packed hidden)^T[d, n_grad] . E[n_grad, V]
   DPPO_TRY(transpose_bf16(hc, T, d, d, ws + L.ht, L.ldt, st, F(L.factor), n_grad));
   gemm::Params g4 = {};
   g4.M = (int)d; g4.N = (int)V; g4.K = (int)T; g4.C = dW; g4.ldc = V; g4.status = status; g4.k_live = n_grad;
+  if (vd) { g4.c_transposed = 1; g4.ldc = d; }      // the same product, stored as dW[V, d]
   DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(ws + L.ht, L.ldt, E, L.lde, g4, st)));   // B = E [T, V], MN-major
 #undef DPPO_TRY
   return DPPO_OK;

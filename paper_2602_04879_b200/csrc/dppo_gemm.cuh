@@ -64,6 +64,7 @@ struct Params {
   const int* k_live;
   const int* row_map;    // EPI_STORE_F32: output row of tile row i (null: i); rows >= *m_live are not stored
   const float* row_scale;  // EPI_STORE_F32: tile row i of the product is multiplied by row_scale[i] (null: 1)
+  int c_transposed;      // EPI_STORE_F32 (no K split, no row map): the product is stored transposed, C[col * ldc + row]
   int allow_empty;       // 1: *m_live == 0 means no tile at all (default: one row of tiles is always processed)
   int n_fastest;         // order of the tiles: 0 = M-fastest (CTAs running together share strips of B through L2),
                          // 1 = N-fastest (they share strips of A: for few tiles along N and a large A)
@@ -393,7 +394,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
 #pragma unroll
               for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * sc);
             }
-            if (splits > 1) {              // partial sum over a K part: add into the zeroed output
+            if (p.c_transposed) {          // the lanes of a warp hold 32 consecutive rows: 128 contiguous bytes per column
+              float* ct = p.C + (int64_t)(n0 + c) * p.ldc + row;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) ct[(int64_t)j * p.ldc] = __uint_as_float(r[j]);
+            } else if (splits > 1) {       // partial sum over a K part: add into the zeroed output
 #pragma unroll
               for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) atomicAdd(dst + j, __uint_as_float(r[j]));
             } else if (n0 + c + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {

@@ -222,6 +222,30 @@ def test_fused_tiny_shapes(T, d, V):
     _check_fused(b, dppo.BINARY_KL, 0.0)
 
 
+@pytest.mark.parametrize("T,d,V,K", [(256, 128, 1024, 0), (300, 72, 1000, 6), (520, 136, 2056, 0)])
+def test_fused_with_the_lm_head_stored_vocabulary_major(T, d, V, K, cta_group):
+    """W given as [V, d] (how a linear layer stores its weight) and dW returned in that layout: same results as with [d, V]."""
+    b = _fused_case(T, d, V, seed=71, resp_len=4, K=K, sigma_w=0.3 if K else None)
+    variant = dppo.TOPK_TV if K else dppo.BINARY_TV
+    tok = (torch.arange(T, device=DEV) % 7 != 2).to(torch.uint8)
+    kw = dict(K=K, mu_topk_ids=b.mu_topk_ids, mu_topk_p=b.mu_topk_p)
+    ref, ora = _check_fused(b, variant, 0.01, tok, K=K)
+    out = dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head.t().contiguous(), b.sampled_ids, b.mu_logp, b.advantages, tok, variant, 0.01,
+                                         w_is_vd=True, **kw)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0 and out["dW"].shape == (V, d)
+    assert torch.equal(out["mask"], ref["mask"])
+    assert torch.allclose(out["divergence"], ref["divergence"], atol=2e-6, rtol=0)
+    H = b.hidden.float().cpu().numpy().astype(np.float64)
+    W = b.lm_head.float().cpu().numpy().astype(np.float64)
+    aP = np.abs(ora["dlogits"])
+    eh = np.abs(out["dHidden"].cpu().numpy() - ora["dHidden"])
+    ew = np.abs(out["dW"].cpu().numpy().T - ora["dW"])
+    assert np.all(eh <= 2.0 ** -8 * (aP @ np.abs(W).T) + 1e-7 * np.abs(ora["dHidden"]).max())
+    assert np.all(ew <= DW_ROUNDING * (np.abs(H).T @ aP) + 1e-7 * np.abs(ora["dW"]).max())
+    P.check_loss(float(out["loss"].item()), ora["loss"], True, ora["row_loss"])
+
+
 def test_fused_with_a_given_divergence():
     """Variant GIVEN_D through the LM-head path: the caller's per-token divergence decides the mask."""
     T, d, V = 260, 128, 1032
