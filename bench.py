@@ -70,7 +70,7 @@ def measured_tensor_peak():
     return 1400.0, "fallback (about 1.4 PFLOP/s sustained, earlier measurement on this pool)"
 
 
-def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
+def bench_fused(dppo, wl, dev, steps=40, warmup=10, T=8192):
     """Fused LM-head variant on its own workload: hidden [8192, 2048] x W [2048, 151936], Binary-TV, delta 0.2."""
     import torch
     d, V = 2048, VOCAB
@@ -99,15 +99,15 @@ def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
     adv_full = b.advantages
     resp = torch.arange(T, device=dev) // 512
     b.advantages = torch.where(resp % 4 == 3, torch.zeros_like(adv_full), adv_full)
-    for _ in range(2):
-        step()
-    e0.record()
-    for _ in range(max(1, steps // 2)):
-        step()
-    e1.record()
-    torch.cuda.synchronize()
-    ms_sparse = e0.elapsed_time(e1) / max(1, steps // 2)
+    ms_sparse = _time_steps(torch, step, steps, warmup)          # same run length as above: the step is power-bound
     b.advantages = adv_full
+    # the same step with the LM head (and its gradient) stored [V, d]
+    w_vd = b.lm_head.t().contiguous()
+    dW_vd = dW.view(V, d)
+    fn_vd = lambda: dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, w_vd, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.BINARY_TV, DELTA,
+                                                   workspace=ws, dHidden=dH, dW=dW_vd, status=status, w_is_vd=True)
+    ms_vd = _time_steps(torch, fn_vd, steps, warmup)
+    del w_vd
     # the same step with the Top-K TV divergence (K = 20): adds W^T and T x K gather dot products to the forward
     ms_topk = None
     if T == 8192:
@@ -116,7 +116,7 @@ def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
         fn = lambda: dppo.dppo_fused_lmhead_fwd_bwd(bk.hidden, bk.lm_head, bk.sampled_ids, bk.mu_logp, bk.advantages, None,
                                                     dppo.TOPK_TV, DELTA, K=20, mu_topk_ids=bk.mu_topk_ids, mu_topk_p=bk.mu_topk_p,
                                                     workspace=wsk, dHidden=dH, dW=dW, status=status)
-        ms_topk = _time_steps(torch, fn, max(1, steps // 2), 2)
+        ms_topk = _time_steps(torch, fn, steps, warmup)
         assert int(status.item()) == 0
         del bk, wsk
     peak, src = measured_tensor_peak()
@@ -127,7 +127,8 @@ def bench_fused(dppo, wl, dev, steps=10, warmup=3, T=8192):
                          "traffic": None, "peak_source": "of " + src,
                          "flop_count": "6*T*d*V (forward, dHidden, dW); nothing is recomputed"},
             "gpu_launches_per_step": 15, "loss": float(out["loss"].item()),
-            "ms_per_step_quarter_of_responses_zero_advantage": ms_sparse, "ms_per_step_topk_tv_k20": ms_topk}
+            "ms_per_step_quarter_of_responses_zero_advantage": ms_sparse, "ms_per_step_topk_tv_k20": ms_topk,
+            "ms_per_step_lm_head_vocab_major": ms_vd}
 
 
 def _time_steps(torch, fn, steps, warmup):
@@ -385,7 +386,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(dev))
     variant = dppo.BINARY_TV if args.variant == "binary_tv" else dppo.BINARY_KL
     if args.fused_only:
-        print(json.dumps({"fused_lm_head": bench_fused(dppo, wl, dev, steps=max(1, min(args.steps, 10)), warmup=max(1, min(args.warmup, 3)), T=args.fused_rows)}))
+        print(json.dumps({"fused_lm_head": bench_fused(dppo, wl, dev, steps=max(1, min(args.steps, 40)), warmup=max(1, min(args.warmup, 10)), T=args.fused_rows)}))
         return
 
     if args.variants_only:
