@@ -144,7 +144,7 @@ def _time_steps(torch, fn, steps, warmup):
     return e0.elapsed_time(e1) / steps
 
 
-def bench_other_configs(dppo, wl, dev, steps=20, warmup=3, n_resp=16):
+def bench_other_configs(dppo, wl, dev, steps=100, warmup=10, n_resp=16):
     """The other streaming configurations at full size (same kernel, other variant switches), and the exact
     full-vocabulary divergence monitor.  Extra objects of the benchmark line; the headline stays Binary-TV."""
     import torch
@@ -285,7 +285,12 @@ class ClockSampler:
                 mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
                 reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
                     else int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
-                self.samples.append((time.perf_counter(), mhz, reasons))
+                mem = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_MEM))
+                try:
+                    watts = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                except Exception:  # noqa: BLE001
+                    watts = None
+                self.samples.append((time.perf_counter(), mhz, reasons, mem, watts))
             except Exception:  # noqa: BLE001
                 pass
             time.sleep(0.01)
@@ -311,7 +316,10 @@ class ClockSampler:
         for s in sel:
             bits |= s[2]
         reasons = sorted(n for b, n in names.items() if bits & b)
-        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(sel)}
+        mem = sorted(s[3] for s in sel)
+        watts = sorted(s[4] for s in sel if s[4] is not None)
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(sel),
+                "mem_mhz": mem[len(mem) // 2], "power_w": watts[len(watts) // 2] if watts else None}
 
 
 # ----------------------------------------------------------------------------------------- oracle arm
@@ -390,7 +398,7 @@ def run_ours(args):
         return
 
     if args.variants_only:
-        print(json.dumps({"other_configs": bench_other_configs(dppo, wl, dev, steps=max(1, min(args.steps, 20)), warmup=max(1, min(args.warmup, 3)),
+        print(json.dumps({"other_configs": bench_other_configs(dppo, wl, dev, steps=max(1, min(args.steps, 100)), warmup=max(1, min(args.warmup, 10)),
                                                                  n_resp=max(1, args.rows // 1024))}))
         return
 
