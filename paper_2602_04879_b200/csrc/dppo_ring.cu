@@ -311,23 +311,29 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
                   for (int i = 0; i < N; ++i) vm = fmaxf(vm, z[k][i]);
                 if (vm != -INFINITY) { ref = vm; nm = -vm * kLog2e; }
               }
-              float acc[kVecPerThread];
+              // exponent arguments and partial sums on pairs of fp32 lanes (one instruction per two elements)
+              const float2 l2 = make_float2(kLog2e, kLog2e), nm2 = make_float2(nm, nm);
+              float2 acc2[kVecPerThread];
 #pragma unroll
               for (int k = 0; k < kVecPerThread; ++k) {
-                float e[N];
+                float2 e2[N / 2];
 #pragma unroll
-                for (int i = 0; i < N; ++i) e[i] = ex2_approx(fmaf(z[k][i], kLog2e, nm));
+                for (int i = 0; i < N / 2; ++i) {
+                  const float2 arg = __ffma2_rn(make_float2(z[k][2 * i], z[k][2 * i + 1]), l2, nm2);
+                  e2[i] = make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
+                }
 #pragma unroll
-                for (int w = 1; w < N; w <<= 1)
+                for (int w = 1; w < N / 2; w <<= 1)
 #pragma unroll
-                  for (int i = 0; i + w < N; i += 2 * w) e[i] += e[i + w];
-                acc[k] = e[0];
+                  for (int i = 0; i + w < N / 2; i += 2 * w) e2[i] = __fadd2_rn(e2[i], e2[i + w]);
+                acc2[k] = e2[0];
               }
 #pragma unroll
               for (int w = 1; w < kVecPerThread; w <<= 1)
 #pragma unroll
-                for (int k = 0; k + w < kVecPerThread; k += 2 * w) acc[k] += acc[k + w];
-              if (acc[0] <= 7.3786976e19f && ref != -INFINITY) { s += acc[0]; done = true; }   // <= 2^66, not NaN
+                for (int k = 0; k + w < kVecPerThread; k += 2 * w) acc2[k] = __fadd2_rn(acc2[k], acc2[k + w]);
+              const float acc = acc2[0].x + acc2[0].y;
+              if (acc <= 7.3786976e19f && ref != -INFINITY) { s += acc; done = true; }   // <= 2^66, not NaN
             }
             if (!done) {
               // tail chunk, or an entry far above the reference (or NaN): vector by vector, moving the reference up
@@ -439,8 +445,13 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
               for (int k = 0; k < kVecPerThread; ++k) {
                 float z[N], v[N];
                 Vec<InT>::unpack(raw[k], z);
+                const float2 l2 = make_float2(kLog2e, kLog2e), c22 = make_float2(coef.c2, coef.c2);
 #pragma unroll
-                for (int i = 0; i < N; ++i) v[i] = ex2_approx(fmaf(z[i], kLog2e, coef.c2));
+                for (int i = 0; i < N; i += 2) {
+                  const float2 arg = __ffma2_rn(make_float2(z[i], z[i + 1]), l2, c22);
+                  v[i] = ex2_approx(arg.x);
+                  v[i + 1] = ex2_approx(arg.y);
+                }
                 if (SH && c == 0 && k == 0 && gtid == 0 && gm.head != 0) store_edge<OutT, N>(drow, 0u, v, sign2, gm.head, gm.xend);
                 else Store<OutT, N>::run(drow, e0 + ((uint32_t)k * kGroupThreads + gtid) * N, v, sign2);
               }
