@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default="binary_tv", choices=["binary_tv", "binary_kl"])
     ap.add_argument("--rows", type=int, default=T_ROWS, help="rows per GPU; anything but the default is a reduced case for profiling, not the benchmark workload")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "ring", "scale", "generic"], help="row kernel of the main measurement")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--fused-only", action="store_true", help="run only the fused LM-head measurement (profiling aid)")
     ap.add_argument("--fused-rows", type=int, default=8192, help="token rows of the fused measurement; anything but 8192 is a reduced profiling case")
@@ -410,9 +411,11 @@ def run_ours(args):
     ws = torch.empty(dppo.dppo_workspace_bytes(T), dtype=torch.uint8, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
 
+    kernel_code = {"auto": dppo.KERNEL_AUTO, "ring": dppo.KERNEL_RING, "scale": dppo.KERNEL_SCALE, "generic": dppo.KERNEL_GENERIC}[args.kernel]
+
     def step():
         return dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, variant, 0, DELTA,
-                                      loss_scale=scale, dlogits=dlogits, workspace=ws, status=status)
+                                      loss_scale=scale, dlogits=dlogits, workspace=ws, status=status, kernel=kernel_code)
 
     def barrier():
         if world > 1:

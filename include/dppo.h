@@ -63,8 +63,11 @@ enum { DPPO_DLOGITS_SAME = 0, DPPO_DLOGITS_F32 = 1 };
 /* opts->kernel.  RING: the bulk-copy (TMA) streaming kernel; it takes logits / dlogits whose bases are 16-byte aligned
  * and whose rows either all start on 16-byte boundaries with V * element size a multiple of 16, or are shifted alike
  * (same element size, row strides in bytes equal modulo 16: e.g. both contiguous with an odd V).  GENERIC: element-wise
- * kernel for any layout (several times slower).  AUTO picks RING whenever it can take the layout. */
-enum { DPPO_KERNEL_AUTO = 0, DPPO_KERNEL_GENERIC = 1, DPPO_KERNEL_RING = 2 };
+ * kernel for any layout (several times slower).  AUTO picks RING whenever it can take the layout.  SCALE: an alternative
+ * streaming kernel with one exponential per logit instead of two (the first sweep writes exp(z - z[a_t]) into dlogits, the
+ * second rescales it): 16-byte aligned rows only, dlogits must not overlap logits; it moves fewer bytes to and from HBM
+ * but is currently slower than RING and therefore never picked by AUTO. */
+enum { DPPO_KERNEL_AUTO = 0, DPPO_KERNEL_GENERIC = 1, DPPO_KERNEL_RING = 2, DPPO_KERNEL_SCALE = 3 };
 
 /* Host-visible error codes. */
 enum {

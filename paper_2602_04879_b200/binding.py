@@ -16,7 +16,7 @@ import torch
 BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL, PPO_CLIP, MINIMAL_MASK, GIVEN_D = 0, 1, 2, 3, 4, 5, 6
 F32, BF16 = 0, 1
 DLOGITS_SAME, DLOGITS_F32 = 0, 1
-KERNEL_AUTO, KERNEL_GENERIC, KERNEL_RING = 0, 1, 2
+KERNEL_AUTO, KERNEL_GENERIC, KERNEL_RING, KERNEL_SCALE = 0, 1, 2, 3
 STATUS_BAD_SAMPLED_ID, STATUS_BAD_TOPK_ID, STATUS_NONFINITE_ROW, STATUS_WAIT_LIMIT = 1, 2, 4, 8
 VARIANTS = {"binary_tv": BINARY_TV, "binary_kl": BINARY_KL, "topk_tv": TOPK_TV, "topk_kl": TOPK_KL, "ppo_clip": PPO_CLIP, "minimal_mask": MINIMAL_MASK, "given_d": GIVEN_D}
 

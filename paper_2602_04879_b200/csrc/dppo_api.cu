@@ -55,7 +55,7 @@ int dppo_loss_fwd_bwd(const void* logits, int64_t T, int64_t V, int64_t logits_r
   if (logits_dtype != DPPO_F32 && logits_dtype != DPPO_BF16) return DPPO_ERR_DTYPE;
   if (o.dlogits_dtype != DPPO_DLOGITS_SAME && o.dlogits_dtype != DPPO_DLOGITS_F32) return DPPO_ERR_DTYPE;
   if (variant < DPPO_BINARY_TV || variant > DPPO_GIVEN_D) return DPPO_ERR_VARIANT;
-  if (o.kernel < DPPO_KERNEL_AUTO || o.kernel > DPPO_KERNEL_RING) return DPPO_ERR_UNSUPPORTED;
+  if (o.kernel < DPPO_KERNEL_AUTO || o.kernel > DPPO_KERNEL_SCALE) return DPPO_ERR_UNSUPPORTED;
   if (!loss || !status) return DPPO_ERR_NULL;
   if (T > 0 && (!logits || !sampled_ids || !mu_logp || !advantages || !divergence || !mask || !dlogits)) return DPPO_ERR_NULL;
   const bool topk = (variant == DPPO_TOPK_TV || variant == DPPO_TOPK_KL);
@@ -82,13 +82,17 @@ int dppo_loss_fwd_bwd(const void* logits, int64_t T, int64_t V, int64_t logits_r
   p.row_absdiff = reinterpret_cast<float*>(ws + kAlign + 2 * per);
 
   const bool ring_ok = dppo::ring_layout_ok(p, logits_dtype, out_dtype);
+  const bool scale_ok = dppo::scale_layout_ok(p, logits_dtype, out_dtype);
   if (o.kernel == DPPO_KERNEL_RING && !ring_ok) return DPPO_ERR_ALIGN;
+  if (o.kernel == DPPO_KERNEL_SCALE && !scale_ok) return DPPO_ERR_ALIGN;
+  const bool use_scale = (o.kernel == DPPO_KERNEL_SCALE);
   const bool use_ring = (o.kernel == DPPO_KERNEL_RING) || (o.kernel == DPPO_KERNEL_AUTO && ring_ok);
 
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (dppo::launch_prelude(p, st) != cudaSuccess) return DPPO_ERR_CUDA;
-  cudaError_t e = use_ring ? dppo::launch_ring(p, logits_dtype, out_dtype, st)
-                           : dppo::launch_generic(p, logits_dtype, out_dtype, st);
+  cudaError_t e = use_scale ? dppo::launch_scale(p, logits_dtype, out_dtype, st)
+                  : use_ring ? dppo::launch_ring(p, logits_dtype, out_dtype, st)
+                             : dppo::launch_generic(p, logits_dtype, out_dtype, st);
   if (e != cudaSuccess) return DPPO_ERR_CUDA;
   if (dppo::launch_finalize(p, st) != cudaSuccess) return DPPO_ERR_CUDA;
   return DPPO_OK;

@@ -203,5 +203,7 @@ cudaError_t launch_finalize(const RowParams& p, cudaStream_t st);
 cudaError_t launch_generic(const RowParams& p, int in_dtype, int out_dtype, cudaStream_t st);
 cudaError_t launch_ring(const RowParams& p, int in_dtype, int out_dtype, cudaStream_t st);
 bool ring_layout_ok(const RowParams& p, int in_dtype, int out_dtype);
+cudaError_t launch_scale(const RowParams& p, int in_dtype, int out_dtype, cudaStream_t st);
+bool scale_layout_ok(const RowParams& p, int in_dtype, int out_dtype);
 
 }  // namespace dppo

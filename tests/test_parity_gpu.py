@@ -410,3 +410,48 @@ def test_host_buffer_entry_with_an_odd_vocabulary():
     assert torch.all((a_ - b_).abs() <= 2.0 ** -7 * b_.abs())
     assert abs(out["loss"] - float(dev["loss"].item())) <= 1e-4 * abs(out["loss"]) + 1e-12
 
+
+# ------------------------------------------------------------------------------------- one-exponential kernel
+
+@pytest.mark.parametrize("variant,K,delta", [(dppo.BINARY_TV, 0, 0.02), (dppo.BINARY_KL, 0, 0.002), (dppo.TOPK_TV, 64, 0.05), (dppo.TOPK_KL, 64, 0.02)])
+def test_scale_kernel_matches_oracle(qwen_rows, variant, K, delta):
+    """KERNEL_SCALE: exp(z - z[a_t]) written into dlogits by the first sweep and rescaled by the second (one exponential per
+    logit instead of two).  Same tolerances as the two-sweep kernel: with a bf16 gradient the value is rounded twice, which
+    stays within one bf16 unit of the rounded oracle value."""
+    _full_check(qwen_rows, variant, K, delta, dppo.KERNEL_SCALE)
+    _full_check(qwen_rows, variant, K, delta, dppo.KERNEL_SCALE, dlogits_f32=True)
+
+
+def test_scale_kernel_tiny_fp32_and_edge_rows():
+    b = wl.tiny_binary_tv(DEV, seed=0)
+    _full_check(b, dppo.BINARY_TV, 0, 0.2, dppo.KERNEL_SCALE)
+    # rows whose sampled token is (nearly) impossible under the trainer policy go through the two-sweep fallback inside
+    # the kernel; -inf entries are probability zero; invalid rows are zero-filled; bad ids / non-finite rows set status bits
+    b = wl.tiny_binary_tv(DEV, seed=4, T=64, V=4096)
+    z = b.logits.clone()
+    z[5] = z[5] * 30.0                                   # spread of several hundred: the sampled token may be far below the maximum
+    z[6, :] = -200.0
+    z[6, 17] = 150.0                                     # pi(a) = e^-350 for a != 17
+    z[7, 3::5] = float("-inf")
+    b.logits = z
+    b.sampled_ids[5] = int(torch.argmin(z[5]).item())
+    b.sampled_ids[6] = 100
+    b.sampled_ids[7] = 4
+    b.mu_logp[5] = -60.0
+    b.mu_logp[6] = -349.5                                # ratio e^-0.5: a real gradient on a row the fast path cannot represent
+    tok = torch.ones(64, dtype=torch.uint8, device=DEV)
+    tok[9] = 0
+    b.token_mask = tok
+    out, ora, _ = _full_check(b, dppo.BINARY_TV, 0, 0.2, dppo.KERNEL_SCALE)
+    assert np.abs(ora["dlogits"][6]).max() > 0 and not out["dlogits"][9].any()
+    ring = _run(b, dppo.BINARY_TV, 0, 0.2, dppo.KERNEL_RING)
+    assert torch.equal(ring["mask"], out["mask"])
+    b.sampled_ids[3] = 4096
+    b.logits[20, 7] = float("nan")
+    bad = _run(b, dppo.BINARY_TV, 0, 0.2, dppo.KERNEL_SCALE)
+    assert int(bad["status"].item()) == (dppo.binding.STATUS_BAD_SAMPLED_ID | dppo.binding.STATUS_NONFINITE_ROW)
+    assert not bad["dlogits"][3].any() and not bad["dlogits"][20].any() and bad["mask"][20].item() == 0
+    # layouts it cannot take: in place, rows that are not whole 16-byte vectors
+    with pytest.raises(dppo.DppoError):
+        _run(b, dppo.BINARY_TV, 0, 0.2, dppo.KERNEL_SCALE, dlogits=b.logits)
+
