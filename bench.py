@@ -255,7 +255,7 @@ TRAFFIC_KERNEL_SHA = "9c2fd02dee131b38"
 def measured_traffic():
     import hashlib
     h = hashlib.sha256()
-    for f in ("dppo_ring.cu", "dppo_common.cuh", "dppo_pipe.cuh"):
+    for f in ("dppo_ring.cu", "dppo_common.cuh", "dppo_pipe.cuh", "dppo_rowtools.cuh"):
         with open(os.path.join(ROOT, "paper_2602_04879_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return TRAFFIC_BYTES_PER_LAUNCH if h.hexdigest()[:16] == TRAFFIC_KERNEL_SHA else None

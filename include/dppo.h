@@ -261,6 +261,13 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
 int dppo_gemm_cta_group(int cta_group);
 
 /*
+ * Tuning switch of the DPPO_KERNEL_SCALE row kernel (process-wide; the paper has no counterpart): how many of the 16 KB
+ * shared-memory slots feed the first sweep (the rest feed the second), and how many chunks beyond one row the first
+ * sweep may run ahead of the second (the rows in between wait in L2).  0 selects the built-in default for either.
+ */
+void dppo_scale_kernel_tuning(int sum_slots, int lead_chunks_beyond_row);
+
+/*
  * The tensor-core GEMM the fused variant is built from, exposed for testing and reuse:
  * C[M, N] (fp32, row stride ldc) = A[M, K] . B[N, K]^T with A and B bf16 row-major (row strides lda, ldb elements,
  * multiples of 8; 16-byte aligned bases), fp32 accumulation.  status: device word, DPPO_STATUS_WAIT_LIMIT on a

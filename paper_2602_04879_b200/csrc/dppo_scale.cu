@@ -28,6 +28,8 @@
 // Layouts: 16-byte aligned rows (as the two-sweep kernel's aligned mode), dlogits not overlapping logits.  With a bf16
 // gradient E is rounded to bf16 before it is rescaled and rounded again: the result is within one bf16 unit of the
 // correctly rounded gradient.  Every wait is bounded (about 2 s, then DPPO_STATUS_WAIT_LIMIT).
+#include <atomic>
+
 #include "dppo_common.cuh"
 #include "dppo_pipe.cuh"
 #include "dppo_rowtools.cuh"
@@ -135,7 +137,7 @@ __device__ __forceinline__ double warp_row_lse(const InT* zrow, int64_t V) {
 }
 
 template <typename InT, typename OutT>
-__global__ void __launch_bounds__(kSThreads, 1) dppo_row_scale_kernel(RowParams p, int nslots) {
+__global__ void __launch_bounds__(kSThreads, 1) dppo_row_scale_kernel(RowParams p, int nslots, int sum_slots, int lead_extra) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int N = Vec<InT>::N;
   ScaleMisc* misc = reinterpret_cast<ScaleMisc*>(smem + (size_t)nslots * kSChunk);
@@ -170,7 +172,8 @@ __global__ void __launch_bounds__(kSThreads, 1) dppo_row_scale_kernel(RowParams 
   const uint32_t erow_bytes = (uint32_t)(p.V * (int64_t)sizeof(OutT));    // launcher guarantees < 2^31
   const int CO = (int)((erow_bytes + kSChunk - 1) / kSChunk);             // chunks of a row of E
   // slots [0, ns_sum) feed the sum warps, [ns_sum, nslots) the grad warps (same split as the two-sweep kernel)
-  const int ns_sum = (2 * nslots + 3) / 7 < 2 ? 2 : (2 * nslots + 3) / 7, ns_grad = nslots - ns_sum;
+  const int ns_sum = (sum_slots >= 2 && sum_slots <= nslots - 2) ? sum_slots : ((2 * nslots + 3) / 7 < 2 ? 2 : (2 * nslots + 3) / 7);
+  const int ns_grad = nslots - ns_sum;
   const int64_t t0 = blockIdx.x, G = gridDim.x;
   const InT* logits = reinterpret_cast<const InT*>(p.logits);
   OutT* dlogits = reinterpret_cast<OutT*>(p.dlogits);
@@ -181,7 +184,7 @@ __global__ void __launch_bounds__(kSThreads, 1) dppo_row_scale_kernel(RowParams 
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));    // the logits are read once
       // at most one row and a few chunks ahead of the second sweep: the rows in between wait in L2 as E
-      const unsigned int lead_chunks = (unsigned int)((C + 7 <= 26 || C + 2 > 26) ? ((C + 7 <= 26) ? C + 7 : C + 2) : 26);
+      const unsigned int lead_chunks = (unsigned int)(C + (lead_extra >= 2 ? lead_extra : 7));
       const unsigned int lead = lead_chunks * (unsigned int)(kSChunk / sizeof(InT));           // in elements
       volatile unsigned int* follow = &misc->grad_elems;
       RingPos pos{0, 0};
@@ -540,6 +543,10 @@ __global__ void __launch_bounds__(kSThreads, 1) dppo_row_scale_kernel(RowParams 
   }
 }
 
+// Tuning of the one-exponential kernel (process-wide): slots of the first sweep's ring (the rest feeds the second sweep)
+// and how many chunks beyond one row the first sweep may run ahead of the second.  0 = built-in defaults.
+std::atomic<int> g_sum_slots{0}, g_lead_extra{0};
+
 int scale_slots(int dev) {
   int max_smem = 0;
   cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
@@ -558,7 +565,7 @@ cudaError_t launch_scale_t(const RowParams& p, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(dppo_row_scale_kernel<InT, OutT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int grid = (int)(p.T < sms ? p.T : sms);
-  dppo_row_scale_kernel<InT, OutT><<<grid, kSThreads, smem, st>>>(p, nslots);
+  dppo_row_scale_kernel<InT, OutT><<<grid, kSThreads, smem, st>>>(p, nslots, g_sum_slots.load(), g_lead_extra.load());
   return cudaGetLastError();
 }
 
@@ -589,3 +596,8 @@ cudaError_t launch_scale(const RowParams& p, int in_dtype, int out_dtype, cudaSt
 }
 
 }  // namespace dppo
+
+extern "C" void dppo_scale_kernel_tuning(int sum_slots, int lead_chunks_beyond_row) {
+  dppo::g_sum_slots.store(sum_slots);
+  dppo::g_lead_extra.store(lead_chunks_beyond_row);
+}
