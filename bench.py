@@ -248,8 +248,8 @@ def bench_other_configs(dppo, wl, dev, steps=100, warmup=10, n_resp=16):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one full-size launch of the row kernel, from the ncu
 # capture summarised under profiles/ (row ring kernel, V = 151936), and the hash of the kernel sources it was
 # taken with: once the kernel changes the figure no longer applies and None is reported.
-TRAFFIC_BYTES_PER_LAUNCH = 5518040064 + 4917037995
-TRAFFIC_KERNEL_SHA = "9c2fd02dee131b38"
+TRAFFIC_BYTES_PER_LAUNCH = 5543847680 + 4916382805
+TRAFFIC_KERNEL_SHA = "c42e24126b7766c9"
 
 
 def measured_traffic():
