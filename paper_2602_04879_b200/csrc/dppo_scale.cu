@@ -67,11 +67,6 @@ struct ScaleMisc {
 };
 static_assert(sizeof(ScaleMisc) <= kSMisc, "misc area");
 
-__device__ __forceinline__ uint4 ldg128_l2(const void* p) {          // served by L2 (not kept in L1)
-  uint4 v;
-  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
 __device__ __forceinline__ uint64_t keep_policy() {
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
@@ -82,14 +77,11 @@ __device__ __forceinline__ void stg128_keep(void* p, uint4 v) {      // stays in
   asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "l"(pol) : "memory");
 }
 
-// N exponentials (one input vector) stored in the output dtype at element j0 of the row, to be read back.
+// N exponentials (one input vector) stored in the output dtype at element j0 of the row, to be read back by bulk copies.
 template <typename OutT, int N> struct KeepE;
 template <> struct KeepE<__nv_bfloat16, 8> {
   static __device__ __forceinline__ void run(__nv_bfloat16* row, uint32_t j0, const float* e) {
     stg128_keep(row + j0, make_uint4(pack_bf16x2(e[0], e[1]), pack_bf16x2(e[2], e[3]), pack_bf16x2(e[4], e[5]), pack_bf16x2(e[6], e[7])));
-  }
-  static __device__ __forceinline__ void load(const __nv_bfloat16* row, uint32_t j0, float* e) {
-    Vec<__nv_bfloat16>::unpack(ldg128_l2(row + j0), e);
   }
 };
 template <> struct KeepE<float, 8> {
@@ -97,16 +89,11 @@ template <> struct KeepE<float, 8> {
     stg128_keep(row + j0, make_uint4(__float_as_uint(e[0]), __float_as_uint(e[1]), __float_as_uint(e[2]), __float_as_uint(e[3])));
     stg128_keep(row + j0 + 4, make_uint4(__float_as_uint(e[4]), __float_as_uint(e[5]), __float_as_uint(e[6]), __float_as_uint(e[7])));
   }
-  static __device__ __forceinline__ void load(const float* row, uint32_t j0, float* e) {
-    Vec<float>::unpack(ldg128_l2(row + j0), e);
-    Vec<float>::unpack(ldg128_l2(row + j0 + 4), e + 4);
-  }
 };
 template <> struct KeepE<float, 4> {
   static __device__ __forceinline__ void run(float* row, uint32_t j0, const float* e) {
     stg128_keep(row + j0, make_uint4(__float_as_uint(e[0]), __float_as_uint(e[1]), __float_as_uint(e[2]), __float_as_uint(e[3])));
   }
-  static __device__ __forceinline__ void load(const float* row, uint32_t j0, float* e) { Vec<float>::unpack(ldg128_l2(row + j0), e); }
 };
 
 // log-sum-exp of one row by one warp, with a running maximum, straight from global memory (fallback rows only).
