@@ -24,6 +24,8 @@ Reinforcement Learning", DPPO):
                                 full-vocabulary TV or KL of ``exact_divergence_row``, which the Binary / Top-K forms
                                 approximate, Sec. 4.4): the mask rule and everything after it are unchanged.
 * ``dppo_fused_lmhead_fwd_bwd`` the same applied to logits = H W with the chain rule into H and W.
+* ``dppo_fused_lmhead_sampled`` the same, with the two gradients evaluated only on chosen columns of dW and rows of
+                                dHidden (for checks at sizes where the full [T, V] gradient does not fit the host).
 
 Readings of points the paper leaves open (each is listed in the design notes):
 the library *minimises*, so loss = -s * sum_t M_t r_t A_t with a caller scale s
@@ -289,3 +291,45 @@ def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token
     o["dHidden"] = o["dlogits"] @ Wm.T
     o["dW"] = H.T @ o["dlogits"]
     return o
+
+
+def dppo_fused_lmhead_sampled(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV,
+                              delta=0.2, loss_scale=None, dW_cols=(), dH_rows=(), K=0, mu_topk_ids=None, mu_topk_p=None,
+                              is_cap=None, eps_low=None, row_block=256):
+    """The LM-head variant where a full evaluation does not fit: loss, D, M, r for ALL rows, but of the two gradients only
+    the columns ``dW_cols`` of dW and the rows ``dH_rows`` of dHidden.  Same definitions as ``dppo_fused_lmhead_fwd_bwd``:
+    logits = hidden @ W in float64, row by row through ``dppo_row``; dlogits_tj = g_t (pi_tj - 1[j = a_t]) (Eq. unified_grad);
+    dW[:, c] = hidden^T @ dlogits[:, c]; dHidden[t] = dlogits[t] @ W^T.  The logits are formed ``row_block`` rows at a
+    time to bound memory; nothing else is blocked.  Returns dict(loss, D, M, r, row_loss, dW_cols [d, len(dW_cols)],
+    dlogits_cols [T, len(dW_cols)], dHidden_rows [len(dH_rows), d], dlogits_rows [len(dH_rows), V], scale)."""
+    H = _f64(hidden)
+    Wm = _f64(W)
+    T, V = H.shape[0], Wm.shape[1]
+    cols = np.asarray(list(dW_cols), dtype=np.int64)
+    rows = [int(t) for t in dH_rows]
+    s = default_scale(T, token_mask) if loss_scale is None else float(loss_scale)
+    D = np.zeros(T)
+    M = np.zeros(T, dtype=np.uint8)
+    r = np.zeros(T)
+    row_loss = np.zeros(T)
+    dl_cols = np.zeros((T, len(cols)))
+    dl_rows = np.zeros((len(rows), V))
+    for t0 in range(0, T, int(row_block)):
+        z = H[t0:t0 + int(row_block)] @ Wm
+        for i in range(z.shape[0]):
+            t = t0 + i
+            if token_mask is not None and not token_mask[t]:
+                continue
+            ids = ps = None
+            if variant in (TOPK_TV, TOPK_KL) and K > 0:
+                ids, ps = mu_topk_ids[t][:K], mu_topk_p[t][:K]
+            o = dppo_row(z[i], sampled_ids[t], mu_logp[t], advantages[t], variant, delta, s, ids, ps, False, is_cap, eps_low)
+            D[t], M[t], r[t], row_loss[t] = o["D"], o["M"], o["r"], o["loss"]
+            a = int(sampled_ids[t])
+            dl_cols[t] = o["g"] * (np.exp(z[i, cols] - o["lse"]) - (cols == a))
+            if t in rows:
+                full = o["g"] * np.exp(z[i] - o["lse"])
+                full[a] -= o["g"]
+                dl_rows[rows.index(t)] = full
+    return dict(loss=float(np.sum(row_loss)), D=D, M=M, r=r, row_loss=row_loss, dW_cols=H.T @ dl_cols, dlogits_cols=dl_cols,
+                dHidden_rows=dl_rows @ Wm.T, dlogits_rows=dl_rows, scale=s)

@@ -389,6 +389,44 @@ def check_fused(O):
     assert abs(fd - o["dW"][0, 4]) < 2e-8
 
 
+def check_fused_sampled(O):
+    """The column / row restricted LM-head form against torch autograd (float64) of the surrogate with the mask held
+    fixed, and against the full form; ragged row blocks, a token mask, Top-K lists, an importance cap."""
+    rng = np.random.default_rng(21)
+    T, d, V, K = 23, 5, 17, 4
+    H = rng.standard_normal((T, d))
+    W = 0.8 * rng.standard_normal((d, V))
+    zmu = H @ W + 0.7 * rng.standard_normal((T, V))
+    mu = np.exp(zmu - scipy.special.logsumexp(zmu, axis=1, keepdims=True))
+    a = np.array([rng.choice(V, p=mu[t]) for t in range(T)])
+    mu_logp = np.log(mu[np.arange(T), a])
+    ids = np.argsort(-mu, axis=1)[:, :K]
+    ps = np.take_along_axis(mu, ids, axis=1)
+    adv = rng.choice([-1.0, 1.0], T) * rng.uniform(0.3, 1.2, T)
+    tok = (np.arange(T) % 6 != 2).astype(np.uint8)
+    cols = [0, 3, int(a[1]), int(a[5]), V - 1]
+    rows = [0, 5, 8, T - 1]                 # row 8 is masked out: a zero row
+    for variant, delta, cap in ((O.BINARY_TV, 0.03, None), (O.TOPK_KL, 0.02, 1.1)):
+        o = O.dppo_fused_lmhead_sampled(H, W, a, mu_logp, adv, tok, variant, delta, None, cols, rows, K, ids, ps, cap, row_block=7)
+        f = O.dppo_fused_lmhead_fwd_bwd(H, W, a, mu_logp, adv, tok, variant, delta, None, K, ids, ps, cap)
+        assert np.array_equal(o["M"], f["M"]) and 0 < int(((o["M"] == 0) & (tok != 0)).sum())
+        np.testing.assert_allclose(o["D"], f["D"], atol=1e-15)
+        assert abs(o["loss"] - f["loss"]) < 1e-14
+        Ht = torch.tensor(H, requires_grad=True)
+        Wt = torch.tensor(W, requires_grad=True)
+        lp = torch.log_softmax(Ht @ Wt, dim=1)[torch.arange(T), torch.tensor(a)]
+        r = torch.exp(lp - torch.tensor(mu_logp))
+        w = r
+        if cap is not None:     # Eq. unified_grad: value min(r, C), gradient min(r, C) grad(log pi)
+            w = torch.where(r.detach() < cap, r, torch.full_like(r, cap) * (1 + lp - lp.detach()))
+        loss = -(o["scale"] * torch.tensor((o["M"] * (tok != 0)).astype(np.float64)) * w * torch.tensor(adv)).sum()
+        loss.backward()
+        np.testing.assert_allclose(o["dW_cols"], Wt.grad.numpy()[:, cols], atol=1e-13)
+        np.testing.assert_allclose(o["dHidden_rows"], Ht.grad.numpy()[rows], atol=1e-13)
+        assert not o["dHidden_rows"][2].any() and o["dlogits_rows"].shape == (len(rows), V)
+        np.testing.assert_allclose(o["dlogits_cols"], f["dlogits"][:, cols], atol=1e-15)
+
+
 def check_is_cap_and_baselines(O):
     """Eq. unified_grad: weight min(r, C); C = inf is Eq. dppo_obj; delta = inf gives the unmasked PG-IS / CISPO baselines."""
     rng = np.random.default_rng(9)
@@ -523,7 +561,7 @@ def check_given_divergence(O):
 
 CHECKS = [check_given_divergence, check_exact_divergence, check_minimal_mask, check_is_cap_and_baselines, check_ppo_clip_variant, check_worked_example, check_log_softmax, check_binary, check_topk_full_and_bounds,
           check_topk_other_bucket, check_topk_equality_conditions, check_edge_conventions,
-          check_mask_truth_table, check_on_policy, check_gradient, check_brute_force_tiny, check_fused]
+          check_mask_truth_table, check_on_policy, check_gradient, check_brute_force_tiny, check_fused, check_fused_sampled]
 
 
 @pytest.mark.parametrize("check", CHECKS, ids=lambda f: f.__name__)
