@@ -20,9 +20,13 @@
  * Conventions shared by every entry point
  * ---------------------------------------
  *  - Unless a parameter says "host", every pointer is a DEVICE pointer owned by
- *    the caller.  The library allocates nothing, keeps no state between calls,
+ *    the caller.  The library allocates nothing and keeps no state between calls
+ *    (every switch is a field of dppo_opts, per call; the one exception is the
+ *    built-in scratch array of dppo_loss_fwd_bwd_static_ws, see there).  It
  *    enqueues its kernels on `cuda_stream` (a cudaStream_t passed as void*,
  *    NULL = the default stream) and never synchronises.
+ *  - Range checks of the ids and the test for a finite log-sum-exp are always on
+ *    (they cost nothing next to the row's traffic); there is no switch for them.
  *  - Return value: DPPO_OK (0) when the kernels were enqueued; a negative
  *    DPPO_ERR_* code for misuse the host can see, in which case nothing was
  *    launched.  dppo_error_string() names a code.
@@ -63,11 +67,13 @@ enum { DPPO_DLOGITS_SAME = 0, DPPO_DLOGITS_F32 = 1 };
 /* opts->kernel.  RING: the bulk-copy (TMA) streaming kernel; it takes logits / dlogits whose bases are 16-byte aligned
  * and whose rows either all start on 16-byte boundaries with V * element size a multiple of 16, or are shifted alike
  * (same element size, row strides in bytes equal modulo 16: e.g. both contiguous with an odd V).  GENERIC: element-wise
- * kernel for any layout (several times slower).  AUTO picks RING whenever it can take the layout.  SCALE: an alternative
- * streaming kernel with one exponential per logit instead of two (the first sweep writes exp(z - z[a_t]) into dlogits, the
- * second rescales it): 16-byte aligned rows only, dlogits must not overlap logits; it moves fewer bytes to and from HBM
- * but is currently slower than RING and therefore never picked by AUTO. */
-enum { DPPO_KERNEL_AUTO = 0, DPPO_KERNEL_GENERIC = 1, DPPO_KERNEL_RING = 2, DPPO_KERNEL_SCALE = 3 };
+ * kernel for any layout (several times slower).  AUTO picks RING whenever it can take the layout. */
+enum { DPPO_KERNEL_AUTO = 0, DPPO_KERNEL_GENERIC = 1, DPPO_KERNEL_RING = 2 };
+/* opts->test_inject (testing only).  NO_COPIES: the copy producers of the kernels issue nothing, so that every on-chip
+ * wait for data runs out after opts->wait_limit_us and the call returns with DPPO_STATUS_WAIT_LIMIT set and undefined
+ * results; nothing faults or hangs, and the next call works normally.  It exists so that the give-up path of the
+ * bounded waits can be exercised. */
+enum { DPPO_INJECT_NO_COPIES = 1 };
 
 /* Host-visible error codes. */
 enum {
@@ -80,7 +86,7 @@ enum {
   DPPO_ERR_STRIDE = -6,      /* a row stride smaller than V                                  */
   DPPO_ERR_ALIGN = -7,       /* pointer / stride alignment the requested kernel cannot take  */
   DPPO_ERR_WORKSPACE = -8,   /* workspace NULL, misaligned or smaller than dppo_workspace_bytes */
-  DPPO_ERR_ALIAS = -9,       /* dlogits aliases logits but the element sizes differ          */
+  DPPO_ERR_ALIAS = -9,       /* dlogits overlaps logits without being the same tensor in place (same base, element size, stride) */
   DPPO_ERR_CUDA = -10,       /* a CUDA runtime call failed (launch, copy)                    */
   DPPO_ERR_UNSUPPORTED = -11, /* combination not implemented                                 */
   DPPO_ERR_TOO_MANY_ROWS = -12 /* T above DPPO_STATIC_WS_MAX_ROWS (dppo_loss_fwd_bwd_static_ws)  */
@@ -107,12 +113,24 @@ typedef struct dppo_opts {
   float eps_low;       /* DPPO_PPO_CLIP only: lower clip range; <= 0: same as delta                      */
   int lm_head_layout;  /* dppo_fused_lmhead_fwd_bwd only: DPPO_LM_HEAD_DV (0) = W and dW are [d, V] row-major;
                           DPPO_LM_HEAD_VD (1) = both are [V, d] row-major (how a linear layer stores its weight)  */
+  int gemm_cta_group;  /* tensor-core GEMMs (fused variant, dppo_gemm_*): 0 or 2 = 256 x 256 tiles on pairs of SMs
+                          (tcgen05 cta_group::2, each SM stages half of the B tile); 1 = 128 x 256 tiles on single SMs.
+                          The results of the two modes agree up to the order of the fp32 additions in the tensor cores */
+  int fused_rows_per_block;  /* dppo_fused_lmhead_fwd_bwd only: R > 0 finishes the rows in blocks of R (forward, scalars,
+                          dHidden, dW += per block, with the scale s and N_valid of the whole call), so that the
+                          workspace is that of min(T, R) rows whatever T is; 0 = all rows at once.  Multiples of 256
+                          use the tensor-core tiles best */
+  int wait_limit_us;   /* how long one on-chip wait (for a copy, for another warp) may take before the kernel gives up
+                          and sets DPPO_STATUS_WAIT_LIMIT, in microseconds; 0 = about 2 s.  Waits normally take
+                          microseconds; the limit only bounds the damage of a lost copy */
+  int test_inject;     /* DPPO_INJECT_* bits, testing only; 0 in production                                          */
 } dppo_opts;
 enum { DPPO_LM_HEAD_DV = 0, DPPO_LM_HEAD_VD = 1 };
 
-/* Bytes of device scratch dppo_loss_fwd_bwd needs for T rows (256-byte aligned
- * pointer expected).  Contents need no initialisation and carry nothing between calls. */
-size_t dppo_workspace_bytes(int64_t T);
+/* Bytes of device scratch dppo_loss_fwd_bwd needs for a call of this shape (256-byte aligned pointer expected;
+ * today a function of T alone: a header and three fp32 values per row).  Contents need no initialisation and carry
+ * nothing between calls. */
+size_t dppo_workspace_bytes(int64_t T, int64_t V, int K, int variant);
 
 /*
  * Forward + backward of the DPPO loss over T token rows (Eq. dppo_obj; gradient:
@@ -140,11 +158,11 @@ size_t dppo_workspace_bytes(int64_t T);
  *  mask            [T]  out: M_t as bytes (0 for invalid rows).
  *  dlogits         [T, V] out, row stride `dlogits_row_stride` (>= V), dtype per opts; may be the
  *                  same buffer as logits (in place) when the element sizes match and the strides
- *                  are equal.
+ *                  are equal; any other overlap of the two tensors is rejected (DPPO_ERR_ALIAS).
  *  stats           [8] out or NULL: N_valid, N_blocked (valid rows with M = 0), sum D, max D,
  *                  sum |pi(a)-mu(a)|, sum r, sum |loss term|, reserved.  Sums skip non-finite D.
  *  status          [1] in/out device word, see DPPO_STATUS_*.
- *  workspace       device scratch of at least dppo_workspace_bytes(T) bytes.
+ *  workspace       device scratch of at least dppo_workspace_bytes(T, V, K, variant) bytes.
  */
 int dppo_loss_fwd_bwd(const void* logits, int64_t T, int64_t V, int64_t logits_row_stride, int logits_dtype,
                       const int32_t* sampled_ids, const float* mu_logp,
@@ -165,13 +183,15 @@ size_t dppo_host_staging_bytes(int64_t rows_per_chunk, int64_t V, int K, int log
  * in chunks of `rows_per_chunk`, processed, and the per-token outputs copied back, with the
  * copies of one chunk overlapping the kernels of the other on two internal streams.  Pointer
  * arguments with the same names as above have the same meaning but are HOST pointers
- * (contiguous rows: stride V).  `dlogits_host` may be NULL, in which case the gradient rows are
- * left in the staging area of the last chunks and not copied back.  `staging` is DEVICE memory
+ * (contiguous rows: stride V).  `dlogits_host` [T, V] receives the gradient (its copy back to the
+ * host overlaps the next chunk's copy to the device); it may be NULL when only loss, divergence and
+ * mask are wanted, in which case the gradient is computed and dropped.  `staging` is DEVICE memory
  * of at least dppo_host_staging_bytes(...) bytes, 256-byte aligned, owned by the caller.
  * `status_host` receives the OR of the device status words.  Because the token-mean scale needs
  * N_valid of the whole batch before the first chunk, it is counted on the host from token_mask.
  * The call synchronises with the device before returning (the results are on the host).
- * Creates and destroys two CUDA streams and events per call; allocates no device memory.
+ * Creates and destroys two CUDA streams and an event per call; allocates no device memory.
+ * Any number of chunks is fine (the chunks' losses are collected every few thousand chunks).
  */
 int dppo_loss_fwd_bwd_host(const void* logits, int64_t T, int64_t V, int logits_dtype,
                            const int32_t* sampled_ids, const float* mu_logp,
@@ -199,7 +219,8 @@ int dppo_loss_fwd_bwd_host(const void* logits, int64_t T, int64_t V, int logits_
  *   - T may not exceed DPPO_STATIC_WS_MAX_ROWS; a larger T returns DPPO_ERR_TOO_MANY_ROWS and
  *     launches nothing (split the batch and pass opts->loss_scale, as for micro-batches).
  *   - The first call on each device looks up the array's device address (with that device
- *     current).  Make that first call outside any stream capture.
+ *     current) and keeps it for the life of the process.  Make that first call outside any
+ *     stream capture, and do not use this entry point again after a cudaDeviceReset.
  *   - All calls on one device share the one array.  Nothing in it needs clearing: each call
  *     rewrites what it reads, and what the previous call left behind is ignored.  Two calls
  *     whose kernels can overlap on the GPU (different streams, no dependency) race on it and give
@@ -234,6 +255,10 @@ size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V, int K);
  *  dW       [d, V] fp32 out: d loss / d W = hidden^T . dlogits (overwritten, not accumulated).
  *  workspace  device scratch of at least dppo_fused_workspace_bytes(T, d, V, K) bytes; it holds packed copies of hidden
  *           and the bf16 exponentials of the logits (about 2 T V bytes; plus W^T, 2 d V bytes, for Top-K variants).
+ *           With opts->fused_rows_per_block = R > 0 the rows are finished R at a time and the workspace needed is
+ *           dppo_fused_workspace_bytes(min(T, R), d, V, K), whatever T is: nothing of size T x V is ever staged.  The
+ *           results are the same up to the order in which the blocks' contributions to dW are added (fixed: block
+ *           after block), and repeated calls give identical bits.
  * Every logits tile is computed once: the forward GEMM writes exp(z - c_t) in bf16 against a per-row reference known
  * beforehand (c_t = the sampled token's logit) together with the fp32 row sums; the per-row factor g_t / S_t that turns
  * those exponentials into the gradient with respect to the logits is applied to the rows of dHidden in fp32 and to the
@@ -253,32 +278,17 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
                               float* stats, int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Tuning switch of the tensor-core GEMM (process-wide; the paper has no counterpart): 2 (default) computes 256 x 256
- * tiles on pairs of SMs (tcgen05 cta_group::2, each SM stages half of the B tile), 1 computes 128 x 256 tiles on single
- * SMs.  Any other value only queries.  Returns the previous setting.  The results of the two modes are the same up to
- * the order of the fp32 additions inside the tensor cores.
- */
-int dppo_gemm_cta_group(int cta_group);
-
-/*
- * Tuning switch of the DPPO_KERNEL_SCALE row kernel (process-wide; the paper has no counterpart): how many of the 16 KB
- * shared-memory slots feed the first sweep (the rest feed the second), and how many chunks beyond one row the first
- * sweep may run ahead of the second (the rows in between wait in L2).  0 selects the built-in default for either.
- */
-void dppo_scale_kernel_tuning(int sum_slots, int lead_chunks_beyond_row);
-
-/*
  * The tensor-core GEMM the fused variant is built from, exposed for testing and reuse:
  * C[M, N] (fp32, row stride ldc) = A[M, K] . B[N, K]^T with A and B bf16 row-major (row strides lda, ldb elements,
  * multiples of 8; 16-byte aligned bases), fp32 accumulation.  status: device word, DPPO_STATUS_WAIT_LIMIT on a
- * bounded wait that ran out (may be NULL).
+ * bounded wait that ran out (may be NULL).  opts (NULL = defaults): gemm_cta_group, wait_limit_us, test_inject.
  */
 int dppo_gemm_tn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,
-                      int32_t* status, void* cuda_stream);
+                      int32_t* status, const dppo_opts* opts, void* cuda_stream);
 
 /* The same with B given as [K, N] row-major (N contiguous, row stride ldb): C[M, N] = A[M, K] . B[K, N]. */
 int dppo_gemm_nn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,
-                      int32_t* status, void* cuda_stream);
+                      int32_t* status, const dppo_opts* opts, void* cuda_stream);
 
 /*
  * Exact full-vocabulary divergence between the rollout policy and the trainer policy, and the trainer policy's
@@ -288,13 +298,16 @@ int dppo_gemm_nn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, in
  *  logits, mu_logits  [T, V] row-major (row strides in elements, >= V), both of `dtype` (DPPO_F32 or DPPO_BF16).
  *  token_mask         [T] bytes or NULL; rows with a zero byte are not read and give 0.
  *  tv, kl, entropy    [T] out: 1/2 sum_j |mu_j - pi_j|,  sum_j mu_j log(mu_j / pi_j),  -sum_j pi_j log pi_j.
+ *                     tv may be NULL: KL and entropy are complete after one sweep over the two rows, only the TV needs a
+ *                     second one (with both normalisers known), which is then left out.
  *  status             device word; DPPO_STATUS_NONFINITE_ROW if a row's log-sum-exp is not finite (outputs 0).
- * Needs no workspace.  Each row is read twice (the second time normally from L2).
+ *  opts               NULL = defaults; wait_limit_us and test_inject are the fields that apply.
+ * Needs no workspace.  With a TV output each row is read twice (the second time normally from L2), without it once.
  */
 int dppo_exact_divergence(const void* logits, const void* mu_logits, int64_t T, int64_t V,
                           int64_t logits_row_stride, int64_t mu_row_stride, int dtype,
                           const uint8_t* token_mask, float* tv, float* kl, float* entropy,
-                          int32_t* status, void* cuda_stream);
+                          int32_t* status, const dppo_opts* opts, void* cuda_stream);
 
 /* Name of an error code (static string, never NULL). */
 const char* dppo_error_string(int code);

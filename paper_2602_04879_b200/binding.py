@@ -16,7 +16,8 @@ import torch
 BINARY_TV, BINARY_KL, TOPK_TV, TOPK_KL, PPO_CLIP, MINIMAL_MASK, GIVEN_D = 0, 1, 2, 3, 4, 5, 6
 F32, BF16 = 0, 1
 DLOGITS_SAME, DLOGITS_F32 = 0, 1
-KERNEL_AUTO, KERNEL_GENERIC, KERNEL_RING, KERNEL_SCALE = 0, 1, 2, 3
+KERNEL_AUTO, KERNEL_GENERIC, KERNEL_RING = 0, 1, 2
+INJECT_NO_COPIES = 1
 STATUS_BAD_SAMPLED_ID, STATUS_BAD_TOPK_ID, STATUS_NONFINITE_ROW, STATUS_WAIT_LIMIT = 1, 2, 4, 8
 VARIANTS = {"binary_tv": BINARY_TV, "binary_kl": BINARY_KL, "topk_tv": TOPK_TV, "topk_kl": TOPK_KL, "ppo_clip": PPO_CLIP, "minimal_mask": MINIMAL_MASK, "given_d": GIVEN_D}
 
@@ -25,8 +26,16 @@ _lib = None
 
 
 class DppoOpts(ctypes.Structure):
+    """dppo_opts of include/dppo.h (all-zero = defaults)."""
     _fields_ = [("loss_scale", c_float), ("dlogits_dtype", c_int), ("kernel", c_int), ("is_cap", c_float), ("eps_low", c_float),
-                ("lm_head_layout", c_int)]
+                ("lm_head_layout", c_int), ("gemm_cta_group", c_int), ("fused_rows_per_block", c_int), ("wait_limit_us", c_int),
+                ("test_inject", c_int)]
+
+
+def _opts(loss_scale=0.0, dlogits_f32=False, kernel=KERNEL_AUTO, is_cap=0.0, eps_low=0.0, w_is_vd=False, cta_group=0,
+          rows_per_block=0, wait_limit_us=0, test_inject=0):
+    return DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), float(is_cap), float(eps_low),
+                    1 if w_is_vd else 0, int(cta_group), int(rows_per_block), int(wait_limit_us), int(test_inject))
 
 
 class DppoError(RuntimeError):
@@ -46,7 +55,7 @@ def lib():
         L.dppo_error_string.restype = c_char_p
         L.dppo_error_string.argtypes = [c_int]
         L.dppo_workspace_bytes.restype = c_size_t
-        L.dppo_workspace_bytes.argtypes = [c_int64]
+        L.dppo_workspace_bytes.argtypes = [c_int64, c_int64, c_int, c_int]
         L.dppo_loss_fwd_bwd.restype = c_int
         L.dppo_loss_fwd_bwd.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p, c_void_p, c_void_p,
                                         c_void_p, c_void_p, c_int, c_int, c_float, POINTER(DppoOpts),
@@ -68,14 +77,12 @@ def lib():
                                                 c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.dppo_exact_divergence.restype = c_int
         L.dppo_exact_divergence.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p,
-                                            c_void_p, c_void_p, c_void_p, c_void_p]
+                                            c_void_p, c_void_p, c_void_p, POINTER(DppoOpts), c_void_p]
         L.dppo_gemm_tn_bf16.restype = c_int
         L.dppo_gemm_tn_bf16.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_int, c_int, c_int, c_void_p, c_int64,
-                                        c_void_p, c_void_p]
+                                        c_void_p, POINTER(DppoOpts), c_void_p]
         L.dppo_gemm_nn_bf16.restype = c_int
         L.dppo_gemm_nn_bf16.argtypes = L.dppo_gemm_tn_bf16.argtypes
-        L.dppo_gemm_cta_group.restype = c_int
-        L.dppo_gemm_cta_group.argtypes = [c_int]
         L.dppo_loss_fwd_bwd_static_ws.restype = c_int
         L.dppo_loss_fwd_bwd_static_ws.argtypes = L.dppo_loss_fwd_bwd.argtypes[:22] + [c_void_p]
         _lib = L
@@ -102,8 +109,8 @@ def _dtype_code(t):
     raise TypeError(f"logits dtype {t.dtype} not supported (float32 or bfloat16)")
 
 
-def dppo_workspace_bytes(T):
-    return int(lib().dppo_workspace_bytes(int(T)))
+def dppo_workspace_bytes(T, V=1, K=0, variant=BINARY_TV):
+    return int(lib().dppo_workspace_bytes(int(T), int(V), int(K), int(variant)))
 
 
 def _divergence_buffer(T, dev, variant, given):
@@ -117,7 +124,7 @@ def _divergence_buffer(T, dev, variant, given):
 def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, K=0, delta=0.2,
                       mu_topk_ids=None, mu_topk_p=None, loss_scale=0.0, dlogits_f32=False, kernel=KERNEL_AUTO,
                       dlogits=None, want_stats=False, workspace=None, status=None, stream=None, is_cap=0.0, eps_low=0.0,
-                      given_divergence=None):
+                      given_divergence=None, wait_limit_us=0, test_inject=0):
     """Calls ``dppo_loss_fwd_bwd`` on CUDA tensors.  Output tensors are allocated with torch unless
     given.  Returns dict(loss[1], divergence[T], mask[T], dlogits[T,V], stats[8] or None, status[1]);
     nothing is synchronised.  ``given_divergence`` [T] fp32: the per-token divergence for variant GIVEN_D (copied into
@@ -135,7 +142,7 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
     stats = torch.empty(8, dtype=torch.float32, device=dev) if want_stats else None
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
-    nbytes = dppo_workspace_bytes(T)
+    nbytes = dppo_workspace_bytes(T, V, K, variant)
     if workspace is None:
         workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
     for name, t, dt in (("sampled_ids", sampled_ids, torch.int32), ("mu_logp", mu_logp, torch.float32),
@@ -143,7 +150,7 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
                         ("mu_topk_ids", mu_topk_ids, torch.int32), ("mu_topk_p", mu_topk_p, torch.float32)):
         if t is not None:
             assert t.is_cuda and t.dtype == dt and t.is_contiguous(), name
-    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), float(is_cap), float(eps_low))
+    opts = _opts(loss_scale, dlogits_f32, kernel, is_cap, eps_low, wait_limit_us=wait_limit_us, test_inject=test_inject)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     with torch.cuda.device(dev):
         rc = lib().dppo_loss_fwd_bwd(_ptr(logits), T, V, logits.stride(0) if T > 0 else V, _dtype_code(logits),
@@ -163,11 +170,13 @@ def dppo_fused_workspace_bytes(T, d, V, K=0):
 
 def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, delta=0.2,
                               loss_scale=0.0, want_stats=False, workspace=None, dHidden=None, dW=None, status=None, stream=None,
-                              is_cap=0.0, eps_low=0.0, K=0, mu_topk_ids=None, mu_topk_p=None, given_divergence=None, w_is_vd=False):
+                              is_cap=0.0, eps_low=0.0, K=0, mu_topk_ids=None, mu_topk_p=None, given_divergence=None, w_is_vd=False,
+                              cta_group=0, rows_per_block=0, wait_limit_us=0, test_inject=0):
     """Calls ``dppo_fused_lmhead_fwd_bwd`` on CUDA tensors: hidden [T,d] bf16, W [d,V] bf16.  Returns
     dict(loss[1], divergence[T], mask[T], dHidden[T,d] fp32, dW[d,V] fp32, stats, status); nothing is synchronised.
     ``given_divergence``: as for ``dppo_loss_fwd_bwd`` (variant GIVEN_D).  ``w_is_vd``: W (and dW) are [V,d], the layout
-    of a linear layer's weight, instead of [d,V]."""
+    of a linear layer's weight, instead of [d,V].  ``cta_group``, ``rows_per_block``, ``wait_limit_us``, ``test_inject``: the
+    fields of dppo_opts of the same names (``rows_per_block`` = fused_rows_per_block)."""
     assert hidden.is_cuda and W.is_cuda and hidden.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
     assert hidden.is_contiguous() and W.is_contiguous() and hidden.shape[1] == W.shape[1 if w_is_vd else 0]
     T, d = hidden.shape
@@ -184,8 +193,9 @@ def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
     if workspace is None:
-        workspace = torch.empty(dppo_fused_workspace_bytes(T, d, V, K), dtype=torch.uint8, device=dev)
-    opts = DppoOpts(float(loss_scale), 0, 0, float(is_cap), float(eps_low), 1 if w_is_vd else 0)
+        rows = min(T, rows_per_block) if rows_per_block > 0 else T
+        workspace = torch.empty(dppo_fused_workspace_bytes(rows, d, V, K), dtype=torch.uint8, device=dev)
+    opts = _opts(loss_scale, False, 0, is_cap, eps_low, w_is_vd, cta_group, rows_per_block, wait_limit_us, test_inject)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     with torch.cuda.device(dev):
         rc = lib().dppo_fused_lmhead_fwd_bwd(_ptr(hidden), _ptr(W), T, d, V, _ptr(sampled_ids), _ptr(mu_logp),
@@ -198,29 +208,31 @@ def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token
     return dict(loss=loss, divergence=D, mask=M, dHidden=dHidden, dW=dW, stats=stats, status=status)
 
 
-def dppo_exact_divergence(logits, mu_logits, token_mask=None, status=None, stream=None):
+def dppo_exact_divergence(logits, mu_logits, token_mask=None, status=None, stream=None, want_tv=True, wait_limit_us=0,
+                          test_inject=0):
     """Calls ``dppo_exact_divergence``: per-row exact TV, KL(mu||pi) and entropy of pi from two [T,V] CUDA logits tensors
-    of the same dtype.  Returns dict(tv, kl, entropy, status)."""
+    of the same dtype.  Returns dict(tv, kl, entropy, status); ``want_tv=False`` passes tv = NULL (one sweep, tv is None)."""
     assert logits.is_cuda and mu_logits.is_cuda and logits.dtype == mu_logits.dtype and logits.shape == mu_logits.shape
     assert logits.stride(1) == 1 and mu_logits.stride(1) == 1
     T, V = logits.shape
     dev = logits.device
-    tv = torch.empty(T, dtype=torch.float32, device=dev)
+    tv = torch.empty(T, dtype=torch.float32, device=dev) if want_tv else None
     kl = torch.empty(T, dtype=torch.float32, device=dev)
     ent = torch.empty(T, dtype=torch.float32, device=dev)
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
+    opts = _opts(wait_limit_us=wait_limit_us, test_inject=test_inject)
     with torch.cuda.device(dev):
         rc = lib().dppo_exact_divergence(_ptr(logits), _ptr(mu_logits), T, V, logits.stride(0) if T > 0 else V,
                                          mu_logits.stride(0) if T > 0 else V, _dtype_code(logits), _ptr(token_mask), _ptr(tv),
-                                         _ptr(kl), _ptr(ent), _ptr(status), c_void_p(st.cuda_stream))
+                                         _ptr(kl), _ptr(ent), _ptr(status), ctypes.byref(opts), c_void_p(st.cuda_stream))
     if rc != 0:
         raise DppoError(rc, "dppo_exact_divergence")
     return dict(tv=tv, kl=kl, entropy=ent, status=status)
 
 
-def dppo_gemm_tn_bf16(A, B, C=None, status=None, stream=None):
+def dppo_gemm_tn_bf16(A, B, C=None, status=None, stream=None, cta_group=0, wait_limit_us=0, test_inject=0):
     """C[M,N] fp32 = A[M,K] . B[N,K]^T for bf16 CUDA matrices (last dimension contiguous)."""
     assert A.is_cuda and B.is_cuda and A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16
     assert A.stride(1) == 1 and B.stride(1) == 1 and A.shape[1] == B.shape[1]
@@ -233,13 +245,14 @@ def dppo_gemm_tn_bf16(A, B, C=None, status=None, stream=None):
     st = stream if stream is not None else torch.cuda.current_stream(A.device)
     with torch.cuda.device(A.device):
         rc = lib().dppo_gemm_tn_bf16(_ptr(A), A.stride(0), _ptr(B), B.stride(0), M, N, K, _ptr(C), C.stride(0), _ptr(status),
+                                     ctypes.byref(_opts(cta_group=cta_group, wait_limit_us=wait_limit_us, test_inject=test_inject)),
                                      c_void_p(st.cuda_stream))
     if rc != 0:
         raise DppoError(rc, "dppo_gemm_tn_bf16")
     return C, status
 
 
-def dppo_gemm_nn_bf16(A, B, C=None, status=None, stream=None):
+def dppo_gemm_nn_bf16(A, B, C=None, status=None, stream=None, cta_group=0, wait_limit_us=0, test_inject=0):
     """C[M,N] fp32 = A[M,K] . B[K,N] for bf16 CUDA matrices (last dimension contiguous)."""
     assert A.is_cuda and B.is_cuda and A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16
     assert A.stride(1) == 1 and B.stride(1) == 1 and A.shape[1] == B.shape[0]
@@ -252,16 +265,11 @@ def dppo_gemm_nn_bf16(A, B, C=None, status=None, stream=None):
     st = stream if stream is not None else torch.cuda.current_stream(A.device)
     with torch.cuda.device(A.device):
         rc = lib().dppo_gemm_nn_bf16(_ptr(A), A.stride(0), _ptr(B), B.stride(0), M, N, K, _ptr(C), C.stride(0), _ptr(status),
+                                     ctypes.byref(_opts(cta_group=cta_group, wait_limit_us=wait_limit_us, test_inject=test_inject)),
                                      c_void_p(st.cuda_stream))
     if rc != 0:
         raise DppoError(rc, "dppo_gemm_nn_bf16")
     return C, status
-
-
-def dppo_gemm_cta_group(cta_group=0):
-    """Sets the tensor-core GEMM's mode (2: pairs of SMs per 256 x 256 tile, the default; 1: single SMs); any other value
-    only queries.  Returns the previous setting."""
-    return int(lib().dppo_gemm_cta_group(int(cta_group)))
 
 
 STATIC_WS_MAX_ROWS = 65536
@@ -269,24 +277,25 @@ STATIC_WS_MAX_ROWS = 65536
 
 def dppo_loss_fwd_bwd_static_ws(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, K=0,
                                 delta=0.2, mu_topk_ids=None, mu_topk_p=None, loss_scale=0.0, dlogits_f32=False,
-                                kernel=KERNEL_AUTO, out=None, stream=None):
+                                kernel=KERNEL_AUTO, out=None, stream=None, is_cap=0.0, eps_low=0.0, given_divergence=None):
     """Calls ``dppo_loss_fwd_bwd_static_ws``: the same operation with the scratch taken from the array
     built into the library, for callers that cannot allocate device memory.  This wrapper does not
     allocate either when ``out`` holds the output tensors (loss[1], divergence[T], mask[T],
     dlogits[T,V], status[1], optionally stats[8]); without ``out`` it creates them with torch for
     convenience.  At most ``STATIC_WS_MAX_ROWS`` rows per call; calls that may overlap on the GPU race on
-    the shared array."""
+    the shared array.  ``given_divergence`` (variant GIVEN_D): without ``out`` it is copied into the new
+    divergence buffer; with ``out`` the caller fills ``out["divergence"]`` itself."""
     assert logits.is_cuda and logits.dim() == 2 and logits.stride(1) == 1
     T, V = logits.shape
     dev = logits.device
     if out is None:
         out = dict(loss=torch.empty(1, dtype=torch.float32, device=dev),
-                   divergence=torch.empty(T, dtype=torch.float32, device=dev),
+                   divergence=_divergence_buffer(T, dev, variant, given_divergence),
                    mask=torch.empty(T, dtype=torch.uint8, device=dev),
                    dlogits=torch.empty((T, V), dtype=torch.float32 if dlogits_f32 else logits.dtype, device=dev),
                    status=torch.zeros(1, dtype=torch.int32, device=dev), stats=None)
     dl = out["dlogits"]
-    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), 0.0, 0.0)
+    opts = _opts(loss_scale, dlogits_f32, kernel, is_cap, eps_low)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     with torch.cuda.device(dev):
         rc = lib().dppo_loss_fwd_bwd_static_ws(_ptr(logits), T, V, logits.stride(0) if T > 0 else V, _dtype_code(logits),
@@ -307,7 +316,7 @@ def dppo_host_staging_bytes(rows_per_chunk, V, K, logits_dtype, dlogits_f32=Fals
 
 def dppo_loss_fwd_bwd_host(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, K=0, delta=0.2,
                            mu_topk_ids=None, mu_topk_p=None, loss_scale=0.0, dlogits_f32=False, kernel=KERNEL_AUTO,
-                           rows_per_chunk=1024, staging=None, want_dlogits=False, device="cuda:0", out=None):
+                           rows_per_chunk=1024, staging=None, want_dlogits=False, device="cuda:0", out=None, is_cap=0.0, eps_low=0.0):
     """Calls ``dppo_loss_fwd_bwd_host`` on CPU tensors (pinned recommended); ``staging`` is a CUDA
     uint8 tensor of at least ``dppo_host_staging_bytes`` bytes (allocated here if None).  Returns
     dict(loss(float), divergence, mask, dlogits or None, status(int)) with host tensors."""
@@ -331,7 +340,7 @@ def dppo_loss_fwd_bwd_host(logits, sampled_ids, mu_logp, advantages, token_mask=
             dl = torch.empty((T, V), dtype=torch.float32 if dlogits_f32 else logits.dtype).pin_memory()
     loss = c_float(0.0)
     status = c_int32(0)
-    opts = DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), 0.0, 0.0)
+    opts = _opts(loss_scale, dlogits_f32, kernel, is_cap, eps_low)
     with torch.cuda.device(staging.device):
         rc = lib().dppo_loss_fwd_bwd_host(_ptr(logits), T, V, dt, _ptr(sampled_ids), _ptr(mu_logp), _ptr(mu_topk_ids),
                                           _ptr(mu_topk_p), _ptr(advantages), _ptr(token_mask), int(variant), int(K),

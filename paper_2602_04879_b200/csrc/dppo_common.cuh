@@ -14,13 +14,18 @@ namespace dppo {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr double kLn2 = 0.6931471805599453;
 
-// Header of the caller's workspace, written by the prelude kernel of each call.
+// Header of the caller's workspace, written by the prelude kernel of each call.  The accumulators are used by calls
+// that finish their rows block by block (the row-block mode of the fused variant): the loss reduction of every block
+// adds its rows to them, in stream order, and the last block writes the results.
 struct WsHeader {
   double scale;        // s of this call
   int n_valid;         // rows with a non-zero token_mask byte
-  int pad[13];
+  int pad0;
+  double acc[6];       // loss, sum D, sum |pi(a) - mu(a)|, sum r, sum |loss term|, blocked rows
+  float max_d;
+  int pad1[15];
 };
-static_assert(sizeof(WsHeader) == 64, "WsHeader layout");
+static_assert(sizeof(WsHeader) == 128, "WsHeader layout");
 
 struct RowParams {
   const void* logits;
@@ -36,6 +41,8 @@ struct RowParams {
   float loss_scale;          // > 0: caller's s
   float is_cap;              // C of Eq. unified_grad (<= 0 or inf: none)
   float eps_low;             // lower clip range of DPPO_PPO_CLIP (<= 0: delta)
+  unsigned long long wait_ns;  // limit of every on-chip wait
+  int inject;                // opts->test_inject
   void* dlogits;
   int64_t ld_out;
   float* divergence;
@@ -91,14 +98,29 @@ __device__ __forceinline__ double xlogx_over_y(double x, double y) {
   return x * (log(x) - log(y));
 }
 
+// Log-sum-exp of a row from the sum over all entries but the sampled one, kept apart so that 1 - pi(a) stays
+// accurate to the relative precision of that sum when pi(a) is close to 1 (1 - exp(z_a - lse) would cancel):
+//   m_o, S_o   maximum and sum of exp(z_j - m_o) over j != a (m_o = -inf, S_o = 0 if there is no such mass)
+//   z_a        the sampled token's logit
+// Gives lse over the whole row and log_other = log sum_{j != a} exp(z_j), so that log(1 - pi(a)) = log_other - lse.
+__device__ __forceinline__ void combine_lse(double m_o, double S_o, double z_a, double& lse, double& log_other) {
+  const bool have_o = (S_o > 0.0) || (S_o != S_o);         // a NaN sum (a NaN logit) is carried into lse
+  log_other = have_o ? m_o + log(S_o) : -INFINITY;
+  if (z_a != z_a) { lse = NAN; return; }
+  const double M = fmax(have_o ? m_o : -INFINITY, z_a);
+  if (M == -INFINITY || M == INFINITY) { lse = M; return; }   // no mass at all / an infinite logit: not finite, the caller reports it
+  lse = M + log((have_o ? S_o * exp(m_o - M) : 0.0) + exp(z_a - M));
+}
+
 // Per-row scalar stage, run by ONE full warp (all 32 lanes call it with the same arguments).
 //   lse        log-sum-exp of the row (double, from fp32 partial sums)
+//   log_other  log of the sum of exp(z_j) over j != a (see combine_lse)
 //   z_at(id, k)  fp32 value of this row's logit `id`; k is its position in the top-K list, -1 for the sampled id
 //   list_at(k, id, pm)  entry k of the row's top-K list (id and rollout probability); a caller that fetched the list
 //                earlier hands it over here, the default reads it from global memory
 // Returns on every lane the same values.  `flags` receives DPPO_STATUS_* bits found here.
 template <typename ZAt, typename ListAt>
-__device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, int a, double lse, double scale,
+__device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, int a, double lse, double log_other, double scale,
                                                  ZAt z_at, ListAt list_at, float& D_out, int& M_out, double& g_out,
                                                  float& r_out, float& absdiff_out, double& pi_a_out, int& flags) {
   const int lane = threadIdx.x & 31;
@@ -123,12 +145,18 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
     D = fabs(mu_a - pi_a);                            // Eq. binary_tv
   } else if (p.variant == DPPO_BINARY_KL) {           // Eq. binary_kl
     double first = (mu_a > 0.0) ? mu_a * (mu_logp - lpa) : 0.0;
-    D = first + xlogx_over_y(-expm1(mu_logp), -expm1(lpa));
+    // (1 - mu(a)) log((1 - mu(a)) / (1 - pi(a))) with log(1 - pi(a)) = log_other - lse
+    const double om_a = -expm1(mu_logp);
+    double second = 0.0;
+    if (om_a > 0.0) second = (log_other == -INFINITY) ? INFINITY : om_a * (log(om_a) - (log_other - lse));
+    D = first + second;
   } else {
     // Reduced categorical over set(top-K ids) u {a} u {other}  (Sec. 4.4, Eq. topk_tv / topk_kl)
     // per list entry in fp32 (log pi from the double lse, then expf / logf: relative error ~1e-7, two orders below the
     // tolerance of D); the lane's partial sums go to double for the reduction across the warp
-    float l_mu = 0.f, l_pi = 0.f, l_tv = 0.f, l_kl = 0.f;
+    // (the two mass sums in double: a lane may hold a probability close to 1 next to a tiny one)
+    double l_mu = 0.0, l_pi = 0.0;
+    float l_tv = 0.f, l_kl = 0.f;
     int in_list = 0, bad = 0;
     for (int k = lane; k < p.K; k += 32) {
       int id;
@@ -137,28 +165,39 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
       if (id < 0 || (int64_t)id >= p.V) { bad = 1; continue; }
       const float lpk = (float)((double)z_at(id, k) - lse);
       const float pk = expf(lpk);
-      l_mu += pm;
-      l_pi += pk;
+      l_mu += (double)pm;
+      if (id != a) l_pi += (double)pk;                     // pi's mass on the list without the sampled token
       l_tv += fabsf(pm - pk);
       if (pm > 0.f) l_kl += pm * (logf(pm) - lpk);
       in_list |= (id == a);
     }
-    double sum_mu = warp_sum((double)l_mu), sum_pi = warp_sum((double)l_pi), tv = warp_sum((double)l_tv), kl = warp_sum((double)l_kl);
+    double sum_mu = warp_sum(l_mu), sum_pi = warp_sum(l_pi), tv = warp_sum((double)l_tv), kl = warp_sum((double)l_kl);
     in_list = __any_sync(0xffffffffu, in_list);
     bad = __any_sync(0xffffffffu, bad);
     if (bad) flags |= DPPO_STATUS_BAD_TOPK_ID;
     if (!in_list) {
       sum_mu += mu_a;
-      sum_pi += pi_a;
       tv += fabs(mu_a - pi_a);
       if (mu_a > 0.0) kl += mu_a * (mu_logp - lpa);
     }
-    double om = 0.0, op = 0.0;                         // "other" bucket; empty when the set is the vocabulary
+    double om = 0.0, op = 0.0, op_raw = 0.0;           // "other" bucket; empty when the set is the vocabulary
     if ((int64_t)p.K + (in_list ? 0 : 1) < p.V) {
       om = fmin(1.0, fmax(0.0, 1.0 - sum_mu));
-      op = fmin(1.0, fmax(0.0, 1.0 - sum_pi));
+      // 1 - sum of pi over the set = (1 - pi(a)) - pi's mass on the rest of the list, with 1 - pi(a) taken from the
+      // sum over the other entries (no cancellation when pi(a) is close to 1)
+      op_raw = exp(log_other - lse) - sum_pi;
+      op = fmin(1.0, fmax(0.0, op_raw));
     }
-    D = (p.variant == DPPO_TOPK_TV) ? 0.5 * (tv + fabs(om - op)) : kl + xlogx_over_y(om, op);
+    if (p.variant == DPPO_TOPK_TV) {
+      D = 0.5 * (tv + fabs(om - op));
+    } else {
+      // When a token of the list other than the sampled one holds nearly all of pi's mass, the difference above is
+      // below what a normaliser summed in fp32 resolves (about 1e-7 absolute) and may come out as zero or negative while
+      // the rollout's own remainder is just as small: that is rounding, not a token that pi excludes, and the bucket's
+      // term, at most of the order of that remainder, is then left out instead of being reported as +inf.
+      const bool unresolved = (op_raw <= 0.0) && (op_raw > -1e-5) && (om < 1e-5);
+      D = kl + (unresolved ? 0.0 : xlogx_over_y(om, op));
+    }
   }
   // Eq. dppo_obj: blocked iff D > delta and the ratio already left 1 on the side the advantage pushes.
   const bool away = (adv > 0.0 && lpa > mu_logp) || (adv < 0.0 && lpa < mu_logp);
@@ -174,13 +213,13 @@ __device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, 
 }
 
 template <typename ZAt>
-__device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, int a, double lse, double scale,
+__device__ __forceinline__ void row_scalars_warp(const RowParams& p, int64_t t, int a, double lse, double log_other, double scale,
                                                  ZAt z_at, float& D_out, int& M_out, double& g_out,
                                                  float& r_out, float& absdiff_out, double& pi_a_out, int& flags) {
   const int32_t* ids = p.topk_ids + t * (int64_t)p.K;
   const float* ps = p.topk_p + t * (int64_t)p.K;
   auto list_at = [&](int k, int& id, float& pm) { id = ids[k]; pm = ps[k]; };
-  row_scalars_warp(p, t, a, lse, scale, z_at, list_at, D_out, M_out, g_out, r_out, absdiff_out, pi_a_out, flags);
+  row_scalars_warp(p, t, a, lse, log_other, scale, z_at, list_at, D_out, M_out, g_out, r_out, absdiff_out, pi_a_out, flags);
 }
 
 // Turns g, lse into the coefficients of the gradient sweep.
@@ -199,11 +238,11 @@ __device__ __forceinline__ RowCoef make_coef(double g, double lse, double pi_a) 
 
 // Launchers implemented in the kernel files.
 cudaError_t launch_prelude(const RowParams& p, cudaStream_t st);
-cudaError_t launch_finalize(const RowParams& p, cudaStream_t st);
+// block_first / block_last: position of these rows in a call that finishes its rows block by block (both true: the
+// whole call at once); the totals of earlier blocks wait in the workspace header
+cudaError_t launch_finalize(const RowParams& p, cudaStream_t st, bool block_first = true, bool block_last = true);
 cudaError_t launch_generic(const RowParams& p, int in_dtype, int out_dtype, cudaStream_t st);
 cudaError_t launch_ring(const RowParams& p, int in_dtype, int out_dtype, cudaStream_t st);
 bool ring_layout_ok(const RowParams& p, int in_dtype, int out_dtype);
-cudaError_t launch_scale(const RowParams& p, int in_dtype, int out_dtype, cudaStream_t st);
-bool scale_layout_ok(const RowParams& p, int in_dtype, int out_dtype);
 
 }  // namespace dppo

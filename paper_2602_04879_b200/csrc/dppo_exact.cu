@@ -22,8 +22,10 @@ struct ExactParams {
   const void* z; const void* zmu;
   int64_t T, V, ld_z, ld_mu;
   const uint8_t* token_mask;
-  float* tv; float* kl; float* entropy;
+  float* tv; float* kl; float* entropy;      // tv may be null: no second sweep
   int32_t* status;
+  unsigned long long wait_ns;
+  int inject;
 };
 
 // running (max, sum e^(x-max), sum e^(x-max) * w): rescaled when the maximum moves
@@ -209,7 +211,7 @@ __global__ void __launch_bounds__(kThreads, 1) dppo_exact_kernel(ExactParams p, 
   const InT* ZM = reinterpret_cast<const InT*>(p.zmu);
   for (int64_t t = blockIdx.x; t < p.T; t += gridDim.x) {
     if (p.token_mask && p.token_mask[t] == 0) {
-      if (tid == 0) { p.tv[t] = 0.f; p.kl[t] = 0.f; p.entropy[t] = 0.f; }
+      if (tid == 0) { if (p.tv) p.tv[t] = 0.f; p.kl[t] = 0.f; p.entropy[t] = 0.f; }
       continue;
     }
     const InT* z = Z + t * p.ld_z;
@@ -265,13 +267,14 @@ __global__ void __launch_bounds__(kThreads, 1) dppo_exact_kernel(ExactParams p, 
           p.entropy[t] = (float)(lse_p - Ap / Sp);
           p.kl[t] = kl_out(Bq / Sq - lse_q + lse_p);
         } else {
-          p.entropy[t] = 0.f; p.kl[t] = 0.f; p.tv[t] = 0.f;
+          p.entropy[t] = 0.f; p.kl[t] = 0.f;
+          if (p.tv) p.tv[t] = 0.f;
           atomicOr(p.status, DPPO_STATUS_NONFINITE_ROW);
         }
       }
     }
     __syncthreads();
-    if (s_bad) { __syncthreads(); continue; }
+    if (s_bad || !p.tv) { __syncthreads(); continue; }
     // ---- sweep 2: total variation with both normalisers known
     const float cp = -s_lse[0] * kLog2e, cq = -s_lse[1] * kLog2e;
     float acc = 0.f;
@@ -315,13 +318,14 @@ constexpr int kXConsumers = 512;
 constexpr int kXWarps = kXConsumers / 32;
 constexpr int kXThreads = kXConsumers + 32;          // + producer warp
 constexpr int kXVec = kXChunk / 16 / kXConsumers;    // 16-byte vectors per thread per chunk and tensor
-constexpr int kXMiscBytes = 1024;
+constexpr int kXMiscBytes = 2048;
 static_assert(kXVec * kXConsumers * 16 == kXChunk, "chunk geometry");
 
 struct XMisc {
   unsigned long long full[kXSlots], empty[kXSlots];
   unsigned long long red[2];             // all consumer warps have posted their partials (sweep 1 / sweep 2)
-  Acc3 pi[kXWarps], mu[kXWarps];
+  Acc3 pi[2][kXWarps], mu[2][kXWarps];   // per-warp partials of a row, two rows deep: without a second sweep a warp may post
+                                          // the next row's partials while another still reads this row's
   double tv[kXWarps];
   int abort_flag;
 };
@@ -357,7 +361,8 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
   XMisc* misc = reinterpret_cast<XMisc*>(smem + (size_t)kXSlots * 2 * kXChunk);
   const uint32_t slots_base = smem_u32(smem);
   const uint32_t full_base = smem_u32(&misc->full[0]), empty_base = smem_u32(&misc->empty[0]), red_base = smem_u32(&misc->red[0]);
-  volatile int* abort_flag = &misc->abort_flag;
+  const WaitCtl wc{&misc->abort_flag, p.wait_ns};
+  const int passes = p.tv ? 2 : 1;          // without a TV output the rows are read once
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     for (int i = 0; i < kXSlots; ++i) { mbar_init(full_base + 8u * i, 1); mbar_init(empty_base + 8u * i, kXWarps); }
@@ -375,7 +380,8 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
 
   if (warp == kXWarps) {
     // ------------------------------------------------------------------ producer (one lane)
-    if (lane == 0) {
+    // (test injection: the producer issues nothing, so that every consumer wait of the CTA runs out)
+    if (lane == 0 && !(p.inject & DPPO_INJECT_NO_COPIES)) {
       uint64_t keep, drop;
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(drop));
@@ -385,22 +391,19 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
         if (p.token_mask && p.token_mask[t] == 0) continue;
         const char* z = reinterpret_cast<const char*>(Z + t * p.ld_z);
         const char* zm = reinterpret_cast<const char*>(ZM + t * p.ld_mu);
-        for (int pass = 0; pass < 2 && ok; ++pass) {
+        for (int pass = 0; pass < passes && ok; ++pass) {
+          const uint64_t policy = (pass + 1 < passes) ? keep : drop;      // kept in L2 only if it is read again
           for (int c = 0; c < C; ++c, ++it) {
             const uint32_t slot = it % kXSlots, use = it / kXSlots;
-            if (use > 0 && !mbar_wait(empty_base + 8u * slot, (use - 1u) & 1u, abort_flag)) { ok = false; break; }
+            if (use > 0 && !mbar_wait(empty_base + 8u * slot, (use - 1u) & 1u, wc)) { ok = false; break; }
             const uint32_t off = (uint32_t)c * kXChunk;
             const uint32_t bytes = (row_bytes - off) < (uint32_t)kXChunk ? (row_bytes - off) : (uint32_t)kXChunk;
             const uint32_t bar = full_base + 8u * slot, dst = slots_base + slot * (2u * kXChunk);
             mbar_arrive_expect_tx(bar, 2u * bytes);
-            bulk_load(dst, z + off, bytes, bar, pass == 0 ? keep : drop);
-            bulk_load(dst + kXChunk, zm + off, bytes, bar, pass == 0 ? keep : drop);
+            bulk_load(dst, z + off, bytes, bar, policy);
+            bulk_load(dst + kXChunk, zm + off, bytes, bar, policy);
           }
         }
-      }
-      if (!ok) {      // gave up: let the copies still in flight land before this CTA's shared memory goes away
-        const unsigned long long t_exit = globaltimer_ns();
-        while (globaltimer_ns() - t_exit < 1000000ull) __nanosleep(1000);
       }
     }
   } else {
@@ -409,14 +412,14 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
     bool ok = true;
     for (int64_t t = blockIdx.x; t < p.T && ok; t += gridDim.x) {
       if (p.token_mask && p.token_mask[t] == 0) {
-        if (tid == 0) { p.tv[t] = 0.f; p.kl[t] = 0.f; p.entropy[t] = 0.f; }
+        if (tid == 0) { if (p.tv) p.tv[t] = 0.f; p.kl[t] = 0.f; p.entropy[t] = 0.f; }
         continue;
       }
       // ---- sweep 1
       Acc3 api{-INFINITY, 0.f, 0.f}, amu{-INFINITY, 0.f, 0.f};
       for (int c = 0; c < C && ok; ++c, ++it) {
         const uint32_t slot = it % kXSlots, use = it / kXSlots;
-        ok = mbar_wait_warp(full_base + 8u * slot, use & 1u, abort_flag);
+        ok = mbar_wait_warp(full_base + 8u * slot, use & 1u, wc);
         if (!ok) break;
         const uint32_t off = (uint32_t)c * kXChunk;
         const uint32_t nvec = ((row_bytes - off) < (uint32_t)kXChunk ? (row_bytes - off) : (uint32_t)kXChunk) / 16u;
@@ -454,12 +457,13 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
         api.merge(x);
         amu.merge(y);
       }
-      if (lane == 0) { misc->pi[warp] = api; misc->mu[warp] = amu; mbar_arrive(red_base); }
-      ok = mbar_wait_warp(red_base, nrow & 1u, abort_flag);
+      const uint32_t pb = nrow & 1u;
+      if (lane == 0) { misc->pi[pb][warp] = api; misc->mu[pb][warp] = amu; mbar_arrive(red_base); }
+      ok = mbar_wait_warp(red_base, nrow & 1u, wc);
       if (!ok) break;
       // every warp merges the warps' partials for itself (the same fp32 rule, the same order: identical results)
       Acc3 xp{-INFINITY, 0.f, 0.f}, xq{-INFINITY, 0.f, 0.f};
-      if (lane < kXWarps) { xp = misc->pi[lane]; xq = misc->mu[lane]; }
+      if (lane < kXWarps) { xp = misc->pi[pb][lane]; xq = misc->mu[pb][lane]; }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
         Acc3 x{__shfl_xor_sync(0xffffffffu, xp.m, o), __shfl_xor_sync(0xffffffffu, xp.s, o), __shfl_xor_sync(0xffffffffu, xp.a, o)};
@@ -478,12 +482,13 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
           atomicOr(p.status, DPPO_STATUS_NONFINITE_ROW);
         }
       }
+      if (passes == 1) { ++nrow; continue; }
       // ---- sweep 2 (a non-finite row still drains its chunks: the producer does not know)
       const float cp = -(float)lse_p * kLog2e, cq = -(float)lse_q * kLog2e;
       float acc = 0.f;
       for (int c = 0; c < C && ok; ++c, ++it) {
         const uint32_t slot = it % kXSlots, use = it / kXSlots;
-        ok = mbar_wait_warp(full_base + 8u * slot, use & 1u, abort_flag);
+        ok = mbar_wait_warp(full_base + 8u * slot, use & 1u, wc);
         if (!ok) break;
         const uint32_t off = (uint32_t)c * kXChunk;
         const uint32_t nvec = ((row_bytes - off) < (uint32_t)kXChunk ? (row_bytes - off) : (uint32_t)kXChunk) / 16u;
@@ -522,7 +527,7 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
       if (!ok) break;
       const double d = warp_sum((double)acc);
       if (lane == 0) { misc->tv[warp] = d; mbar_arrive(red_base + 8u); }
-      ok = mbar_wait_warp(red_base + 8u, nrow & 1u, abort_flag);
+      ok = mbar_wait_warp(red_base + 8u, nrow & 1u, wc);
       if (!ok) break;
       if (tid == 0) {
         double tot = 0;
@@ -533,7 +538,10 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
     }
   }
   __syncwarp();
-  if (*abort_flag && lane == 0) atomicOr(p.status, DPPO_STATUS_WAIT_LIMIT);
+  if (wc.aborted()) {      // every warp stays until copies that may still be in flight have landed
+    if (lane == 0) atomicOr(p.status, DPPO_STATUS_WAIT_LIMIT);
+    drain_after_abort();
+  }
 }
 
 }  // namespace
@@ -542,17 +550,18 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
 extern "C" int dppo_exact_divergence(const void* logits, const void* mu_logits, int64_t T, int64_t V,
                                      int64_t logits_row_stride, int64_t mu_row_stride, int dtype,
                                      const uint8_t* token_mask, float* tv, float* kl, float* entropy,
-                                     int32_t* status, void* cuda_stream) {
+                                     int32_t* status, const dppo_opts* opts, void* cuda_stream) {
   using namespace dppo;
   if (T < 0 || V < 1) return DPPO_ERR_SHAPE;
   if (dtype != DPPO_F32 && dtype != DPPO_BF16) return DPPO_ERR_DTYPE;
   if (!status) return DPPO_ERR_NULL;
-  if (T > 0 && (!logits || !mu_logits || !tv || !kl || !entropy)) return DPPO_ERR_NULL;
+  if (T > 0 && (!logits || !mu_logits || !kl || !entropy)) return DPPO_ERR_NULL;
   if (logits_row_stride < V || mu_row_stride < V) return DPPO_ERR_STRIDE;
   const size_t esz = dtype == DPPO_BF16 ? 2 : 4;
   if (((uintptr_t)logits % esz) || ((uintptr_t)mu_logits % esz)) return DPPO_ERR_ALIGN;
   if (T == 0) return DPPO_OK;
-  ExactParams p = {logits, mu_logits, T, V, logits_row_stride, mu_row_stride, token_mask, tv, kl, entropy, status};
+  ExactParams p = {logits, mu_logits, T, V, logits_row_stride, mu_row_stride, token_mask, tv, kl, entropy, status,
+                   wait_limit_ns(opts ? opts->wait_limit_us : 0), opts ? opts->test_inject : 0};
   const int vec_ok = ((uintptr_t)logits % 16 == 0) && ((uintptr_t)mu_logits % 16 == 0) &&
                      ((logits_row_stride * esz) % 16 == 0) && ((mu_row_stride * esz) % 16 == 0);
   int dev = 0, sms = 148;

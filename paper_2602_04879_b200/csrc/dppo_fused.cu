@@ -24,7 +24,6 @@
 // dHidden and dW are d = thousands of columns wide, far more than the 512 accumulator columns of tensor memory, so they
 // cannot be accumulated on chip across the vocabulary; the bf16 exponentials E (not the logits) are therefore staged in
 // the caller's workspace between steps 3 and 6/7.
-#include <atomic>
 #include <mutex>
 
 #include "dppo_common.cuh"
@@ -65,9 +64,6 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 1: one CTA per tile (cta_group::1); 2: pairs of CTAs per 256 x 256 tile (cta_group::2).  Set by dppo_gemm_cta_group.
-std::atomic<int> g_cta_group{2};
-
 template <int EPI, bool B_MN, int CG>
 cudaError_t launch_gemm_cg(const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
   using C = gemm::Cfg<CG>;
@@ -105,12 +101,28 @@ cudaError_t launch_gemm_cg(const void* A, int64_t lda, const void* B, int64_t ld
   return cudaLaunchKernelEx(&cfg, kernel, ma, mb, p);
 }
 
+// What every GEMM launch of a call takes from the caller's options.
+struct GemmOpts {
+  int cta_group;                 // 1: one CTA per 128 x 256 tile (cta_group::1); 2: pairs of CTAs per 256 x 256 tile (cta_group::2)
+  unsigned long long wait_ns;
+  int inject;
+};
+GemmOpts gemm_opts(const dppo_opts& o) {
+  GemmOpts g;
+  g.cta_group = (o.gemm_cta_group == 1) ? 1 : 2;
+  g.wait_ns = wait_limit_ns(o.wait_limit_us);
+  g.inject = o.test_inject;
+  return g;
+}
+
 // B_MN = false: B is [N, K] with leading dimension ldb; B_MN = true: B is [K, N] with leading dimension ldb.
 template <int EPI, bool B_MN = false>
-cudaError_t launch_gemm(const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
+cudaError_t launch_gemm(const GemmOpts& go, const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
   if (p.M <= 0 || p.N <= 0 || p.K <= 0) return cudaSuccess;
-  return g_cta_group.load() == 2 ? launch_gemm_cg<EPI, B_MN, 2>(A, lda, B, ldb, p, st)
-                                 : launch_gemm_cg<EPI, B_MN, 1>(A, lda, B, ldb, p, st);
+  p.wait_ns = go.wait_ns;
+  p.inject = go.inject;
+  return go.cta_group == 2 ? launch_gemm_cg<EPI, B_MN, 2>(A, lda, B, ldb, p, st)
+                           : launch_gemm_cg<EPI, B_MN, 1>(A, lda, B, ldb, p, st);
 }
 
 // out[c, r] = scale[r] * in[r, c] for bf16 matrices (scale optional: rows at and beyond *n_live count as scale 0);
@@ -245,8 +257,11 @@ __global__ void __launch_bounds__(256) fused_topk_logits_kernel(const __nv_bfloa
 // Stable two-class partition of the rows (one block): idx = the rows of class 0 in order, then those of class 1;
 // pos[t] = the place of row t in idx, or -1 for dropped rows; n[0] = rows of class 0, n[1] = rows of both classes.
 //   flag given:  class 0 = rows with flag[t] != 0, everything else dropped
-//   otherwise:   class 0 = valid rows (token_mask byte non-zero, or no mask) with adv[t] != 0, class 1 = the other valid rows
+//   otherwise:   class 0 = valid rows (token_mask byte non-zero, or no mask) with adv[t] != 0, class 1 = the other valid rows;
+//                rows whose sampled id lies outside [0, V) are dropped (the scalar stage reports them): they must not get
+//                a row of exponentials, which would be taken against reference 0 and could overflow
 __global__ void __launch_bounds__(1024) fused_partition_rows_kernel(const uint8_t* mask8, const float* adv, const int32_t* flag,
+                                                                    const int32_t* ids, int64_t V,
                                                                     int64_t T, int32_t* idx, int32_t* pos, int32_t* n) {
   __shared__ int warp_tot[2][32];
   __shared__ int total[2];
@@ -256,6 +271,7 @@ __global__ void __launch_bounds__(1024) fused_partition_rows_kernel(const uint8_
   auto cls = [&](int64_t t) -> int {
     if (flag) return flag[t] != 0 ? 0 : -1;
     if (mask8 && mask8[t] == 0) return -1;
+    if (ids[t] < 0 || (int64_t)ids[t] >= V) return -1;
     return adv[t] != 0.f ? 0 : 1;
   };
   int cnt[2] = {0, 0};
@@ -309,7 +325,7 @@ __global__ void __launch_bounds__(256) fused_gather_rows_kernel(GatherArgs g) {
 
 // What the single-pass scalar stage adds to RowParams.
 struct ExpArgs {
-  const float* psum;        // [rows, tiles_n] partial sums of exp(z - c), packed row order
+  const float* psum;        // [rows, tiles_n] partial sums of exp(z - c) over the entries other than the sampled token's, packed row order
   int tiles_n;
   const float* z_a;         // [rows] z at the sampled id, packed row order
   const float* cref2;       // [rows] c in log2 units, packed row order
@@ -332,33 +348,35 @@ __global__ void __launch_bounds__(256) fused_scalar_exp_kernel(RowParams p, ExpA
   const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (t >= p.T) return;
   const double scale = p.hdr->scale;
-  const int64_t ts = (int64_t)x.pos[t];                 // < 0: token_mask says invalid
+  const int64_t ts = (int64_t)x.pos[t];                 // < 0: token_mask says invalid, or the sampled id is out of range
   bool valid = ts >= 0;
   int flags = 0, resc = 0;
   const int a = p.sampled_ids[t];
-  if (valid && (a < 0 || (int64_t)a >= p.V)) { valid = false; flags = DPPO_STATUS_BAD_SAMPLED_ID; }
+  if ((!p.token_mask || p.token_mask[t] != 0) && (a < 0 || (int64_t)a >= p.V)) { valid = false; flags = DPPO_STATUS_BAD_SAMPLED_ID; }
   float D = 0.f, r = 0.f, absdiff = 0.f, factor = 0.f;
   int M = 0;
   double g = 0.0;
   if (valid) {
-    double S = 0.0;
-    for (int i = lane; i < x.tiles_n; i += 32) S += (double)x.psum[ts * x.tiles_n + i];
-    S = warp_sum(S);
+    double S_o = 0.0;                                   // over the entries other than the sampled token's
+    for (int i = lane; i < x.tiles_n; i += 32) S_o += (double)x.psum[ts * x.tiles_n + i];
+    S_o = warp_sum(S_o);
+    const float za = x.z_a[ts];
+    const double S = S_o + exp2((double)za * (double)kLog2e - (double)x.cref2[ts]);
     if (!(S > 0.0) || !(S <= kMaxSafeSum)) {
       resc = 1;                                         // outputs of this row are written by the rescue pass
     } else {
       const double lse = ((double)x.cref2[ts] + log2(S)) / (double)kLog2e;
+      const double log_other = (S_o > 0.0) ? ((double)x.cref2[ts] + log2(S_o)) / (double)kLog2e : -INFINITY;
       double pi_a;
       int f2 = 0;
-      const float za = x.z_a[ts];
       const float* zk = x.z_topk ? x.z_topk + t * (int64_t)p.K : nullptr;
       auto z_at = [&](int, int k) { return k < 0 ? za : zk[k]; };   // sampled id, or position k of the top-K list
-      row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
+      row_scalars_warp(p, t, a, lse, log_other, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
       if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
       else if (g != 0.0) {
         factor = (float)(g / S);
-        // the sampled token's entry: g (pi_a - 1) = (g / S) (E_a - S)
-        if (lane == 0 && ts < (int64_t)*x.n_grad) x.E[ts * x.lde + a] = __float2bfloat16_rn((float)((pi_a - 1.0) * S));
+        // the sampled token's entry: g (pi_a - 1) = (g / S) (E_a - S) = -(g / S) S_o
+        if (lane == 0 && ts < (int64_t)*x.n_grad) x.E[ts * x.lde + a] = __float2bfloat16_rn((float)(-S_o));
       }
     }
   }
@@ -412,17 +430,18 @@ __global__ void __launch_bounds__(256) fused_scalar_rescue_kernel(RowParams p, R
     const float2 pr = x.part[ts * x.tiles_n + i];
     if (pr.y > 0.f || pr.y != pr.y) S += (double)pr.y * exp((double)pr.x - (double)mm);
   }
-  S = warp_sum(S);
-  const double lse = (double)mm + log(S);
+  S = warp_sum(S);                                       // over the entries other than the sampled token's
+  const float za = x.z_a[ts];
+  double lse, log_other;
+  combine_lse((double)mm, S, (double)za, lse, log_other);
   if (!isfinite(lse)) {
     flags |= DPPO_STATUS_NONFINITE_ROW;
   } else {
     double pi_a;
     int f2 = 0;
-    const float za = x.z_a[ts];
     const float* zk = x.z_topk ? x.z_topk + t * (int64_t)p.K : nullptr;
     auto z_at = [&](int, int k) { return k < 0 ? za : zk[k]; };
-    row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
+    row_scalars_warp(p, t, a, lse, log_other, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
     if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
     else coef = make_coef(g, lse, pi_a);
   }
@@ -483,9 +502,161 @@ FusedLayout fused_layout(int64_t T, int64_t d, int64_t V, int K) {
   L.rescue = take((size_t)T * 4);
   L.rmap = take((size_t)T * 4);
   L.counts = take(4 * sizeof(int32_t));
-  L.loss_ws = take(dppo_workspace_bytes(T));
+  L.loss_ws = take(dppo_workspace_bytes(T, V, K, 0));
   L.total = off;
   return L;
+}
+
+
+// Everything one call of the fused variant needs, for all of its row blocks.
+struct FusedCall {
+  const __nv_bfloat16* hidden;
+  const __nv_bfloat16* W;
+  int64_t T, d, V;
+  const int32_t* sampled_ids;
+  const float* mu_logp;
+  const int32_t* topk_ids;
+  const float* topk_p;
+  const float* adv;
+  const uint8_t* token_mask;
+  int variant, K;
+  float delta;
+  dppo_opts o;
+  float* loss;
+  float* divergence;
+  uint8_t* mask;
+  float* dHidden;
+  float* dW;
+  float* stats;
+  int32_t* status;
+  char* ws;
+  FusedLayout L;              // laid out for the rows of one block
+  const __nv_bfloat16* wt;    // rows of W^T (Top-K gather, reference logits), or null
+  cudaStream_t st;
+};
+
+// Steps 1-7 of the file header for the rows [r0, r0 + Tb) of the call.  The scale s and N_valid come from the prelude
+// over all rows of the call (already in the workspace header).  `first` / `last`: position of the block in the call;
+// the loss reduction adds the block's rows to the totals of the earlier blocks, and dW is overwritten by the first block
+// and added to by the later ones (same stream: a fixed order, the result does not depend on timing).
+int fused_rows(const FusedCall& c, int64_t r0, int64_t Tb, bool first, bool last) {
+  const FusedLayout& L = c.L;
+  const int64_t d = c.d, V = c.V;
+  const int K = c.K;
+  cudaStream_t st = c.st;
+  char* ws = c.ws;
+  const bool vd = (c.o.lm_head_layout == DPPO_LM_HEAD_VD);      // W and dW given as [V, d]
+  const GemmOpts go = gemm_opts(c.o);
+  const int32_t* ids_t = c.sampled_ids + r0;
+  const uint8_t* tok = c.token_mask ? c.token_mask + r0 : nullptr;
+  const int32_t* tk_ids = c.topk_ids ? c.topk_ids + r0 * K : nullptr;
+
+  RowParams p = {};
+  p.T = Tb; p.V = V; p.sampled_ids = ids_t; p.mu_logp = c.mu_logp + r0; p.adv = c.adv + r0; p.token_mask = tok;
+  p.variant = c.variant; p.K = K; p.topk_ids = tk_ids; p.topk_p = c.topk_p ? c.topk_p + r0 * K : nullptr;
+  p.delta = c.delta; p.loss_scale = c.o.loss_scale; p.is_cap = c.o.is_cap; p.eps_low = c.o.eps_low;
+  p.divergence = c.divergence + r0; p.mask = c.mask + r0; p.loss = c.loss; p.stats = c.stats; p.status = c.status;
+  char* lws = ws + L.loss_ws;
+  const size_t per = round_up((size_t)Tb * sizeof(float), kAlign);
+  p.hdr = reinterpret_cast<WsHeader*>(lws);
+  p.row_loss = reinterpret_cast<float*>(lws + kAlign);
+  p.row_r = reinterpret_cast<float*>(lws + kAlign + per);
+  p.row_absdiff = reinterpret_cast<float*>(lws + kAlign + 2 * per);
+
+#define DPPO_TRY(call) do { if ((call) != cudaSuccess) return DPPO_ERR_CUDA; } while (0)
+  auto F = [&](size_t off) { return reinterpret_cast<float*>(ws + off); };
+  auto I = [&](size_t off) { return reinterpret_cast<int32_t*>(ws + off); };
+  const __nv_bfloat16* hid = c.hidden + r0 * d;
+  const __nv_bfloat16* Wb = c.W;
+  __nv_bfloat16* hc = reinterpret_cast<__nv_bfloat16*>(ws + L.hc);
+  __nv_bfloat16* E = reinterpret_cast<__nv_bfloat16*>(ws + L.E);
+  int32_t* counts = I(L.counts);
+  const int32_t *n_grad = counts, *n_valid = counts + 1, *n_resc = counts + 2;
+  const unsigned row_warps = (unsigned)((Tb + 7) / 8);
+  const int T = (int)Tb;
+  // 1. rows with a gradient to come (valid, advantage not zero) first, then the other valid rows
+  fused_partition_rows_kernel<<<1, 1024, 0, st>>>(tok, c.adv + r0, nullptr, ids_t, V, Tb, I(L.idx), I(L.pos), counts);
+  DPPO_TRY(cudaGetLastError());
+  {
+    GatherArgs ga = {};
+    ga.idx = I(L.idx); ga.n = n_valid; ga.d = d; ga.src = hid; ga.dst = hc; ga.ids_in = ids_t; ga.ids_out = I(L.ids_c);
+    ga.zero_fill = 1;
+    fused_gather_rows_kernel<<<(unsigned)Tb, 256, 0, st>>>(ga);
+    DPPO_TRY(cudaGetLastError());
+  }
+  // 2. reference exponent of every packed row
+  if (c.wt)      // W^T is there: contiguous rows instead of strided columns (rows past the valid ones are zero: reference 0)
+    fused_topk_logits_kernel<<<row_warps, 256, 0, st>>>(hc, c.wt, Tb, d, V, I(L.ids_c), 1, F(L.cref2), kLog2e);
+  else
+    fused_ref_logit_kernel<<<row_warps, 256, 0, st>>>(hc, Wb, Tb, d, V, I(L.ids_c), n_valid, F(L.cref2));
+  DPPO_TRY(cudaGetLastError());
+  // 3. forward GEMM: exponentials, their sums, z at the sampled id
+  DPPO_TRY(cudaMemsetAsync(F(L.z_a), 0, (size_t)Tb * 4, st));
+  gemm::Params g1 = {};
+  g1.M = T; g1.N = (int)V; g1.K = (int)d; g1.psum = F(L.psum); g1.z_a = F(L.z_a); g1.ids = I(L.ids_c); g1.cref2 = F(L.cref2);
+  g1.P = E; g1.ldp = L.lde; g1.status = c.status; g1.m_live = n_valid; g1.e_live = n_grad;
+  if (vd) DPPO_TRY((launch_gemm<gemm::EPI_EXP, false>(go, hc, d, Wb, d, g1, st)));     // B = W [V, d], K-major
+  else DPPO_TRY((launch_gemm<gemm::EPI_EXP, true>(go, hc, d, Wb, V, g1, st)));         // B = W [d, V], MN-major
+  // 4. per-row scalars
+  float* z_topk = nullptr;
+  if (K > 0) {      // logits at the rollout policy's top-K ids: T x K dot products against rows of W^T
+    z_topk = F(L.z_topk);
+    fused_topk_logits_kernel<<<(unsigned)((Tb * K + 7) / 8), 256, 0, st>>>(hid, c.wt, Tb, d, V, tk_ids, K, z_topk, 1.f);
+    DPPO_TRY(cudaGetLastError());
+  }
+  {
+    ExpArgs x = {};
+    x.psum = F(L.psum); x.tiles_n = L.tiles_n; x.z_a = F(L.z_a); x.cref2 = F(L.cref2); x.pos = I(L.pos); x.n_grad = n_grad;
+    x.z_topk = z_topk; x.row_factor = F(L.factor); x.rescue = I(L.rescue); x.E = E; x.lde = L.lde;
+    fused_scalar_exp_kernel<<<row_warps, 256, 0, st>>>(p, x);
+    DPPO_TRY(cudaGetLastError());
+  }
+  // 5. rescue pass over the rows flagged by the scalar kernel (normally none: the GEMMs then have no tile to process)
+  {
+    fused_partition_rows_kernel<<<1, 1024, 0, st>>>(nullptr, nullptr, I(L.rescue), nullptr, V, Tb, I(L.idx_r), I(L.pos_r), counts + 2);
+    DPPO_TRY(cudaGetLastError());
+    GatherArgs ga = {};
+    ga.idx = I(L.idx_r); ga.n = n_resc; ga.d = d; ga.src = hid; ga.dst = reinterpret_cast<__nv_bfloat16*>(ws + L.hr);
+    ga.ids_in = ids_t; ga.ids_out = I(L.ids_r); ga.zero_fill = 0;
+    fused_gather_rows_kernel<<<(unsigned)Tb, 256, 0, st>>>(ga);
+    DPPO_TRY(cudaGetLastError());
+    DPPO_TRY(cudaMemsetAsync(F(L.z_ar), 0, (size_t)Tb * 4, st));
+    gemm::Params gs = {};
+    gs.M = T; gs.N = (int)V; gs.K = (int)d; gs.part = reinterpret_cast<float2*>(ws + L.part); gs.z_a = F(L.z_ar);
+    gs.ids = I(L.ids_r); gs.status = c.status; gs.m_live = n_resc; gs.allow_empty = 1;
+    if (vd) DPPO_TRY((launch_gemm<gemm::EPI_STATS, false>(go, ws + L.hr, d, Wb, d, gs, st)));
+    else DPPO_TRY((launch_gemm<gemm::EPI_STATS, true>(go, ws + L.hr, d, Wb, V, gs, st)));
+    RescueArgs x = {};
+    x.rescue = I(L.rescue); x.pos_r = I(L.pos_r); x.pos_e = I(L.pos);
+    x.part = reinterpret_cast<const float2*>(ws + L.part); x.tiles_n = L.tiles_n; x.z_a = F(L.z_ar); x.z_topk = z_topk;
+    x.c2 = F(L.c2); x.sgn = F(L.sgn); x.fix = F(L.fix); x.p_row_map = I(L.rmap); x.row_factor = F(L.factor);
+    fused_scalar_rescue_kernel<<<row_warps, 256, 0, st>>>(p, x);
+    DPPO_TRY(cudaGetLastError());
+    gemm::Params gg = {};
+    gg.M = T; gg.N = (int)V; gg.K = (int)d; gg.ids = I(L.ids_r); gg.c2 = F(L.c2); gg.sgn = F(L.sgn); gg.fix = F(L.fix);
+    gg.P = E; gg.ldp = L.lde; gg.status = c.status; gg.m_live = n_resc; gg.allow_empty = 1; gg.p_row_map = I(L.rmap);
+    if (vd) DPPO_TRY((launch_gemm<gemm::EPI_GRAD, false>(go, ws + L.hr, d, Wb, d, gg, st)));
+    else DPPO_TRY((launch_gemm<gemm::EPI_GRAD, true>(go, ws + L.hr, d, Wb, V, gg, st)));
+  }
+  DPPO_TRY(launch_finalize(p, st, first, last));
+  // 6. dHidden[idx[i], :] = factor[i] * (E[i, :] . W[d, V]^T) for the rows with a gradient; the other rows stay zero.
+  //    Few output tiles, very long K: K is cut in two when that fills the waves better (two partial sums added into
+  //    zeros, in either order the same result).
+  gemm::Params g3 = {};
+  g3.M = T; g3.N = (int)d; g3.K = (int)V; g3.C = c.dHidden + r0 * d; g3.ldc = d; g3.status = c.status;
+  g3.m_live = n_grad; g3.row_map = I(L.idx); g3.row_scale = F(L.factor); g3.splits = -1;
+  g3.n_fastest = 1;      // d / 256 tiles along N: the CTAs of a wave then share each 2 V-byte row block of E instead of re-reading it
+  if (vd) DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(go, E, L.lde, Wb, d, g3, st)));     // B = W as [K = V, N = d], MN-major
+  else DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(go, E, L.lde, Wb, V, g3, st));                // B = W as [N = d, K = V], K-major
+  // 7. dW[d, V] (+)= (factor * packed hidden)^T[d, n_grad] . E[n_grad, V]
+  DPPO_TRY(transpose_bf16(hc, Tb, d, d, ws + L.ht, L.ldt, st, F(L.factor), n_grad));
+  gemm::Params g4 = {};
+  g4.M = (int)d; g4.N = (int)V; g4.K = T; g4.C = c.dW; g4.ldc = V; g4.status = c.status; g4.k_live = n_grad;
+  g4.accumulate = first ? 0 : 1;
+  if (vd) { g4.c_transposed = 1; g4.ldc = d; }      // the same product, stored as dW[V, d]
+  DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(go, ws + L.ht, L.ldt, E, L.lde, g4, st)));   // B = E [T, V], MN-major
+#undef DPPO_TRY
+  return DPPO_OK;
 }
 
 }  // namespace
@@ -498,36 +669,33 @@ size_t dppo_fused_workspace_bytes(int64_t T, int64_t d, int64_t V, int K) {
   return dppo::fused_layout(T, d, V, K).total;
 }
 
-int dppo_gemm_cta_group(int cta_group) {
-  const int prev = dppo::g_cta_group.load();
-  if (cta_group == 1 || cta_group == 2) dppo::g_cta_group.store(cta_group);
-  return prev;
+static int gemm_bf16_checked(bool b_mn, const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C,
+                             int64_t ldc, int32_t* status, const dppo_opts* opts, void* cuda_stream) {
+  if (M < 0 || N < 0 || K < 0) return DPPO_ERR_SHAPE;
+  if (M == 0 || N == 0) return DPPO_OK;
+  if (!A || !B || !C) return DPPO_ERR_NULL;
+  if (lda < K || ldb < (b_mn ? N : K) || ldc < N) return DPPO_ERR_STRIDE;
+  if (((uintptr_t)A % 16) || ((uintptr_t)B % 16) || (lda % 8) || (ldb % 8) || ((uintptr_t)C % 4)) return DPPO_ERR_ALIGN;
+  dppo_opts o = {};
+  if (opts) o = *opts;
+  if (o.gemm_cta_group < 0 || o.gemm_cta_group > 2 || o.wait_limit_us < 0) return DPPO_ERR_UNSUPPORTED;
+  dppo::gemm::Params p = {};
+  p.M = M; p.N = N; p.K = K; p.C = C; p.ldc = ldc; p.status = status;
+  const dppo::GemmOpts go = dppo::gemm_opts(o);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const cudaError_t e = b_mn ? dppo::launch_gemm<dppo::gemm::EPI_STORE_F32, true>(go, A, lda, B, ldb, p, st)
+                             : dppo::launch_gemm<dppo::gemm::EPI_STORE_F32, false>(go, A, lda, B, ldb, p, st);
+  return e == cudaSuccess ? DPPO_OK : DPPO_ERR_CUDA;
 }
 
 int dppo_gemm_tn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,
-                      int32_t* status, void* cuda_stream) {
-  if (M < 0 || N < 0 || K < 0) return DPPO_ERR_SHAPE;
-  if (M == 0 || N == 0) return DPPO_OK;
-  if (!A || !B || !C) return DPPO_ERR_NULL;
-  if (lda < K || ldb < K || ldc < N) return DPPO_ERR_STRIDE;
-  if (((uintptr_t)A % 16) || ((uintptr_t)B % 16) || (lda % 8) || (ldb % 8) || ((uintptr_t)C % 4)) return DPPO_ERR_ALIGN;
-  dppo::gemm::Params p = {};
-  p.M = M; p.N = N; p.K = K; p.C = C; p.ldc = ldc; p.status = status;
-  return dppo::launch_gemm<dppo::gemm::EPI_STORE_F32>(A, lda, B, ldb, p, reinterpret_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
-             ? DPPO_OK : DPPO_ERR_CUDA;
+                      int32_t* status, const dppo_opts* opts, void* cuda_stream) {
+  return gemm_bf16_checked(false, A, lda, B, ldb, M, N, K, C, ldc, status, opts, cuda_stream);
 }
 
 int dppo_gemm_nn_bf16(const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K, float* C, int64_t ldc,
-                      int32_t* status, void* cuda_stream) {
-  if (M < 0 || N < 0 || K < 0) return DPPO_ERR_SHAPE;
-  if (M == 0 || N == 0) return DPPO_OK;
-  if (!A || !B || !C) return DPPO_ERR_NULL;
-  if (lda < K || ldb < N || ldc < N) return DPPO_ERR_STRIDE;
-  if (((uintptr_t)A % 16) || ((uintptr_t)B % 16) || (lda % 8) || (ldb % 8) || ((uintptr_t)C % 4)) return DPPO_ERR_ALIGN;
-  dppo::gemm::Params p = {};
-  p.M = M; p.N = N; p.K = K; p.C = C; p.ldc = ldc; p.status = status;
-  return dppo::launch_gemm<dppo::gemm::EPI_STORE_F32, true>(A, lda, B, ldb, p, reinterpret_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
-             ? DPPO_OK : DPPO_ERR_CUDA;
+                      int32_t* status, const dppo_opts* opts, void* cuda_stream) {
+  return gemm_bf16_checked(true, A, lda, B, ldb, M, N, K, C, ldc, status, opts, cuda_stream);
 }
 
 int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int64_t d, int64_t V,
@@ -550,126 +718,44 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   if (((uintptr_t)hidden % 16) || ((uintptr_t)W % 16) || (d % 8) || (V % 8)) return DPPO_ERR_ALIGN;
   if (((uintptr_t)dHidden % 16) || ((uintptr_t)dW % 16)) return DPPO_ERR_ALIGN;
   if (o.lm_head_layout != DPPO_LM_HEAD_DV && o.lm_head_layout != DPPO_LM_HEAD_VD) return DPPO_ERR_UNSUPPORTED;
-  const bool vd = (o.lm_head_layout == DPPO_LM_HEAD_VD);      // W and dW given as [V, d]
-  const FusedLayout L = fused_layout(T, d, V, K);
-  if (!workspace || ((uintptr_t)workspace % kAlign) || workspace_bytes < L.total) return DPPO_ERR_WORKSPACE;
+  if (o.gemm_cta_group < 0 || o.gemm_cta_group > 2 || o.wait_limit_us < 0 || o.fused_rows_per_block < 0) return DPPO_ERR_UNSUPPORTED;
+  const bool vd = (o.lm_head_layout == DPPO_LM_HEAD_VD);
+  // row-block mode: the rows are finished block by block and the workspace is sized for one block
+  const int64_t Tb_max = (o.fused_rows_per_block > 0 && (int64_t)o.fused_rows_per_block < T) ? (int64_t)o.fused_rows_per_block : T;
+  FusedCall c = {};
+  c.L = fused_layout(Tb_max, d, V, K);
+  if (!workspace || ((uintptr_t)workspace % kAlign) || workspace_bytes < c.L.total) return DPPO_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   char* ws = reinterpret_cast<char*>(workspace);
+  c.hidden = reinterpret_cast<const __nv_bfloat16*>(hidden); c.W = reinterpret_cast<const __nv_bfloat16*>(W);
+  c.T = T; c.d = d; c.V = V; c.sampled_ids = sampled_ids; c.mu_logp = mu_logp; c.topk_ids = mu_topk_ids; c.topk_p = mu_topk_p;
+  c.adv = advantages; c.token_mask = token_mask; c.variant = variant; c.K = K; c.delta = delta; c.o = o;
+  c.loss = loss; c.divergence = divergence; c.mask = mask; c.dHidden = dHidden; c.dW = dW; c.stats = stats; c.status = status;
+  c.ws = ws; c.st = st;
 
-  RowParams p = {};
-  p.T = T; p.V = V; p.sampled_ids = sampled_ids; p.mu_logp = mu_logp; p.adv = advantages; p.token_mask = token_mask;
-  p.variant = variant; p.K = K; p.topk_ids = mu_topk_ids; p.topk_p = mu_topk_p;
-  p.delta = delta; p.loss_scale = o.loss_scale; p.is_cap = o.is_cap; p.eps_low = o.eps_low;
-  p.divergence = divergence; p.mask = mask; p.loss = loss; p.stats = stats; p.status = status;
-  char* lws = ws + L.loss_ws;
-  const size_t per = round_up((size_t)T * sizeof(float), kAlign);
-  p.hdr = reinterpret_cast<WsHeader*>(lws);
-  p.row_loss = reinterpret_cast<float*>(lws + kAlign);
-  p.row_r = reinterpret_cast<float*>(lws + kAlign + per);
-  p.row_absdiff = reinterpret_cast<float*>(lws + kAlign + 2 * per);
-
-#define DPPO_TRY(call) do { if ((call) != cudaSuccess) return DPPO_ERR_CUDA; } while (0)
-  DPPO_TRY(launch_prelude(p, st));
+  // N_valid and the scale s over ALL rows of the call
+  RowParams p0 = {};
+  p0.T = T; p0.token_mask = token_mask; p0.loss_scale = o.loss_scale;
+  p0.hdr = reinterpret_cast<WsHeader*>(ws + c.L.loss_ws);
+  p0.loss = loss; p0.stats = stats; p0.status = status;
+  if (launch_prelude(p0, st) != cudaSuccess) return DPPO_ERR_CUDA;
   // dW is written by a GEMM whose K dimension is T: with no rows it is all zero
   if (T == 0) {
-    DPPO_TRY(cudaMemsetAsync(dW, 0, (size_t)d * V * sizeof(float), st));
-    DPPO_TRY(launch_finalize(p, st));
-    return DPPO_OK;
+    if (cudaMemsetAsync(dW, 0, (size_t)d * V * sizeof(float), st) != cudaSuccess) return DPPO_ERR_CUDA;
+    return launch_finalize(p0, st) == cudaSuccess ? DPPO_OK : DPPO_ERR_CUDA;
   }
-  auto F = [&](size_t off) { return reinterpret_cast<float*>(ws + off); };
-  auto I = [&](size_t off) { return reinterpret_cast<int32_t*>(ws + off); };
-  const __nv_bfloat16* hid = reinterpret_cast<const __nv_bfloat16*>(hidden);
-  const __nv_bfloat16* Wb = reinterpret_cast<const __nv_bfloat16*>(W);
-  __nv_bfloat16* hc = reinterpret_cast<__nv_bfloat16*>(ws + L.hc);
-  __nv_bfloat16* E = reinterpret_cast<__nv_bfloat16*>(ws + L.E);
-  int32_t* counts = I(L.counts);
-  const int32_t *n_grad = counts, *n_valid = counts + 1, *n_resc = counts + 2;
-  const unsigned row_warps = (unsigned)((T + 7) / 8);
-  // 1. rows with a gradient to come (valid, advantage not zero) first, then the other valid rows; W^T for the Top-K gather
-  // rows of W^T for the gather dot products: W itself when it is stored [V, d]
-  const __nv_bfloat16* wt = vd ? Wb : reinterpret_cast<const __nv_bfloat16*>(ws + L.wt);
-  if (K > 0 && !vd) DPPO_TRY(transpose_bf16(W, d, V, V, ws + L.wt, d, st));
-  fused_partition_rows_kernel<<<1, 1024, 0, st>>>(token_mask, advantages, nullptr, T, I(L.idx), I(L.pos), counts);
-  DPPO_TRY(cudaGetLastError());
-  {
-    GatherArgs ga = {};
-    ga.idx = I(L.idx); ga.n = n_valid; ga.d = d; ga.src = hid; ga.dst = hc; ga.ids_in = sampled_ids; ga.ids_out = I(L.ids_c);
-    ga.zero_fill = 1;
-    fused_gather_rows_kernel<<<(unsigned)T, 256, 0, st>>>(ga);
-    DPPO_TRY(cudaGetLastError());
+  // rows of W^T for the gather dot products: W itself when it is stored [V, d]; otherwise a transposed copy, made once
+  // per call, when the Top-K lists need it
+  c.wt = vd ? c.W : nullptr;
+  if (K > 0 && !vd) {
+    if (transpose_bf16(W, d, V, V, ws + c.L.wt, d, st) != cudaSuccess) return DPPO_ERR_CUDA;
+    c.wt = reinterpret_cast<const __nv_bfloat16*>(ws + c.L.wt);
   }
-  // 2. reference exponent of every packed row
-  if (K > 0 || vd)      // W^T is there: contiguous rows instead of strided columns (rows past the valid ones are zero: reference 0)
-    fused_topk_logits_kernel<<<row_warps, 256, 0, st>>>(hc, wt, T, d, V, I(L.ids_c), 1, F(L.cref2), kLog2e);
-  else
-    fused_ref_logit_kernel<<<row_warps, 256, 0, st>>>(hc, Wb, T, d, V, I(L.ids_c), n_valid, F(L.cref2));
-  DPPO_TRY(cudaGetLastError());
-  // 3. forward GEMM: exponentials, their sums, z at the sampled id
-  DPPO_TRY(cudaMemsetAsync(F(L.z_a), 0, (size_t)T * 4, st));
-  gemm::Params g1 = {};
-  g1.M = (int)T; g1.N = (int)V; g1.K = (int)d; g1.psum = F(L.psum); g1.z_a = F(L.z_a); g1.ids = I(L.ids_c); g1.cref2 = F(L.cref2);
-  g1.P = E; g1.ldp = L.lde; g1.status = status; g1.m_live = n_valid; g1.e_live = n_grad;
-  if (vd) DPPO_TRY((launch_gemm<gemm::EPI_EXP, false>(hc, d, W, d, g1, st)));     // B = W [V, d], K-major
-  else DPPO_TRY((launch_gemm<gemm::EPI_EXP, true>(hc, d, W, V, g1, st)));         // B = W [d, V], MN-major
-  // 4. per-row scalars
-  float* z_topk = nullptr;
-  if (K > 0) {      // logits at the rollout policy's top-K ids: T x K dot products against rows of W^T
-    z_topk = F(L.z_topk);
-    fused_topk_logits_kernel<<<(unsigned)((T * K + 7) / 8), 256, 0, st>>>(
-        hid, wt, T, d, V, mu_topk_ids, K, z_topk, 1.f);
-    DPPO_TRY(cudaGetLastError());
+  for (int64_t r0 = 0; r0 < T; r0 += Tb_max) {
+    const int64_t Tb = (T - r0 < Tb_max) ? (T - r0) : Tb_max;
+    const int rc = fused_rows(c, r0, Tb, r0 == 0, r0 + Tb >= T);
+    if (rc != DPPO_OK) return rc;
   }
-  {
-    ExpArgs x = {};
-    x.psum = F(L.psum); x.tiles_n = L.tiles_n; x.z_a = F(L.z_a); x.cref2 = F(L.cref2); x.pos = I(L.pos); x.n_grad = n_grad;
-    x.z_topk = z_topk; x.row_factor = F(L.factor); x.rescue = I(L.rescue); x.E = E; x.lde = L.lde;
-    fused_scalar_exp_kernel<<<row_warps, 256, 0, st>>>(p, x);
-    DPPO_TRY(cudaGetLastError());
-  }
-  // 5. rescue pass over the rows flagged by the scalar kernel (normally none: the GEMMs then have no tile to process)
-  {
-    fused_partition_rows_kernel<<<1, 1024, 0, st>>>(nullptr, nullptr, I(L.rescue), T, I(L.idx_r), I(L.pos_r), counts + 2);
-    DPPO_TRY(cudaGetLastError());
-    GatherArgs ga = {};
-    ga.idx = I(L.idx_r); ga.n = n_resc; ga.d = d; ga.src = hid; ga.dst = reinterpret_cast<__nv_bfloat16*>(ws + L.hr);
-    ga.ids_in = sampled_ids; ga.ids_out = I(L.ids_r); ga.zero_fill = 0;
-    fused_gather_rows_kernel<<<(unsigned)T, 256, 0, st>>>(ga);
-    DPPO_TRY(cudaGetLastError());
-    DPPO_TRY(cudaMemsetAsync(F(L.z_ar), 0, (size_t)T * 4, st));
-    gemm::Params gs = {};
-    gs.M = (int)T; gs.N = (int)V; gs.K = (int)d; gs.part = reinterpret_cast<float2*>(ws + L.part); gs.z_a = F(L.z_ar);
-    gs.ids = I(L.ids_r); gs.status = status; gs.m_live = n_resc; gs.allow_empty = 1;
-    if (vd) DPPO_TRY((launch_gemm<gemm::EPI_STATS, false>(ws + L.hr, d, W, d, gs, st)));
-    else DPPO_TRY((launch_gemm<gemm::EPI_STATS, true>(ws + L.hr, d, W, V, gs, st)));
-    RescueArgs x = {};
-    x.rescue = I(L.rescue); x.pos_r = I(L.pos_r); x.pos_e = I(L.pos);
-    x.part = reinterpret_cast<const float2*>(ws + L.part); x.tiles_n = L.tiles_n; x.z_a = F(L.z_ar); x.z_topk = z_topk;
-    x.c2 = F(L.c2); x.sgn = F(L.sgn); x.fix = F(L.fix); x.p_row_map = I(L.rmap); x.row_factor = F(L.factor);
-    fused_scalar_rescue_kernel<<<row_warps, 256, 0, st>>>(p, x);
-    DPPO_TRY(cudaGetLastError());
-    gemm::Params gg = {};
-    gg.M = (int)T; gg.N = (int)V; gg.K = (int)d; gg.ids = I(L.ids_r); gg.c2 = F(L.c2); gg.sgn = F(L.sgn); gg.fix = F(L.fix);
-    gg.P = E; gg.ldp = L.lde; gg.status = status; gg.m_live = n_resc; gg.allow_empty = 1; gg.p_row_map = I(L.rmap);
-    if (vd) DPPO_TRY((launch_gemm<gemm::EPI_GRAD, false>(ws + L.hr, d, W, d, gg, st)));
-    else DPPO_TRY((launch_gemm<gemm::EPI_GRAD, true>(ws + L.hr, d, W, V, gg, st)));
-  }
-  DPPO_TRY(launch_finalize(p, st));
-  // 6. dHidden[idx[i], :] = factor[i] * (E[i, :] . W[d, V]^T) for the rows with a gradient; the other rows stay zero.
-  //    Few output tiles, very long K: K is cut in two when that fills the waves better (two partial sums added into
-  //    zeros, in either order the same result).
-  gemm::Params g3 = {};
-  g3.M = (int)T; g3.N = (int)d; g3.K = (int)V; g3.C = dHidden; g3.ldc = d; g3.status = status;
-  g3.m_live = n_grad; g3.row_map = I(L.idx); g3.row_scale = F(L.factor); g3.splits = -1;
-  g3.n_fastest = 1;      // d / 256 tiles along N: the CTAs of a wave then share each 2 V-byte row block of E instead of re-reading it
-  if (vd) DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(E, L.lde, W, d, g3, st)));     // B = W as [K = V, N = d], MN-major
-  else DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(E, L.lde, W, V, g3, st));                // B = W as [N = d, K = V], K-major
-  // 7. dW[d, V] = (factor * packed hidden)^T[d, n_grad] . E[n_grad, V]
-  DPPO_TRY(transpose_bf16(hc, T, d, d, ws + L.ht, L.ldt, st, F(L.factor), n_grad));
-  gemm::Params g4 = {};
-  g4.M = (int)d; g4.N = (int)V; g4.K = (int)T; g4.C = dW; g4.ldc = V; g4.status = status; g4.k_live = n_grad;
-  if (vd) { g4.c_transposed = 1; g4.ldc = d; }      // the same product, stored as dW[V, d]
-  DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(ws + L.ht, L.ldt, E, L.lde, g4, st)));   // B = E [T, V], MN-major
-#undef DPPO_TRY
   return DPPO_OK;
 }
 

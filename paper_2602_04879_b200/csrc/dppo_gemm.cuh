@@ -28,6 +28,7 @@
 #include <stdint.h>
 
 #include "../../include/dppo.h"
+#include "dppo_pipe.cuh"
 
 namespace dppo {
 namespace gemm {
@@ -88,42 +89,11 @@ struct Params {
   float* psum;           // [M, tiles_n]
   const int* e_live;     // rows of E that later steps read: rows below max(64, *e_live rounded up to 64) are written
   int32_t* status;
+  unsigned long long wait_ns;   // limit of every on-chip wait
+  int inject;            // opts->test_inject
+  int accumulate;        // EPI_STORE_F32 (no K split, no row map): the product is added to what C holds
 };
 
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void bar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void bar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool bar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long timer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait (about 2 s); false = gave up (abort flag set) or somebody else did.
-__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (bar_try(bar, parity)) return true;
-  const unsigned long long t0 = timer_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (bar_try(bar, parity)) return true;
-    if ((it & 0xff) == 0) {
-      if (*abort_flag) return false;
-      if (timer_ns() - t0 > 2000000000ull) { *abort_flag = 1; return false; }
-    }
-  }
-}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
@@ -228,28 +198,28 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   // 1024-byte alignment for the 128-byte swizzle atoms (the same offset in both CTAs of a pair)
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + STAGES * STAGE_BYTES);
-  const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + STAGES);
-  const uint32_t tfull0 = smem_addr(bars + 2 * STAGES), tempty0 = smem_addr(bars + 2 * STAGES + 2);
+  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
+  const uint32_t tfull0 = smem_u32(bars + 2 * STAGES), tempty0 = smem_u32(bars + 2 * STAGES + 2);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const WaitCtl wc{reinterpret_cast<volatile int*>(tmem_slot + 1), p.wait_ns};
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = (CG == 2) ? cluster_ctarank() : 0u;       // 0: leader of the pair
   const int group = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int ngroups = (CG == 2) ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
   if (tid == 0) {
-    for (int i = 0; i < STAGES; ++i) { bar_init(full0 + 8 * i, 1); bar_init(empty0 + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) { bar_init(tfull0 + 8 * i, 1); bar_init(tempty0 + 8 * i, 4 * CG); }
-    *abort_flag = 0;
+    for (int i = 0; i < STAGES; ++i) { mbar_init(full0 + 8 * i, 1); mbar_init(empty0 + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tfull0 + 8 * i, 1); mbar_init(tempty0 + 8 * i, 4 * CG); }
+    *wc.flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {   // the MMA warp owns the tensor memory (in a pair: the same warp of both CTAs, together)
     if (CG == 2) {
-      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
       asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     } else {
-      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
       asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
   }
@@ -284,11 +254,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   }
   const int kper = (kblocks + splits - 1) / splits;
   const int nunits = ntiles * splits;
-  const uint32_t smem_base = smem_addr(smem);
+  const uint32_t smem_base = smem_u32(smem);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (of this CTA's operand slices)
-    if (lane == 0) {
+    // (test injection: the producer issues nothing, so that every consumer wait of the CTA runs out)
+    if (lane == 0 && !(p.inject & DPPO_INJECT_NO_COPIES)) {
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
@@ -298,13 +269,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
         const int m0 = tm * C::TILE_M + (int)rank * BM, n0 = tn * BN + (int)rank * C::B_COLS;
         const int kb0 = part * kper, kb1 = (kb0 + kper < kblocks) ? kb0 + kper : kblocks;
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!bar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, wc)) { ok = false; break; }
           const uint32_t a_dst = smem_base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
           if (CG == 2) {
             // both CTAs' bytes are counted on the leader's barrier (the leader may post its expectation after the
             // peer's bytes have begun to land: the phase cannot complete before the leader's own arrival)
             const uint32_t bar = map_to_cta(full0 + 8 * s, 0);
-            if (rank == 0) bar_expect_tx(full0 + 8 * s, 2 * STAGE_BYTES);
+            if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * s, 2 * STAGE_BYTES);
             tma_load_2d_pair(a_dst, &map_a, kb * BK, m0, bar);
             if (B_MN) {
 #pragma unroll
@@ -313,7 +284,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
               tma_load_2d_pair(b_dst, &map_b, kb * BK, n0, bar);
             }
           } else {
-            bar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+            mbar_arrive_expect_tx(full0 + 8 * s, STAGE_BYTES);
             tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
             if (B_MN) {
 #pragma unroll
@@ -324,10 +295,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
-      }
-      if (!ok) {      // gave up: let the copies still in flight land before this CTA's shared memory goes away
-        const unsigned long long t0 = timer_ns();
-        while (timer_ns() - t0 < 100000ull) { }
       }
     }
   } else if (warp == 1) {
@@ -342,11 +309,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
         const int part = u / ntiles;
         const int kb0 = part * kper, kb1 = (kb0 + kper < kblocks) ? kb0 + kper : kblocks;
         const uint32_t b = it & 1u, use = it >> 1;
-        if (!bar_wait(tempty0 + 8 * b, (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }   // epilogues drained this buffer
+        if (!mbar_wait(tempty0 + 8 * b, (use & 1u) ^ 1u, wc)) { ok = false; break; }   // epilogues drained this buffer
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t tmem_c = tmem_base + b * BN;
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!bar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(full0 + 8 * s, ph, wc)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t a_src = smem_base + s * STAGE_BYTES, b_src = a_src + A_STAGE_BYTES;
           const uint64_t adesc = make_desc_k_sw128(a_src);
@@ -374,7 +341,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       const int tm = p.n_fastest ? tile / tiles_n : tile % tiles_m, nb = p.n_fastest ? tile % tiles_n : tile / tiles_m;
       const int m0 = tm * C::TILE_M + (int)rank * BM, n0 = nb * BN;
       const uint32_t b = it & 1u, use = it >> 1;
-      const bool ok = __all_sync(0xffffffffu, bar_wait(tfull0 + 8 * b, use & 1u, abort_flag));
+      const bool ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * b, use & 1u, wc));
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int row = m0 + q * 32 + lane;
@@ -396,8 +363,28 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
             }
             if (p.c_transposed) {          // the lanes of a warp hold 32 consecutive rows: 128 contiguous bytes per column
               float* ct = p.C + (int64_t)(n0 + c) * p.ldc + row;
+              if (p.accumulate) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) ct[(int64_t)j * p.ldc] = __uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) ct[(int64_t)j * p.ldc] += __uint_as_float(r[j]);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) ct[(int64_t)j * p.ldc] = __uint_as_float(r[j]);
+              }
+            } else if (p.accumulate) {     // added to the rows finished by earlier calls (a later row block of the same dW)
+              if (n0 + c + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+                float4 old[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) old[j] = *reinterpret_cast<const float4*>(dst + 4 * j);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  old[j].x += __uint_as_float(r[4 * j]); old[j].y += __uint_as_float(r[4 * j + 1]);
+                  old[j].z += __uint_as_float(r[4 * j + 2]); old[j].w += __uint_as_float(r[4 * j + 3]);
+                  *reinterpret_cast<float4*>(dst + 4 * j) = old[j];
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) dst[j] += __uint_as_float(r[j]);
+              }
             } else if (splits > 1) {       // partial sum over a K part: add into the zeroed output
 #pragma unroll
               for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) atomicAdd(dst + j, __uint_as_float(r[j]));
@@ -422,6 +409,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             float z = (col0 + j < p.N) ? __uint_as_float(r[j]) : -INFINITY;
+            if (col0 + j == a) { p.z_a[row] = z; z = -INFINITY; }     // the sampled token's entry is left out of the sums
             r[j] = __float_as_uint(z);
             vm = fmaxf(vm, z);
           }
@@ -432,10 +420,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
 #pragma unroll
             for (int j = 0; j < 32; ++j) acc += ex2(fmaf(__uint_as_float(r[j]), 1.4426950408889634f, nm));
             s += acc;
-          }
-          if (a >= col0 && a < col0 + 32) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) if (col0 + j == a) p.z_a[row] = __uint_as_float(r[j]);
           }
         }
         if (row_ok) p.part[(int64_t)row * tiles_n + nb] = make_float2(m, s);
@@ -463,10 +447,16 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
               __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
               o[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
             }
-            s += acc0 + acc1;
-            if (a >= col0 && a < col0 + 32) {
+            if (a >= col0 && a < col0 + 32) {      // the sampled token's entry is left out of the row's sum
+              float s2 = 0.f;
 #pragma unroll
-              for (int j = 0; j < 32; ++j) if (col0 + j == a) p.z_a[row] = __uint_as_float(r[j]);
+              for (int j = 0; j < 32; ++j) {
+                if (col0 + j == a) p.z_a[row] = __uint_as_float(r[j]);
+                else if (col0 + j < p.N) s2 += ex2(fmaf(__uint_as_float(r[j]), 1.4426950408889634f, ncr));
+              }
+              s += s2;
+            } else {
+              s += acc0 + acc1;
             }
             if (store) {
               __nv_bfloat16* dst = p.P + (int64_t)row * p.ldp + col0;
@@ -524,7 +514,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       __syncwarp();
       if (lane == 0) {       // buffer drained: tell the MMA issuer (the leader's, in a pair)
         if (CG == 2 && rank != 0) bar_arrive_cluster(map_to_cta(tempty0 + 8 * b, 0));
-        else bar_arrive(tempty0 + 8 * b);
+        else mbar_arrive(tempty0 + 8 * b);
       }
     }
   }
@@ -532,9 +522,15 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  // A CTA in which a wait ran out stays for a moment: loads it issued may still be on their way (to its own shared
+  // memory and, in a pair, to the leader's barrier), and tensor-core work issued before may still be running; both
+  // finish within microseconds.  A CTA that did not give up has nothing in flight: its last accumulator was read.
+  if (wc.aborted()) {
+    if (tid == 0 && p.status) atomicOr(p.status, DPPO_STATUS_WAIT_LIMIT);
+    drain_after_abort();
+  }
   // a pair leaves together: neither CTA's shared or tensor memory may go away while the other can still reach it
   if (CG == 2) cluster_sync_all();
-  if (*abort_flag && tid == 0 && p.status) atomicOr(p.status, DPPO_STATUS_WAIT_LIMIT);
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (CG == 2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");

@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(1024) dppo_prelude_kernel(RowParams p) {
 // ---------------------------------------------------------------------------------------------
 // Finalize: loss = sum_t row_loss[t] in double, fixed order; optional statistics.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) dppo_finalize_kernel(RowParams p) {
+__global__ void __launch_bounds__(1024) dppo_finalize_kernel(RowParams p, int block_first, int block_last) {
   constexpr int NT = 1024;
   __shared__ double red[6][NT / 32];
   __shared__ float redmax[NT / 32];
@@ -69,16 +69,27 @@ __global__ void __launch_bounds__(1024) dppo_finalize_kernel(RowParams p) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) maxD = fmaxf(maxD, __shfl_xor_sync(0xffffffffu, maxD, o));
     if (lane == 0) {
-      *p.loss = (float)v[0];
-      if (p.stats) {
-        p.stats[0] = (float)p.hdr->n_valid;
-        p.stats[1] = (float)v[5];
-        p.stats[2] = (float)v[1];
-        p.stats[3] = maxD;
-        p.stats[4] = (float)v[2];
-        p.stats[5] = (float)v[3];
-        p.stats[6] = (float)v[4];
-        p.stats[7] = 0.f;
+      if (!block_first) {          // rows finished by earlier blocks of this call (same stream: a fixed order)
+#pragma unroll
+        for (int i = 0; i < 6; ++i) v[i] += p.hdr->acc[i];
+        maxD = fmaxf(maxD, p.hdr->max_d);
+      }
+      if (!block_last) {
+#pragma unroll
+        for (int i = 0; i < 6; ++i) p.hdr->acc[i] = v[i];
+        p.hdr->max_d = maxD;
+      } else {
+        *p.loss = (float)v[0];
+        if (p.stats) {
+          p.stats[0] = (float)p.hdr->n_valid;
+          p.stats[1] = (float)v[5];
+          p.stats[2] = (float)v[1];
+          p.stats[3] = maxD;
+          p.stats[4] = (float)v[2];
+          p.stats[5] = (float)v[3];
+          p.stats[6] = (float)v[4];
+          p.stats[7] = 0.f;
+        }
       }
     }
   }
@@ -89,8 +100,8 @@ cudaError_t launch_prelude(const RowParams& p, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_finalize(const RowParams& p, cudaStream_t st) {
-  dppo_finalize_kernel<<<1, 1024, 0, st>>>(p);
+cudaError_t launch_finalize(const RowParams& p, cudaStream_t st, bool block_first, bool block_last) {
+  dppo_finalize_kernel<<<1, 1024, 0, st>>>(p, block_first ? 1 : 0, block_last ? 1 : 0);
   return cudaGetLastError();
 }
 
@@ -120,9 +131,10 @@ __global__ void __launch_bounds__(kGenericThreads) dppo_row_generic_kernel(RowPa
       if (a < 0 || (int64_t)a >= p.V) { valid = false; flags |= DPPO_STATUS_BAD_SAMPLED_ID; }
     }
     if (valid) {
-      // sweep 1: per-thread online (max, sum of exp)
+      // sweep 1: per-thread online (max, sum of exp) over the entries other than the sampled token's
       float m = -INFINITY, s = 0.f;
       for (int64_t j = tid; j < p.V; j += kGenericThreads) {
+        if (j == (int64_t)a) continue;
         float z = to_f32<InT>(zrow[j]);
         if (z > m) {                                  // z is finite or +inf here
           s = s * ex2_approx((m - z) * kLog2e);
@@ -152,14 +164,15 @@ __global__ void __launch_bounds__(kGenericThreads) dppo_row_generic_kernel(RowPa
         double S = 0.0;
         for (int w = 0; w < kGenericThreads / 32; ++w)
           if (s_s[w] > 0.f || s_s[w] != s_s[w]) S += (double)s_s[w] * exp((double)s_m[w] - (double)mm);
-        double lse = (double)mm + log(S);
+        double lse, log_other;
+        combine_lse((double)mm, S, (double)to_f32<InT>(zrow[a]), lse, log_other);
         if (!isfinite(lse)) {
           flags |= DPPO_STATUS_NONFINITE_ROW;
         } else {
           double pi_a;
           int f2 = 0;
           auto z_at = [&](int id, int) { return to_f32<InT>(zrow[id]); };
-          row_scalars_warp(p, t, a, lse, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
+          row_scalars_warp(p, t, a, lse, log_other, scale, z_at, D, M, g, r, absdiff, pi_a, f2);
           if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
           else coef = make_coef(g, lse, pi_a);
         }

@@ -32,22 +32,41 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: gives up after ~2 s (or when another thread already gave up) and returns false.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// What every bounded wait of a CTA shares: the CTA's abort flag (shared memory; set by the first wait that runs out,
+// seen by all others) and the time a single wait may take.
+struct WaitCtl {
+  volatile int* flag;
+  unsigned long long limit_ns;
+  __device__ __forceinline__ bool aborted() const { return *flag != 0; }
+  __device__ __forceinline__ void abort() const { *flag = 1; }
+};
+constexpr unsigned long long kDefaultWaitNs = 2000000000ull;      // about 2 s
+// opts->wait_limit_us as nanoseconds (0: the default)
+inline unsigned long long wait_limit_ns(int wait_limit_us) {
+  return wait_limit_us > 0 ? (unsigned long long)wait_limit_us * 1000ull : kDefaultWaitNs;
+}
+// Bounded wait: gives up after the limit (or when another thread already gave up) and returns false.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtl& w) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 0xff) == 0) {
-      if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > 2000000000ull) { *abort_flag = 1; return false; }
+    if ((it & 0x3f) == 0) {
+      if (w.aborted()) return false;
+      if (globaltimer_ns() - t0 > w.limit_ns) { w.abort(); return false; }
     }
   }
 }
 // All lanes of a warp wait; the warp proceeds only if every lane saw the phase complete.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  const bool ok = mbar_wait(bar, parity, abort_flag);
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const WaitCtl& w) {
+  const bool ok = mbar_wait(bar, parity, w);
   return __all_sync(0xffffffffu, ok);
+}
+// After a wait ran out: time for bulk copies that may still be in flight towards this CTA's shared memory (or, in a
+// CTA pair, towards a barrier of the peer) to land before the CTA's shared memory goes away.
+__device__ __forceinline__ void drain_after_abort() {
+  const unsigned long long t0 = globaltimer_ns();
+  while (globaltimer_ns() - t0 < 1000000ull) __nanosleep(1000);
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
   asm volatile(

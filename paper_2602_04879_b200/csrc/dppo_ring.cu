@@ -75,7 +75,7 @@ __device__ __forceinline__ RowGeom row_geom(const RowParams& p, int64_t t, uint3
 template <typename InT, bool SH>
 __device__ __forceinline__ void produce_stream(const RowParams& p, uint32_t slots_base, unsigned char* slots_ptr, uint32_t full_base,
                                                uint32_t empty_base, int first_slot, int nslots, uint32_t row_bytes, int C, uint64_t policy,
-                                               volatile int* abort_flag, volatile unsigned int* follow, unsigned int lead) {
+                                               const WaitCtl& wc, volatile unsigned int* follow, unsigned int lead) {
   const char* logits = reinterpret_cast<const char*>(p.logits);
   const int64_t t0 = blockIdx.x, G = gridDim.x;
   RingPos pos{0, 0};
@@ -93,15 +93,15 @@ __device__ __forceinline__ void produce_stream(const RowParams& p, uint32_t slot
           if (issued - *follow >= lead) {
             const unsigned long long w0 = globaltimer_ns();
             while (issued - *follow >= lead) {
-              if (*abort_flag) return;
-              if (globaltimer_ns() - w0 > 2000000000ull) { *abort_flag = 1; return; }
+              if (wc.aborted()) return;
+              if (globaltimer_ns() - w0 > wc.limit_ns) { wc.abort(); return; }
               __nanosleep(64);
             }
           }
           ++issued;
         }
         // lap u >= 1 of a slot needs its (u-1)-th release: parity (u-1)&1 = phase^1
-        if (!first_lap && !mbar_wait(empty_base + 8u * slot, pos.phase ^ 1u, abort_flag)) return;
+        if (!first_lap && !mbar_wait(empty_base + 8u * slot, pos.phase ^ 1u, wc)) return;
         const uint32_t off = (uint32_t)c * kChunkBytes;
         const uint32_t bar = full_base + 8u * slot;
         if (!SH) {
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
   const uint32_t empty_base = smem_u32(&misc->empty[0]);
   const uint32_t part_full = smem_u32(&misc->part_full[0]), part_empty = smem_u32(&misc->part_empty[0]);
   const uint32_t coef_full = smem_u32(&misc->coef_full[0]), coef_empty = smem_u32(&misc->coef_empty[0]);
-  volatile int* abort_flag = &misc->abort_flag;
+  const WaitCtl wc{&misc->abort_flag, p.wait_ns};
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // slots [0, ns_sum) feed the sum warps, [ns_sum, nslots) the grad warps; the second read comes from L2 with a
   // shorter latency but is issued as early as possible, so the grad ring gets the larger share (4 + 10 of 14)
@@ -182,7 +182,8 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
 
   if (warp >= 2 * kGroupWarps + 1) {
     // ------------------------------------------------------------------ producers (one lane each)
-    if (lane == 0) {
+    // (test injection: the producers issue nothing, so that every consumer wait of the CTA runs out)
+    if (lane == 0 && !(p.inject & DPPO_INJECT_NO_COPIES)) {
       uint64_t policy;
       if (warp == 2 * kGroupWarps + 1) {
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
@@ -191,11 +192,11 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         // occupy about #SMs x lead chunks of L2 (61 MB at V = 151936 bf16); a longer lead makes the second
         // read miss L2, a shorter one leaves the sum warps idle.  Measured optimum on B200: C + 7.
         const int lead = (C + 7 <= 26 || C + 2 > 26) ? ((C + 7 <= 26) ? C + 7 : C + 2) : 26;
-        produce_stream<InT, SH>(p, slots_base, smem, full_base, empty_base, 0, ns_sum, row_bytes, C, policy, abort_flag,
+        produce_stream<InT, SH>(p, slots_base, smem, full_base, empty_base, 0, ns_sum, row_bytes, C, policy, wc,
                                 &misc->grad_chunks, (unsigned int)lead);
       } else {
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-        produce_stream<InT, SH>(p, slots_base, smem, full_base, empty_base, ns_sum, ns_grad, row_bytes, C, policy, abort_flag, nullptr, 0u);
+        produce_stream<InT, SH>(p, slots_base, smem, full_base, empty_base, ns_sum, ns_grad, row_bytes, C, policy, wc, nullptr, 0u);
       }
     }
   } else if (warp < kGroupWarps) {
@@ -206,16 +207,21 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
     int meta = load_meta(p, t0);
     for (int64_t t = t0; t < p.T; t += G) {
       const int meta_next = load_meta(p, t + G);
-      if (__shfl_sync(0xffffffffu, *abort_flag, 0)) break;
+      if (__shfl_sync(0xffffffffu, (int)wc.aborted(), 0)) break;
       if (meta >= 0) {
         // per-thread partial: s = sum exp(z - ref); ref is the maximum of the thread's first entries
         // and moves up only when a chunk's sum shows that an entry exceeds it by > 44
+        // the sampled token's entry is left out of the sums (the scalar warp adds it: 1 - pi(a) then comes from the
+        // sum over the other entries and keeps its relative accuracy when pi(a) is close to 1)
         float ref = -INFINITY, nm = 0.f, s = 0.f;
         const RowGeom gm = row_geom<InT, SH>(p, t, row_bytes, C);
+        const uint32_t a_img = (uint32_t)meta + gm.head / (uint32_t)sizeof(InT);   // the sampled token's place in the image
         for (int c = 0; c < gm.C; ++c) {
-          const bool ok = mbar_wait_warp(full_base + 8u * pos.slot, pos.phase, abort_flag);
+          const bool ok = mbar_wait_warp(full_base + 8u * pos.slot, pos.phase, wc);
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
           const uint32_t sbase = slots_base + (uint32_t)pos.slot * kChunkBytes;
+          const uint32_t a_loc = a_img - cbase / (uint32_t)sizeof(InT);            // its place in this chunk (if below the chunk's size)
+          const bool has_a = a_loc < (uint32_t)(kChunkBytes / sizeof(InT));        // warp-uniform
           if (ok) {
             // chunks that the bulk copy filled completely take the straight-line path
             const bool full_chunk = cbase + (uint32_t)kChunkBytes <= gm.xa;
@@ -232,6 +238,13 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
 #pragma unroll
                 for (int i = 0; i < N; ++i)
                   if ((uint32_t)i * (uint32_t)sizeof(InT) < gm.head) z[0][i] = -INFINITY;
+              }
+              if (has_a) {
+#pragma unroll
+                for (int k = 0; k < kVecPerThread; ++k)
+#pragma unroll
+                  for (int i = 0; i < N; ++i)
+                    if (((uint32_t)k * kGroupThreads + gtid) * N + i == a_loc) z[k][i] = -INFINITY;
               }
               if (ref == -INFINITY) {            // first chunk of the row: reference = maximum of the first entries
                 float vm = z[0][0];
@@ -281,6 +294,11 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
                       if (pos_b < gm.head || pos_b >= gm.xend) z[i] = -INFINITY;
                     }
                   }
+                  if (has_a) {
+#pragma unroll
+                    for (int i = 0; i < N; ++i)
+                      if (off / (uint32_t)sizeof(InT) + i == a_loc) z[i] = -INFINITY;
+                  }
                   float vm = z[0];
 #pragma unroll
                   for (int i = 1; i < N; ++i) vm = fmaxf(vm, z[i]);
@@ -311,7 +329,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         if (lane == 0) {
           const uint32_t b = vrow & 1u;
           bool ok = true;
-          if (vrow >= 2) ok = mbar_wait(part_empty + 8u * b, ((vrow >> 1) & 1u) ^ 1u, abort_flag);
+          if (vrow >= 2) ok = mbar_wait(part_empty + 8u * b, ((vrow >> 1) & 1u) ^ 1u, wc);
           if (ok) {
             misc->part[b][warp] = make_float2(ref, s);
             mbar_arrive(part_full + 8u * b);
@@ -331,7 +349,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
     int meta = load_meta(p, t0);
     for (int64_t t = t0; t < p.T; t += G) {
       const int meta_next = load_meta(p, t + G);
-      if (__shfl_sync(0xffffffffu, *abort_flag, 0)) break;
+      if (__shfl_sync(0xffffffffu, (int)wc.aborted(), 0)) break;
       OutT* drow = dlogits + t * p.ld_out;
       const RowGeom gm = row_geom<InT, SH>(p, t, row_bytes, C);
       // shifted rows: the output row is shifted by the same number of bytes (same element size, same misalignment, the
@@ -350,7 +368,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         }
       } else {
         const uint32_t b = vrow & 1u;
-        const bool have = mbar_wait_warp(coef_full + 8u * b, (vrow >> 1) & 1u, abort_flag);
+        const bool have = mbar_wait_warp(coef_full + 8u * b, (vrow >> 1) & 1u, wc);
         RowCoef coef = misc->coef[b];
         __syncwarp();
         if (lane == 0 && have) mbar_arrive(coef_empty + 8u * b);
@@ -359,7 +377,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         const uint32_t a = (uint32_t)meta + head_e;                    // the sampled token's place in the image
         for (int c = 0; c < gm.C; ++c) {
           const int slot = ns_sum + pos.slot;
-          const bool ok = mbar_wait_warp(full_base + 8u * slot, pos.phase, abort_flag);
+          const bool ok = mbar_wait_warp(full_base + 8u * slot, pos.phase, wc);
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
           const uint32_t sbase = slots_base + (uint32_t)slot * kChunkBytes;
           if (ok) {
@@ -431,7 +449,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
     int meta = load_meta(p, t0);
     for (int64_t t = t0; t < p.T; t += G) {
       const int meta_next = load_meta(p, t + G);
-      if (__shfl_sync(0xffffffffu, *abort_flag, 0)) break;
+      if (__shfl_sync(0xffffffffu, (int)wc.aborted(), 0)) break;
       int flags = (meta == -2) ? DPPO_STATUS_BAD_SAMPLED_ID : 0;
       float D = 0.f, r = 0.f, absdiff = 0.f;
       int M = 0;
@@ -459,7 +477,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           for (int i = 0; i < kPre; ++i)
             if (id_pre[i] >= 0 && (int64_t)id_pre[i] < p.V) zk_pre[i] = to_f32<InT>(zrow[id_pre[i]]);
         }
-        const bool have = mbar_wait_warp(part_full + 8u * b, (vrow >> 1) & 1u, abort_flag);
+        const bool have = mbar_wait_warp(part_full + 8u * b, (vrow >> 1) & 1u, wc);
         float2 pr = make_float2(-INFINITY, 0.f);
         if (lane < kGroupWarps) pr = misc->part[b][lane];
         __syncwarp();
@@ -472,8 +490,9 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
           double part = 0.0;
           if (pr.y > 0.f || pr.y != pr.y) part = (double)pr.y * exp((double)pr.x - (double)mm);
-          const double S = warp_sum(part);
-          const double lse = (double)mm + log(S);
+          const double S_o = warp_sum(part);                 // sum over the entries other than the sampled token
+          double lse, log_other;
+          combine_lse((double)mm, S_o, (double)z_a, lse, log_other);
           if (!isfinite(lse)) {
             flags |= DPPO_STATUS_NONFINITE_ROW;
           } else {
@@ -490,14 +509,14 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
               if (k < 32 * kPre) { id = pick(id_pre, k >> 5); pm = pick(pm_pre, k >> 5); }
               else { id = p.topk_ids[t * (int64_t)p.K + k]; pm = p.topk_p[t * (int64_t)p.K + k]; }
             };
-            row_scalars_warp(p, t, a, lse, scale, z_at, list_at, D, M, g, r, absdiff, pi_a, f2);
+            row_scalars_warp(p, t, a, lse, log_other, scale, z_at, list_at, D, M, g, r, absdiff, pi_a, f2);
             if (f2) { flags |= f2; D = 0.f; M = 0; g = 0.0; r = 0.f; absdiff = 0.f; }
             else coef = make_coef(g, lse, pi_a);
           }
         }
         if (lane == 0) {
           bool ok = have;
-          if (ok && vrow >= 2) ok = mbar_wait(coef_empty + 8u * b, ((vrow >> 1) & 1u) ^ 1u, abort_flag);
+          if (ok && vrow >= 2) ok = mbar_wait(coef_empty + 8u * b, ((vrow >> 1) & 1u) ^ 1u, wc);
           if (ok) {
             misc->coef[b] = coef;
             mbar_arrive(coef_full + 8u * b);
@@ -518,11 +537,9 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
   }
 
   __syncwarp();
-  if (*abort_flag) {
+  if (wc.aborted()) {
     if (lane == 0) atomicOr(p.status, DPPO_STATUS_WAIT_LIMIT);
-    // leave time for bulk copies that may still be in flight towards this CTA's shared memory
-    const unsigned long long t_exit = globaltimer_ns();
-    while (globaltimer_ns() - t_exit < 1000000ull) __nanosleep(1000);
+    drain_after_abort();
   }
 }
 

@@ -17,7 +17,9 @@ static __device__ __align__(256) unsigned char g_static_ws[kStaticBytes];
 std::mutex g_mu;
 void* g_ws_ptr[kMaxDevices] = {};
 
-// Device address of the array on the current device; looked up once per device.
+// Device address of the array on the current device; looked up once per device and kept for the life of the
+// process (so the entry point must not be used again after a cudaDeviceReset of that device: the kept address
+// would be stale).
 int static_ws_for_current_device(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DPPO_ERR_CUDA;
