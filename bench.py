@@ -30,7 +30,6 @@ DELTA = 0.2
 METRIC = "tokens/sec fwd+bwd DPPO loss at V=151936 bf16"
 BYTES_PER_TOKEN = 4 * VOCAB          # bf16 logits read (2V) + bf16 dlogits written (2V)
 WORKLOAD = "qwen3_vocab_binary_tv: T=16384 (16 responses x 1024), V=151936, bf16 logits, Binary-TV, delta=0.2"
-ORACLE_ROWS_PER_STEP = 192           # CPU oracle sample per step (about a second of numpy work)
 
 
 def parse_args():
@@ -41,7 +40,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default="binary_tv", choices=["binary_tv", "binary_kl"])
     ap.add_argument("--rows", type=int, default=T_ROWS, help="rows per GPU; anything but the default is a reduced case for profiling, not the benchmark workload")
-    ap.add_argument("--kernel", default="auto", choices=["auto", "ring", "scale", "generic"], help="row kernel of the main measurement")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "ring", "generic"], help="row kernel of the main measurement")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--fused-only", action="store_true", help="run only the fused LM-head measurement (profiling aid)")
     ap.add_argument("--fused-rows", type=int, default=8192, help="token rows of the fused measurement; anything but 8192 is a reduced profiling case")
@@ -120,6 +119,14 @@ def bench_fused(dppo, wl, dev, steps=40, warmup=10, T=8192):
         ms_topk = _time_steps(torch, fn, steps, warmup)
         assert int(status.item()) == 0
         del bk, wsk
+    # the same step finished in blocks of 2048 rows: the workspace is that of 2048 rows (0.7 GB instead of 2.6 GB)
+    R = 2048
+    ws_b = torch.empty(dppo.dppo_fused_workspace_bytes(min(T, R), d, V), dtype=torch.uint8, device=dev)
+    fn_b = lambda: dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.BINARY_TV, DELTA,
+                                                  workspace=ws_b, dHidden=dH, dW=dW, status=status, rows_per_block=R)
+    ms_blocks = _time_steps(torch, fn_b, steps, warmup)
+    ws_bytes, ws_b_bytes = ws.numel(), ws_b.numel()
+    del ws_b
     peak, src = measured_tensor_peak()
     useful = 6.0 * T * d * V / (ms * 1e-3) / 1e12          # forward + dHidden + dW; every logits tile is computed once
     return {"workload": ("" if T == 8192 else f"REDUCED to {T} rows (profiling case): ") + "fused_lm_head_binary_tv: hidden [8192,2048] bf16 x W [2048,151936] bf16, delta=0.2",
@@ -129,7 +136,8 @@ def bench_fused(dppo, wl, dev, steps=40, warmup=10, T=8192):
                          "flop_count": "6*T*d*V (forward, dHidden, dW); nothing is recomputed"},
             "gpu_launches_per_step": 15, "loss": float(out["loss"].item()),
             "ms_per_step_quarter_of_responses_zero_advantage": ms_sparse, "ms_per_step_topk_tv_k20": ms_topk,
-            "ms_per_step_lm_head_vocab_major": ms_vd}
+            "ms_per_step_lm_head_vocab_major": ms_vd,
+            "ms_per_step_row_blocks_2048": ms_blocks, "workspace_bytes": ws_bytes, "workspace_bytes_row_blocks_2048": ws_b_bytes}
 
 
 def _time_steps(torch, fn, steps, warmup):
@@ -206,6 +214,20 @@ def bench_other_configs(dppo, wl, dev, steps=100, warmup=10, n_resp=16):
     ms = _time_steps(torch, lambda: dppo.dppo_exact_divergence(b.logits, zmu, status=status), steps, warmup)
     out["exact_divergence"] = entry(ms, T, T, T * BYTES_PER_TOKEN, f"dppo_exact_divergence, T={T}, V=151936, bf16; bytes = both logits tensors read once "
                                     "(the second sweep is served by L2); 4 exp per element pair: the special-function pipe, not HBM, bounds it")
+    # the monitor without the TV (tv = NULL): KL and entropy need one sweep, so each tensor is read once and nothing again
+    ms1 = _time_steps(torch, lambda: dppo.dppo_exact_divergence(b.logits, zmu, status=status, want_tv=False), steps, warmup)
+    out["exact_kl_only"] = entry(ms1, T, T, T * BYTES_PER_TOKEN, f"dppo_exact_divergence with tv = NULL (KL(mu||pi) and entropy only), T={T}, V=151936, bf16; "
+                                 "bytes = both logits tensors read once; 2 exp per element pair")
+    out["exact_kl_only"]["roofline"] = {"bound": "hbm", "achieved": out["exact_kl_only"]["achieved_gbs"], "peak": peak, "unit": "GB/s",
+                                        "frac": out["exact_kl_only"]["frac_of_hbm_peak"], "peak_source": "of " + src}
+    # DPPO with the exact KL as its trust region (the paper's delta_KL = 0.05): one-sweep monitor, then the loss kernel
+    def exact_kl_then_loss():
+        ex = dppo.dppo_exact_divergence(b.logits, zmu, status=status, want_tv=False)
+        return dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.GIVEN_D, 0, 0.05,
+                                      dlogits=dl, workspace=ws, status=status, given_divergence=ex["kl"])
+    ms3 = _time_steps(torch, exact_kl_then_loss, steps, warmup)
+    out["exact_kl_trust_region"] = entry(ms3, T, T, T * (BYTES_PER_TOKEN + 2 * VOCAB),
+                                         f"dppo_exact_divergence(tv = NULL) + dppo_loss_fwd_bwd(GIVEN_D, delta 0.05), T={T}; bytes = both logits tensors read once + dlogits written")
     # DPPO with the exact TV as its trust region: the monitor, then the loss kernel on the divergence it produced
     def exact_then_loss():
         ex = dppo.dppo_exact_divergence(b.logits, zmu, status=status)
@@ -242,6 +264,30 @@ def bench_other_configs(dppo, wl, dev, steps=100, warmup=10, n_resp=16):
     out["topk_kl_k64_ragged_delta0.05"] = entry(ms, T2, valid, valid * BYTES_PER_TOKEN + (T2 - valid) * 2 * VOCAB,
                                                 f"responses 0 and 1 of the 64 as padded blocks of 8192 rows ({valid} valid of {T2}); "
                                                 "bytes = valid rows read + every row of dlogits written (padding rows are zero-filled)")
+    del lg, dl, blocks
+    torch.cuda.empty_cache()
+    if n_resp == 16:
+        # the whole batch of 64 ragged responses (159 GB of padded logits: more than the device holds), streamed as 64 calls
+        # of one padded block each with the global scale; each block is regenerated on the device (untimed), run once to
+        # warm up and then timed over three calls; the batch time is the sum over the 64 blocks
+        dl = torch.empty((8192, VOCAB), dtype=torch.bfloat16, device=dev)
+        ws = torch.empty(dppo.dppo_workspace_bytes(8192), dtype=torch.uint8, device=dev)
+        tot_ms, loss_sum = 0.0, 0.0
+        for i in range(len(lengths)):
+            x = wl.ragged_response(dev, i, lengths)
+            fn = lambda: dppo.dppo_loss_fwd_bwd(x.logits, x.sampled_ids, x.mu_logp, x.advantages, x.token_mask, dppo.TOPK_KL, 64, 0.05,
+                                                x.mu_topk_ids, x.mu_topk_p, loss_scale=scale, dlogits=dl, workspace=ws, status=status)
+            tot_ms += _time_steps(torch, fn, 3, 1)
+            loss_sum += float(fn()["loss"].item())
+            del x
+        assert int(status.item()) == 0
+        nv, nrows = int(sum(lengths)), 8192 * len(lengths)
+        e = entry(tot_ms, nrows, nv, nv * BYTES_PER_TOKEN + (nrows - nv) * 2 * VOCAB,
+                  f"all 64 responses ({nv} valid of {nrows} padded rows), one call per padded block of 8192 rows, global scale 1/{nv}; "
+                  "ms_per_step is the sum of the 64 calls; bytes = valid rows read + every row of dlogits written")
+        e["loss"] = loss_sum
+        e["calls"] = len(lengths)
+        out["topk_kl_k64_ragged_whole_batch"] = e
     return out
 
 
@@ -264,16 +310,31 @@ def measured_traffic():
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU from a thread (NVML) while the GPU works."""
 
-    def __init__(self, index):
+    def __init__(self, index, uuid=None):
         self.samples = []
         self.stop_flag = False
         self.thread = None
         self.ok = False
+        self.by = None
         try:
             import pynvml
             self.nv = pynvml
             pynvml.nvmlInit()
-            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            # NVML numbers the GPUs of the machine, CUDA those this process may see: resolve the handle from the CUDA
+            # device's UUID, and fall back to the index only when that fails
+            self.h = None
+            if uuid:
+                u = str(uuid)
+                for cand in (u, "GPU-" + u, u.replace("GPU-", "")):
+                    try:
+                        self.h = pynvml.nvmlDeviceGetHandleByUUID(cand.encode() if hasattr(cand, "encode") else cand)
+                        self.by = "uuid"
+                        break
+                    except Exception:  # noqa: BLE001
+                        self.h = None
+            if self.h is None:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+                self.by = "index"
             self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
             self.ok = True
         except Exception:  # noqa: BLE001
@@ -297,6 +358,7 @@ class ClockSampler:
             time.sleep(0.01)
 
     def start(self):
+        self.stop_flag = False
         if self.ok:
             self.thread = threading.Thread(target=self._run, daemon=True)
             self.thread.start()
@@ -311,7 +373,7 @@ class ClockSampler:
                  0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting"}
         sel = [s for s in self.samples if t0 <= s[0] <= t1] or self.samples
         if not sel:
-            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "nvml_handle_by": self.by}
         mhz = sorted(s[1] for s in sel)
         bits = 0
         for s in sel:
@@ -320,31 +382,99 @@ class ClockSampler:
         mem = sorted(s[3] for s in sel)
         watts = sorted(s[4] for s in sel if s[4] is not None)
         return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(sel),
-                "mem_mhz": mem[len(mem) // 2], "power_w": watts[len(watts) // 2] if watts else None}
+                "mem_mhz": mem[len(mem) // 2], "power_w": watts[len(watts) // 2] if watts else None, "nvml_handle_by": self.by}
 
 
 # ----------------------------------------------------------------------------------------- oracle arm
 
-def oracle_tokens_per_s(rows, seed, variant_code, chunk=1024):
-    """Times the float64 oracle, as it stands, on the first `rows` rows of the workload, generated on the CPU and
-    handed over `chunk` rows at a time (bounded host memory); only the oracle calls are timed."""
-    import numpy as np
-    import torch
-    from paper_2602_04879_b200 import workloads as wl
-    from oracle import dppo_oracle as O
-    dt = 0.0
-    for row0 in range(0, rows, chunk):
-        n = min(chunk, rows - row0)
-        b = wl.qwen_vocab_rows("cpu", seed=seed, row0=row0, rows=n)
-        z = b.logits.float().numpy().astype(np.float64)
-        ids = b.sampled_ids.numpy()
-        mu = b.mu_logp.numpy().astype(np.float64)
-        adv = b.advantages.numpy().astype(np.float64)
-        t0 = time.perf_counter()
-        O.dppo_loss_fwd_bwd(z, ids, mu, adv, None, variant_code, 0, DELTA, 1.0 / T_ROWS)
-        dt += time.perf_counter() - t0
-        del b, z
-    return rows / dt, dt, torch.get_num_threads()
+GEN_BLOCK = 512                      # rows per generator block of the workload (any block can be regenerated alone)
+ORACLE_ROWS_PER_WORKER = 64
+
+
+def host_cores():
+    """Cores this process may use: the scheduler affinity, cut by a cgroup CPU quota if there is one."""
+    try:
+        n = len(os.sched_getaffinity(0))
+    except AttributeError:
+        n = os.cpu_count() or 1
+    try:
+        with open("/sys/fs/cgroup/cpu.max") as f:
+            quota, period = f.read().split()
+        if quota != "max":
+            n = min(n, max(1, int(float(quota) / float(period))))
+    except Exception:  # noqa: BLE001
+        pass
+    return max(1, n)
+
+
+def oracle_workers():
+    """One oracle process per host core, bounded so that the processes (an interpreter with torch and about 0.4 GB of
+    float64 rows each) stay far inside the host's memory."""
+    n = min(host_cores(), 96)
+    try:
+        with open("/proc/meminfo") as f:
+            avail_kb = next(int(l.split()[1]) for l in f if l.startswith("MemAvailable"))
+        n = min(n, max(1, int(avail_kb / 1048576 / 3)))
+    except Exception:  # noqa: BLE001
+        pass
+    return max(1, n)
+
+
+def _oracle_worker(w, seed, variant_code, iters, reps, barrier, queue):
+    """One process of the CPU arm: regenerates its own 64 rows of the workload (untimed), then, `iters` times, meets the
+    other workers at the barrier and runs the float64 oracle, as it stands, `reps` times over those rows."""
+    try:
+        import numpy as np
+        import torch
+        torch.set_num_threads(1)
+        from paper_2602_04879_b200 import workloads as wl
+        from oracle import dppo_oracle as O
+        n = ORACLE_ROWS_PER_WORKER
+        blocks = T_ROWS // GEN_BLOCK
+        blk, m = w % blocks, (w // blocks) % (GEN_BLOCK // n)
+        # a block is generated from its first row on: take the prefix that ends with this worker's rows
+        b = wl.qwen_vocab_rows("cpu", seed=seed, row0=GEN_BLOCK * blk, rows=n * (m + 1))
+        z = b.logits[n * m:].float().numpy().astype(np.float64)
+        ids = b.sampled_ids[n * m:].numpy()
+        mu = b.mu_logp[n * m:].numpy().astype(np.float64)
+        adv = b.advantages[n * m:].numpy().astype(np.float64)
+        del b
+        for it in range(iters):
+            barrier.wait(timeout=600)
+            t0 = time.perf_counter()
+            for _ in range(reps):
+                O.dppo_loss_fwd_bwd(z, ids, mu, adv, None, variant_code, 0, DELTA, 1.0 / T_ROWS)
+            queue.put((w, it, t0, time.perf_counter()))
+    except Exception as e:  # noqa: BLE001
+        queue.put((w, -1, repr(e), 0.0))
+
+
+def oracle_parallel(seed, variant_code, iters, reps, workers=None):
+    """Runs the oracle on `workers` processes at once (spawned: safe after CUDA has been initialised).  Returns per
+    iteration the wall time from the first worker's start to the last worker's end (one monotonic clock for all
+    processes of the machine), the rows processed per iteration, and the worker count."""
+    import multiprocessing as mp
+    W = workers or oracle_workers()
+    ctx = mp.get_context("spawn")
+    barrier, queue = ctx.Barrier(W), ctx.Queue()
+    procs = [ctx.Process(target=_oracle_worker, args=(w, seed, variant_code, iters, reps, barrier, queue), daemon=True) for w in range(W)]
+    for p in procs:
+        p.start()
+    spans = {}
+    try:
+        for _ in range(W * iters):
+            w, it, t0, t1 = queue.get(timeout=1200)
+            if it < 0:
+                raise RuntimeError(f"oracle worker {w} failed: {t0}")
+            lo, hi = spans.get(it, (t0, t1))
+            spans[it] = (min(lo, t0), max(hi, t1))
+    finally:
+        for p in procs:
+            p.join(timeout=30)
+            if p.is_alive():
+                p.kill()
+    times = [spans[i][1] - spans[i][0] for i in range(iters)]
+    return times, W * ORACLE_ROWS_PER_WORKER * reps, W
 
 
 def run_reference(args):
@@ -355,21 +485,18 @@ def run_reference(args):
     code = O.BINARY_TV if args.variant == "binary_tv" else O.BINARY_KL
     steps = max(1, min(args.steps, 8))
     warm = max(0, min(args.warmup, 1))
-    for _ in range(warm):
-        oracle_tokens_per_s(ORACLE_ROWS_PER_STEP, 1, code)
-    tot_rows, tot_t = 0, 0.0
-    for _ in range(steps):
-        tps, dt, _ = oracle_tokens_per_s(ORACLE_ROWS_PER_STEP, 1, code)
-        tot_rows += ORACLE_ROWS_PER_STEP
-        tot_t += dt
-    value = tot_rows / tot_t
-    sample = f"{ORACLE_ROWS_PER_STEP} rows of the workload per step (first rows of the seeded batch), {steps} steps timed"
+    reps = 24                                     # 64 rows x 24 per worker and step: between one and two seconds of float64 numpy
+    times, rows_per_step, W = oracle_parallel(1, code, warm + steps, reps)
+    tot_t = sum(times[warm:])
+    value = rows_per_step * steps / tot_t
+    sample = (f"{W} processes (one per host core), each running the oracle {reps} times per step over its own "
+              f"{ORACLE_ROWS_PER_WORKER} rows of the seeded batch = {rows_per_step} token rows per step; {steps} steps timed")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": steps, "warmup": warm, "ms_per_step": 1e3 * tot_t / steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "variant": args.variant, "note": "float64 numpy oracle on host cores"},
-        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "config": {"workload": WORKLOAD, "variant": args.variant, "note": "float64 numpy oracle on the host cores"},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": W, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
@@ -411,7 +538,7 @@ def run_ours(args):
     ws = torch.empty(dppo.dppo_workspace_bytes(T), dtype=torch.uint8, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
 
-    kernel_code = {"auto": dppo.KERNEL_AUTO, "ring": dppo.KERNEL_RING, "scale": dppo.KERNEL_SCALE, "generic": dppo.KERNEL_GENERIC}[args.kernel]
+    kernel_code = {"auto": dppo.KERNEL_AUTO, "ring": dppo.KERNEL_RING, "generic": dppo.KERNEL_GENERIC}[args.kernel]
 
     def step():
         return dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, variant, 0, DELTA,
@@ -422,7 +549,11 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
+    try:
+        uuid = torch.cuda.get_device_properties(local).uuid
+    except Exception:  # noqa: BLE001
+        uuid = None
+    sampler = ClockSampler(local, uuid)
     for _ in range(max(3, args.warmup)):
         out = step()
     barrier()
@@ -462,6 +593,33 @@ def run_ours(args):
     roofline["traffic"] = measured_traffic()
     clocks = sampler.summary(t_host0, t_host1)
 
+    # the same step for a further stretch, long enough for the power management to settle (the timed region above is a
+    # burst of some tens of milliseconds): what a training loop would see, with the clock it ran at
+    sus_steps = max(200, args.steps)
+    sus = ClockSampler(local, uuid)
+    barrier()
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sus.start()
+    th0 = time.perf_counter()
+    s0.record()
+    for _ in range(sus_steps):
+        step()
+    s1.record()
+    barrier()
+    th1 = time.perf_counter()
+    sus.stop()
+    sus_ms = s0.elapsed_time(s1) / sus_steps
+    if world > 1:
+        t = torch.tensor([sus_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        sus_ms = float(t.item())
+    sc = sus.summary(th0, th1)
+    sus_gbs = T * BYTES_PER_TOKEN / (sus_ms * 1e-3) / 1e9
+    roofline["sustained"] = {"steps": sus_steps, "ms_per_step": sus_ms, "achieved": sus_gbs, "frac": sus_gbs / peak,
+                             "sm_mhz": sc.get("sm_mhz"), "reasons": sc.get("reasons"), "power_w": sc.get("power_w"),
+                             "ms_times_ghz": None if not sc.get("sm_mhz") else sus_ms * sc["sm_mhz"] / 1e3}
+    assert int(status.item()) == 0
+
     line = {
         "metric": METRIC, "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -471,19 +629,23 @@ def run_ours(args):
                    "parallelism": f"dp{world} row shards, no data-path collective", "logits_dtype": "bf16", "dlogits_dtype": "bf16"},
         "roofline": roofline, "clocks": clocks, "gpu_launches": 3 * args.steps, "loss": loss_val,
         "ms_per_step_best": per_step[0], "ms_per_step_median": per_step[len(per_step) // 2],
+        "ms_times_ghz": None if not clocks.get("sm_mhz") else ms_per_step * clocks["sm_mhz"] / 1e3,
     }
 
-    # end to end through the host-buffer entry point: pinned host inputs -> device -> loss / D / M back on the host
+    # end to end through the host-buffer entry point: pinned host inputs -> device -> loss, divergence, mask AND the
+    # gradient back in pinned host memory (the gradient's copy back overlaps the next chunk's copy in)
     if not args.no_e2e:
         rows_per_chunk = 1024
         pin = lambda x: x.cpu().pin_memory()
         h = dict(logits=pin(b.logits), ids=pin(b.sampled_ids), mu=pin(b.mu_logp), adv=pin(b.advantages))
-        outbuf = dict(divergence=torch.empty(T, dtype=torch.float32).pin_memory(), mask=torch.empty(T, dtype=torch.uint8).pin_memory())
+        outbuf = dict(divergence=torch.empty(T, dtype=torch.float32).pin_memory(), mask=torch.empty(T, dtype=torch.uint8).pin_memory(),
+                      dlogits=torch.empty((T, VOCAB), dtype=torch.bfloat16).pin_memory())
         staging = torch.empty(dppo.dppo_host_staging_bytes(rows_per_chunk, VOCAB, 0, dppo.BF16), dtype=torch.uint8, device=dev)
 
         def e2e_step():
             return dppo.dppo_loss_fwd_bwd_host(h["logits"], h["ids"], h["mu"], h["adv"], None, variant, 0, DELTA,
-                                               loss_scale=scale, rows_per_chunk=rows_per_chunk, staging=staging, out=outbuf)
+                                               loss_scale=scale, rows_per_chunk=rows_per_chunk, staging=staging, out=outbuf,
+                                               want_dlogits=True)
         e2e_steps = max(1, min(args.steps, 5))
         e2e_step()
         barrier()
@@ -497,10 +659,14 @@ def run_ours(args):
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             dt = float(t.item())
         assert r["status"] == 0
-        line["e2e"] = {"value": world * T * e2e_steps / dt, "unit": "tokens/s",
-                       "h2d_bytes_per_step": T * VOCAB * 2 + T * 12, "d2h_bytes_per_step": T * 5 + 8,
-                       "steps": e2e_steps, "note": "dppo_loss_fwd_bwd_host: pinned host logits/ids/mu_logp/advantages in, loss + divergence + mask out; dlogits stay on the device"}
-        del h, staging
+        # the gradient that arrived on the host is the one the device-resident step computed
+        probe = [0, 1, T // 2, T - 1]
+        same = bool(torch.equal(outbuf["dlogits"][probe], out["dlogits"][torch.as_tensor(probe, device=dev)].cpu()))
+        line["e2e"] = {"gradient_on_host_equals_device_step": same,"value": world * T * e2e_steps / dt, "unit": "tokens/s",
+                       "h2d_bytes_per_step": T * VOCAB * 2 + T * 12, "d2h_bytes_per_step": T * VOCAB * 2 + T * 5 + 8,
+                       "steps": e2e_steps, "note": "dppo_loss_fwd_bwd_host: pinned host logits/ids/mu_logp/advantages in; loss, divergence, mask "
+                                                   "and the bf16 gradient [T, V] out to pinned host memory"}
+        del h, staging, outbuf
 
     if world == 1 and not args.no_fused and T == T_ROWS:
         del dlogits
@@ -514,10 +680,16 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import dppo_oracle as O
         code = O.BINARY_TV if args.variant == "binary_tv" else O.BINARY_KL
-        rows = min(T, 12288)                  # about 10 s of float64 numpy at the full size
-        tps, dt, _ = oracle_tokens_per_s(rows, 1, code)
-        line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": 1, "kind": "oracle",
-                                "sample": f"first {rows} rows of the workload regenerated on the CPU, {dt:.1f} s of float64 numpy"}
+        reps = 96                                 # 64 rows x 96 per process: several seconds of float64 numpy each
+        times, rows, W = oracle_parallel(1, code, 1, reps)
+        line["cpu_baseline"] = {"value": rows / times[0], "unit": "tokens/s", "cores": W, "kind": "oracle",
+                                "sample": f"{W} processes (one per host core) each ran the float64 numpy oracle {reps} times over its own "
+                                          f"{ORACLE_ROWS_PER_WORKER} rows of the workload, regenerated on the CPU: {rows} token rows in {times[0]:.1f} s"}
+    if "fused_lm_head" in line:      # the tensor-bound variant's figures once more, compact, at the very end of the line
+        f = line["fused_lm_head"]
+        line["fused_summary"] = {"ms_per_step": f["ms_per_step"], "frac": f["roofline"]["frac"], "peak": f["roofline"]["peak"],
+                                 "unit": "TFLOP/s", "achieved": f["roofline"]["achieved"], "steps": f["steps"],
+                                 "ms_per_step_row_blocks": f.get("ms_per_step_row_blocks_2048")}
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

@@ -51,6 +51,7 @@ def test_workspace_bytes(binding):
     assert binding.dppo_workspace_bytes(1) == 256 + 3 * 256
     assert binding.dppo_workspace_bytes(16384) == 256 + 3 * 65536
     assert binding.dppo_workspace_bytes(65) == 256 + 3 * 512
+    assert binding.dppo_workspace_bytes(65, 151936, 64, binding.TOPK_KL) == 256 + 3 * 512       # a function of T alone today
     assert binding.dppo_host_staging_bytes(0, 10, 0, 0) == 0
     a = binding.dppo_host_staging_bytes(128, 4096, 0, binding.BF16)
     b = binding.dppo_host_staging_bytes(128, 4096, 0, binding.BF16, dlogits_f32=True)
@@ -97,6 +98,15 @@ def test_misuse_is_rejected_before_launch(binding):
     assert _call(B, ws_bytes=100) == -8
     assert _call(B, dl=0x10000, opts=B.DppoOpts(0.0, B.DLOGITS_F32, 0, 0.0, 0.0)) == -9
     assert _call(B, dl=0x10000, ld_out=128) == -9
+    # dlogits may be the logits buffer itself (in place) or a disjoint one; any other overlap is refused, for every kernel
+    row = 64 * 2
+    for kern in (B.KERNEL_AUTO, B.KERNEL_GENERIC, B.KERNEL_RING):
+        o = B.DppoOpts(0.0, 0, kern, 0.0, 0.0)
+        assert _call(B, dl=0x10000 + row, opts=o) == -9         # shifted by one row
+        assert _call(B, dl=0x10000 + 3 * row + 32, opts=o) == -9    # starts inside the last row
+        assert _call(B, dl=0x10000 - 2 * row, opts=o) == -9     # ends inside the logits
+        assert _call(B, logits=0x10000, ld=128, dl=0x10000 + row, ld_out=128, opts=o) == -9   # interleaved rows of one allocation
+    assert _call(B, opts=B.DppoOpts(0.0, 0, 0, 0.0, 0.0, 0, 0, 0, -5)) == -11      # negative wait limit
     # forcing the bulk-copy kernel on a layout it cannot take
     assert _call(B, V=63, ld=63, ld_out=64, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0.0, 0.0)) == -7     # rows shifted differently
     assert _call(B, logits=0x10002, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0.0, 0.0)) == -7

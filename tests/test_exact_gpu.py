@@ -21,6 +21,11 @@ def _check(z, zm, tok=None, rows=None):
     out = dppo.dppo_exact_divergence(z, zm, tok)
     torch.cuda.synchronize()
     assert int(out["status"].item()) == 0
+    # without a TV output (tv = NULL) the second sweep is left out; KL and entropy are the same bits
+    one = dppo.dppo_exact_divergence(z, zm, tok, want_tv=False)
+    torch.cuda.synchronize()
+    assert int(one["status"].item()) == 0 and one["tv"] is None
+    assert torch.equal(one["kl"], out["kl"]) and torch.equal(one["entropy"], out["entropy"])
     T = z.shape[0]
     rows = range(T) if rows is None else rows
     zh, zmh = z.float().cpu().numpy().astype(np.float64), zm.float().cpu().numpy().astype(np.float64)
@@ -85,7 +90,7 @@ def test_exact_divergence_as_the_trust_region(which, delta, kernel):
     mu_logp = torch.log_softmax(zm.float(), 1).gather(1, a.long()[:, None])[:, 0].contiguous()
     adv = torch.where(torch.arange(T, device=DEV) % 2 == 0, 1.0, -0.5).to(torch.float32)
     tok = (torch.arange(T, device=DEV) % 6 != 4).to(torch.uint8)
-    ex = dppo.dppo_exact_divergence(z, zm, tok)
+    ex = dppo.dppo_exact_divergence(z, zm, tok, want_tv=(which == "tv"))
     code = dppo.KERNEL_RING if kernel == "ring" else dppo.KERNEL_GENERIC
     out = dppo.dppo_loss_fwd_bwd(z, a, mu_logp, adv, tok, dppo.GIVEN_D, 0, delta, kernel=code, given_divergence=ex[which],
                                  dlogits_f32=True)
@@ -105,3 +110,24 @@ def test_exact_divergence_as_the_trust_region(which, delta, kernel):
     binary = dppo.dppo_loss_fwd_bwd(z, a, mu_logp, adv, tok, dppo.BINARY_TV if which == "tv" else dppo.BINARY_KL, 0, delta, kernel=code)
     assert torch.all(out["mask"] <= binary["mask"])          # App. B: D_bin <= D_full, so the exact region blocks a superset
 
+
+
+def test_exact_kl_only_full_vocabulary_many_rows():
+    """The one-sweep mode (KL and entropy, no TV) on more rows than CTAs at V=151936: several rows per CTA back to back,
+    where the warps' partials of consecutive rows alternate between two buffers."""
+    T, V = 700, 151936
+    z, zm = _pair(T, V, torch.bfloat16, seed=77, noise=0.3)
+    tok = (torch.arange(T, device=DEV) % 9 != 4).to(torch.uint8)
+    one = dppo.dppo_exact_divergence(z, zm, tok, want_tv=False)
+    two = dppo.dppo_exact_divergence(z, zm, tok)
+    torch.cuda.synchronize()
+    assert int(one["status"].item()) == 0 and torch.equal(one["kl"], two["kl"]) and torch.equal(one["entropy"], two["entropy"])
+    rows = [0, 1, 147, 148, 149, 295, 296, 443, 592, 699]
+    zh, zmh = z[rows].float().cpu().numpy().astype(np.float64), zm[rows].float().cpu().numpy().astype(np.float64)
+    for i, t in enumerate(rows):
+        if tok[t].item() == 0:
+            assert one["kl"][t].item() == 0 and one["entropy"][t].item() == 0
+            continue
+        o_tv, o_kl, o_ent = O.exact_divergence_row(zh[i], zmh[i])
+        assert abs(one["kl"][t].item() - o_kl) <= 1e-5 and abs(one["entropy"][t].item() - o_ent) <= 2e-5 * max(1.0, o_ent)
+        assert abs(two["tv"][t].item() - o_tv) <= 1e-5
