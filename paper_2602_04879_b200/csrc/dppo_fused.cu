@@ -64,6 +64,9 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+constexpr int kMaxStreamKSms = 160;                         // SMs the partial-sum buffer of the workspace is sized for
+constexpr size_t kStreamKBytes = (size_t)kMaxStreamKSms * 2 * gemm::BM * gemm::BN * sizeof(float);
+
 template <int EPI, bool B_MN, int CG>
 cudaError_t launch_gemm_cg(const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
   using C = gemm::Cfg<CG>;
@@ -77,17 +80,10 @@ cudaError_t launch_gemm_cg(const void* A, int64_t lda, const void* B, int64_t ld
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int64_t ntiles = (int64_t)((p.M + C::TILE_M - 1) / C::TILE_M) * ((p.N + gemm::BN - 1) / gemm::BN);
-  p.sms = sms;
-  int max_splits = 1;
-  if (EPI == gemm::EPI_STORE_F32) max_splits = p.splits > 1 ? p.splits : (p.splits < 0 ? 2 : 1);
-  // partial sums are added into zeros; with a row map the rows that no tile row maps to stay zero
-  if (EPI == gemm::EPI_STORE_F32 && (max_splits > 1 || p.row_map)) {
-    cudaError_t ez = cudaMemset2DAsync(p.C, (size_t)p.ldc * sizeof(float), 0, (size_t)p.N * sizeof(float), (size_t)p.M, st);
-    if (ez != cudaSuccess) return ez;
-  }
-  const int64_t nunits = ntiles * max_splits;
   const int slots = sms / CG;                               // CTA groups that can be resident at once
-  const int groups = (int)(nunits < slots ? nunits : slots);
+  const int groups = (int)(ntiles < slots ? ntiles : slots);
+  // stream-K needs its partial-sum buffer to hold two tiles per group
+  if (EPI != gemm::EPI_STORE_F32 || p.c_transposed || p.accumulate || groups < 2 || groups * CG > kMaxStreamKSms) p.sk_part = nullptr;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(groups * CG));
   cfg.blockDim = dim3(gemm::THREADS);
@@ -98,7 +94,11 @@ cudaError_t launch_gemm_cg(const void* A, int64_t lda, const void* B, int64_t ld
   attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (CG > 1) ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, kernel, ma, mb, p);
+  e = cudaLaunchKernelEx(&cfg, kernel, ma, mb, p);
+  if (e != cudaSuccess || !p.sk_part) return e;
+  // the tiles of the partial wave: their partial sums are added up in a fixed order
+  gemm::gemm_streamk_fixup_kernel<CG><<<dim3((unsigned)(groups - 1), (unsigned)(C::TILE_M / 32)), 256, 0, st>>>(p, groups);
+  return cudaGetLastError();
 }
 
 // What every GEMM launch of a call takes from the caller's options.
@@ -301,6 +301,16 @@ __global__ void __launch_bounds__(1024) fused_partition_rows_kernel(const uint8_
   }
 }
 
+// dHidden rows of the tokens without a gradient (not valid, or zero advantage): zeros.  The rows with a gradient are
+// written by the dHidden GEMM through its row map.
+__global__ void __launch_bounds__(256) fused_zero_rows_kernel(const int32_t* pos, const int32_t* n_grad, float* out, int64_t d) {
+  const int64_t t = blockIdx.x;
+  const int ps = pos[t];
+  if (ps >= 0 && ps < *n_grad) return;
+  float4* row = reinterpret_cast<float4*>(out + t * d);
+  for (int64_t j = threadIdx.x; j < d / 4; j += blockDim.x) row[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
 // Row i of the compact copies = row idx[i] of the sources for i < *n; after that zeros (zero_fill) or left alone.
 struct GatherArgs {
   const int32_t* idx;
@@ -467,7 +477,7 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct FusedLayout {
   size_t wt, ht, hc, hr, E, psum, part, z_a, z_ar, z_topk, cref2, factor, c2, sgn, fix, ids_c, ids_r, idx, pos, idx_r, pos_r,
-      rescue, rmap, counts, loss_ws, total;
+      rescue, rmap, counts, loss_ws, skpart, total;
   int64_t lde, ldt;
   int tiles_n;
 };
@@ -503,6 +513,7 @@ FusedLayout fused_layout(int64_t T, int64_t d, int64_t V, int K) {
   L.rmap = take((size_t)T * 4);
   L.counts = take(4 * sizeof(int32_t));
   L.loss_ws = take(dppo_workspace_bytes(T, V, K, 0));
+  L.skpart = take(kStreamKBytes);                  // partial tiles of the dHidden GEMM (stream-K)
   L.total = off;
   return L;
 }
@@ -639,12 +650,14 @@ int fused_rows(const FusedCall& c, int64_t r0, int64_t Tb, bool first, bool last
     else DPPO_TRY((launch_gemm<gemm::EPI_GRAD, true>(go, ws + L.hr, d, Wb, V, gg, st)));
   }
   DPPO_TRY(launch_finalize(p, st, first, last));
-  // 6. dHidden[idx[i], :] = factor[i] * (E[i, :] . W[d, V]^T) for the rows with a gradient; the other rows stay zero.
-  //    Few output tiles, very long K: K is cut in two when that fills the waves better (two partial sums added into
-  //    zeros, in either order the same result).
+  // 6. dHidden[idx[i], :] = factor[i] * (E[i, :] . W[d, V]^T) for the rows with a gradient; the other rows are zero.
+  //    Few output tiles, very long K: the K iterations of the tiles that do not fill a whole wave of CTA groups are
+  //    dealt out evenly to all groups (stream-K) and their partial tiles added up in a fixed order.
+  fused_zero_rows_kernel<<<(unsigned)Tb, 256, 0, st>>>(I(L.pos), n_grad, c.dHidden + r0 * d, d);
+  DPPO_TRY(cudaGetLastError());
   gemm::Params g3 = {};
   g3.M = T; g3.N = (int)d; g3.K = (int)V; g3.C = c.dHidden + r0 * d; g3.ldc = d; g3.status = c.status;
-  g3.m_live = n_grad; g3.row_map = I(L.idx); g3.row_scale = F(L.factor); g3.splits = -1;
+  g3.m_live = n_grad; g3.row_map = I(L.idx); g3.row_scale = F(L.factor); g3.sk_part = F(L.skpart);
   g3.n_fastest = 1;      // d / 256 tiles along N: the CTAs of a wave then share each 2 V-byte row block of E instead of re-reading it
   if (vd) DPPO_TRY((launch_gemm<gemm::EPI_STORE_F32, true>(go, E, L.lde, Wb, d, g3, st)));     // B = W as [K = V, N = d], MN-major
   else DPPO_TRY(launch_gemm<gemm::EPI_STORE_F32>(go, E, L.lde, Wb, V, g3, st));                // B = W as [N = d, K = V], K-major

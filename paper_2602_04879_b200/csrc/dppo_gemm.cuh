@@ -55,9 +55,11 @@ struct Params {
   // EPI_STORE_F32
   float* C;
   int64_t ldc;
-  int splits;            // EPI_STORE_F32: K is cut into this many parts whose results are added into a zeroed C (0/1: none;
-                         // < 0: two parts when that fills the waves of `sms` CTAs better, decided from the live tile count)
-  int sms;               // CTAs the split decision assumes (splits < 0)
+  float* sk_part;        // EPI_STORE_F32 (no transposed store, no accumulation): when the tiles do not fill whole waves of
+                         // CTA groups, the K iterations of the tiles of the last, partial wave are dealt out evenly to
+                         // all groups; each group leaves at most two partial tiles here ([2 * groups] slots of
+                         // TILE_M x BN floats), which gemm_streamk_fixup_kernel adds up in a fixed order.  null: whole
+                         // tiles only
   // Live extents, read from device memory at kernel start (null: the static M / K).  Rows of A at and beyond *m_live
   // get no output tile (at least one tile is always processed); K blocks at and beyond *k_live are not read (at least
   // one is), so the operands must hold zeros from *k_live to the end of that block.
@@ -187,6 +189,53 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// The list of work units of one CTA group.  First its whole tiles (tile = group, group + ngroups, ...).  With stream-K
+// (store epilogue with a partial-sum buffer) the whole tiles are those of the full waves only, and the K iterations of
+// the remaining tiles (fewer than there are groups) are dealt out evenly: group g takes the iterations
+// [g * ipg, (g + 1) * ipg) of the sequence (tile, k block), which touches at most two tiles; each such piece is a unit
+// whose accumulator goes to the partial-sum slot 2 * g + piece instead of C.
+struct Plan {
+  int whole;            // whole-tile units of this group
+  int pieces;           // 0, 1 or 2 partial units after them
+  int first_sk_tile;    // tile index of the first tile of the partial wave
+  int sk_tiles;         // tiles of the partial wave (0: no stream-K)
+  int ipg;              // K iterations per group in the partial wave
+  int lo, hi;           // this group's iterations of the partial wave
+  int kblocks, group, ngroups;
+  __device__ __forceinline__ int units() const { return whole + pieces; }
+  // unit i -> tile, K blocks [kb0, kb1), partial-sum slot (-1: the result goes to C)
+  __device__ __forceinline__ void unit(int i, int& tile, int& kb0, int& kb1, int& slot) const {
+    if (i < whole) { tile = group + i * ngroups; kb0 = 0; kb1 = kblocks; slot = -1; return; }
+    const int pc = i - whole, t0 = lo / kblocks;
+    if (pc == 0) { tile = t0; kb0 = lo - t0 * kblocks; kb1 = (hi - t0 * kblocks < kblocks) ? hi - t0 * kblocks : kblocks; }
+    else { tile = t0 + 1; kb0 = 0; kb1 = hi - (t0 + 1) * kblocks; }
+    tile += first_sk_tile;
+    slot = 2 * group + pc;
+  }
+};
+template <int CG>
+__device__ __forceinline__ Plan make_plan(bool allow_sk, int ntiles, int kblocks, int group, int ngroups) {
+  Plan pl;
+  pl.kblocks = kblocks; pl.group = group; pl.ngroups = ngroups;
+  const int full_waves = ntiles / ngroups, rem = ntiles - full_waves * ngroups;
+  // worth it when the partial wave would leave a tenth or more of the groups idle and K is long
+  const bool sk = allow_sk && rem > 0 && rem * 10 <= ngroups * 9 && kblocks >= 8 && (long long)rem * kblocks < (1ll << 30);
+  pl.sk_tiles = sk ? rem : 0;
+  pl.first_sk_tile = full_waves * ngroups;
+  pl.pieces = 0; pl.ipg = 0; pl.lo = pl.hi = 0;
+  if (!sk) {
+    pl.whole = group < ntiles ? (ntiles - group + ngroups - 1) / ngroups : 0;
+    return pl;
+  }
+  pl.whole = full_waves;
+  const int total = rem * kblocks;
+  pl.ipg = (total + ngroups - 1) / ngroups;          // rem < ngroups, so ipg <= kblocks: a range touches at most two tiles
+  pl.lo = group * pl.ipg < total ? group * pl.ipg : total;
+  pl.hi = pl.lo + pl.ipg < total ? pl.lo + pl.ipg : total;
+  if (pl.lo < pl.hi) pl.pieces = (pl.lo / kblocks != (pl.hi - 1) / kblocks) ? 2 : 1;
+  return pl;
+}
+
 // B_MN = false: B given as [N, K] (K contiguous).  B_MN = true: B given as [K, N] (N contiguous, "NN" product); its tile is
 // then loaded as boxes of 64 columns x 64 k-rows.  CG = 2: launched as clusters of two CTAs (see the top of the file).
 template <int EPI, bool B_MN, int CG>
@@ -240,20 +289,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   const int tiles_m = m_lim > 0 ? (m_lim + C::TILE_M - 1) / C::TILE_M : (p.allow_empty ? 0 : 1), tiles_n = (p.N + BN - 1) / BN;
   const int ntiles = tiles_m * tiles_n;
   const int kblocks = k_lim > 0 ? (k_lim + BK - 1) / BK : 1;
-  // work unit u = part * ntiles + tile: all tiles of one K part are in flight together and share operand strips
-  int splits = 1;
-  if (EPI == EPI_STORE_F32) {
-    if (p.splits > 1) splits = p.splits;
-    else if (p.splits < 0 && p.sms > 0 && kblocks >= 8) {
-      // few output tiles, very long K: cut K in two when the halves fill whole waves of CTA groups better
-      const int slots = p.sms / CG;
-      const float w1 = (float)ntiles / (float)(((ntiles + slots - 1) / slots) * slots);
-      const float w2 = (float)(2 * ntiles) / (float)(((2 * ntiles + slots - 1) / slots) * slots);
-      if (w2 > w1 + 0.05f) splits = 2;
-    }
-  }
-  const int kper = (kblocks + splits - 1) / splits;
-  const int nunits = ntiles * splits;
+  const Plan pl = make_plan<CG>(EPI == EPI_STORE_F32 && p.sk_part != nullptr, ntiles, kblocks, group, ngroups);
   const uint32_t smem_base = smem_u32(smem);
 
   if (warp == 0) {
@@ -263,11 +299,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int u = group; u < nunits && ok; u += ngroups) {
-        const int tile = u % ntiles, part = u / ntiles;
+      for (int u = 0; u < pl.units() && ok; ++u) {
+        int tile, kb0, kb1, slot;
+        pl.unit(u, tile, kb0, kb1, slot);
         const int tm = p.n_fastest ? tile / tiles_n : tile % tiles_m, tn = p.n_fastest ? tile % tiles_n : tile / tiles_m;
         const int m0 = tm * C::TILE_M + (int)rank * BM, n0 = tn * BN + (int)rank * C::B_COLS;
-        const int kb0 = part * kper, kb1 = (kb0 + kper < kblocks) ? kb0 + kper : kblocks;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, wc)) { ok = false; break; }
           const uint32_t a_dst = smem_base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
@@ -305,9 +341,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       uint32_t it = 0;
       bool ok = true;
       constexpr uint32_t idesc = make_idesc(CG, B_MN);
-      for (int u = group; u < nunits && ok; u += ngroups, ++it) {
-        const int part = u / ntiles;
-        const int kb0 = part * kper, kb1 = (kb0 + kper < kblocks) ? kb0 + kper : kblocks;
+      for (int u = 0; u < pl.units() && ok; ++u, ++it) {
+        int tile, kb0, kb1, slot;
+        pl.unit(u, tile, kb0, kb1, slot);
         const uint32_t b = it & 1u, use = it >> 1;
         if (!mbar_wait(tempty0 + 8 * b, (use & 1u) ^ 1u, wc)) { ok = false; break; }   // epilogues drained this buffer
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -336,8 +372,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
     // ------------------------------------------------------------------ epilogue warps (TMEM lane quarter = warp % 4)
     const int q = warp & 3;
     uint32_t it = 0;
-    for (int u = group; u < nunits; u += ngroups, ++it) {
-      const int tile = u % ntiles;
+    for (int u = 0; u < pl.units(); ++u, ++it) {
+      int tile, kb0, kb1, slot;
+      pl.unit(u, tile, kb0, kb1, slot);
       const int tm = p.n_fastest ? tile / tiles_n : tile % tiles_m, nb = p.n_fastest ? tile % tiles_n : tile / tiles_m;
       const int m0 = tm * C::TILE_M + (int)rank * BM, n0 = nb * BN;
       const uint32_t b = it & 1u, use = it >> 1;
@@ -349,7 +386,17 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
       // a later GEMM and must hold finite values), unless the gradient rows go through a row map
       const bool row_ok = (EPI == EPI_STORE_F32 || (EPI == EPI_GRAD && p.p_row_map)) ? row < m_lim : row < p.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * BN;
-      if (EPI == EPI_STORE_F32) {
+      if (EPI == EPI_STORE_F32 && slot >= 0) {
+        // a piece of a tile's K range: the raw partial sums of this CTA's 128 rows go to the group's slot
+        float* dst = p.sk_part + ((int64_t)slot * C::TILE_M + (int)rank * BM + q * 32 + lane) * BN;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) *reinterpret_cast<uint4*>(dst + c + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+        }
+      } else if (EPI == EPI_STORE_F32) {
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
           uint32_t r[32];
@@ -385,9 +432,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
 #pragma unroll
                 for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) dst[j] += __uint_as_float(r[j]);
               }
-            } else if (splits > 1) {       // partial sum over a K part: add into the zeroed output
-#pragma unroll
-              for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) atomicAdd(dst + j, __uint_as_float(r[j]));
             } else if (n0 + c + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
 #pragma unroll
               for (int j = 0; j < 32; j += 4) *reinterpret_cast<uint4*>(dst + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
@@ -535,6 +579,47 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (CG == 2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// Second half of stream-K: adds up the partial tiles that gemm_tn_kernel<EPI_STORE_F32> left in p.sk_part, group after
+// group (a fixed order: the result does not depend on timing), applies the row factor and the row map and stores the
+// tile.  Launch with the same Params and the same number of CTA groups; grid = (ngroups - 1, TILE_M / 32), 256 threads.
+template <int CG>
+__global__ void __launch_bounds__(256) gemm_streamk_fixup_kernel(Params p, int ngroups) {
+  using C = Cfg<CG>;
+  int m_lim = p.M, k_lim = p.K;
+  if (p.m_live) { const int v = *p.m_live; m_lim = v < 0 ? 0 : (v < p.M ? v : p.M); }
+  if (p.k_live) { const int v = *p.k_live; k_lim = v < 0 ? 0 : (v < p.K ? v : p.K); }
+  const int tiles_m = m_lim > 0 ? (m_lim + C::TILE_M - 1) / C::TILE_M : (p.allow_empty ? 0 : 1), tiles_n = (p.N + BN - 1) / BN;
+  const int ntiles = tiles_m * tiles_n;
+  const int kblocks = k_lim > 0 ? (k_lim + BK - 1) / BK : 1;
+  const Plan pl = make_plan<CG>(p.sk_part != nullptr, ntiles, kblocks, 0, ngroups);
+  const int r = blockIdx.x;                             // tile of the partial wave
+  if (r >= pl.sk_tiles) return;
+  const int tile = pl.first_sk_tile + r;
+  const int tm = p.n_fastest ? tile / tiles_n : tile % tiles_m, nb = p.n_fastest ? tile % tiles_n : tile / tiles_m;
+  const int g0 = (r * kblocks) / pl.ipg, g1 = ((r + 1) * kblocks - 1) / pl.ipg;      // groups whose ranges meet this tile
+  const int lrow = blockIdx.y * 32 + (threadIdx.x >> 3);                              // row of the tile: 32 rows per block,
+  const int row = tm * C::TILE_M + lrow;                                              // 8 threads per row
+  if (row >= m_lim) return;
+  const float sc = p.row_scale ? p.row_scale[row] : 1.f;
+  float* out = p.C + (int64_t)(p.row_map ? p.row_map[row] : row) * p.ldc + nb * BN;
+  for (int c4 = (threadIdx.x & 7); c4 < BN / 4; c4 += 8) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int g = g0; g <= g1; ++g) {
+      const int pc = ((g * pl.ipg) / kblocks == r) ? 0 : 1;       // the group's first piece lies in this tile, or its second
+      const float4 v = *reinterpret_cast<const float4*>(p.sk_part + ((int64_t)(2 * g + pc) * C::TILE_M + lrow) * BN + 4 * c4);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    acc.x *= sc; acc.y *= sc; acc.z *= sc; acc.w *= sc;
+    const int col = nb * BN + 4 * c4;
+    if (col + 4 <= p.N && ((reinterpret_cast<uintptr_t>(out + 4 * c4) & 15) == 0)) {
+      *reinterpret_cast<float4*>(out + 4 * c4) = acc;
+    } else {
+      const float a4[4] = {acc.x, acc.y, acc.z, acc.w};
+      for (int j = 0; j < 4; ++j) if (col + j < p.N) out[4 * c4 + j] = a4[j];
+    }
   }
 }
 

@@ -215,13 +215,15 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         // sum over the other entries and keeps its relative accuracy when pi(a) is close to 1)
         float ref = -INFINITY, nm = 0.f, s = 0.f;
         const RowGeom gm = row_geom<InT, SH>(p, t, row_bytes, C);
-        const uint32_t a_img = (uint32_t)meta + gm.head / (uint32_t)sizeof(InT);   // the sampled token's place in the image
+        constexpr uint32_t kChunkElems = kChunkBytes / sizeof(InT);
+        const uint32_t a_img = (uint32_t)meta + gm.head / (uint32_t)sizeof(InT);   // the sampled token's place in the image,
+        const int a_chunk = (int)(a_img / kChunkElems);                            // the chunk that holds it
+        const uint32_t a_loc = a_img % kChunkElems;                                // and its place in that chunk
         for (int c = 0; c < gm.C; ++c) {
           const bool ok = mbar_wait_warp(full_base + 8u * pos.slot, pos.phase, wc);
           const uint32_t cbase = (uint32_t)c * kChunkBytes;
           const uint32_t sbase = slots_base + (uint32_t)pos.slot * kChunkBytes;
-          const uint32_t a_loc = a_img - cbase / (uint32_t)sizeof(InT);            // its place in this chunk (if below the chunk's size)
-          const bool has_a = a_loc < (uint32_t)(kChunkBytes / sizeof(InT));        // warp-uniform
+          const bool has_a = (c == a_chunk);                                       // warp-uniform
           if (ok) {
             // chunks that the bulk copy filled completely take the straight-line path
             const bool full_chunk = cbase + (uint32_t)kChunkBytes <= gm.xa;
