@@ -127,6 +127,10 @@ def bench_fused(dppo, wl, dev, steps=40, warmup=10, T=8192):
     ms_blocks = _time_steps(torch, fn_b, steps, warmup)
     ws_bytes, ws_b_bytes = ws.numel(), ws_b.numel()
     del ws_b
+    # the two-pass mode (each logits tile computed twice, dW with one bf16 rounding instead of two)
+    fn_2 = lambda: dppo.dppo_fused_lmhead_fwd_bwd(b.hidden, b.lm_head, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.BINARY_TV, DELTA,
+                                                  workspace=ws, dHidden=dH, dW=dW, status=status, two_pass=True)
+    ms_two_pass = _time_steps(torch, fn_2, steps, warmup)
     peak, src = measured_tensor_peak()
     useful = 6.0 * T * d * V / (ms * 1e-3) / 1e12          # forward + dHidden + dW; every logits tile is computed once
     return {"workload": ("" if T == 8192 else f"REDUCED to {T} rows (profiling case): ") + "fused_lm_head_binary_tv: hidden [8192,2048] bf16 x W [2048,151936] bf16, delta=0.2",
@@ -134,10 +138,10 @@ def bench_fused(dppo, wl, dev, steps=40, warmup=10, T=8192):
             "roofline": {"bound": "tensor", "achieved": useful, "peak": peak, "unit": "TFLOP/s", "frac": useful / peak,
                          "traffic": None, "peak_source": "of " + src,
                          "flop_count": "6*T*d*V (forward, dHidden, dW); nothing is recomputed"},
-            "gpu_launches_per_step": 15, "loss": float(out["loss"].item()),
+            "gpu_launches_per_step": 17, "loss": float(out["loss"].item()),
             "ms_per_step_quarter_of_responses_zero_advantage": ms_sparse, "ms_per_step_topk_tv_k20": ms_topk,
             "ms_per_step_lm_head_vocab_major": ms_vd,
-            "ms_per_step_row_blocks_2048": ms_blocks, "workspace_bytes": ws_bytes, "workspace_bytes_row_blocks_2048": ws_b_bytes}
+            "ms_per_step_row_blocks_2048": ms_blocks, "ms_per_step_two_pass": ms_two_pass, "workspace_bytes": ws_bytes, "workspace_bytes_row_blocks_2048": ws_b_bytes}
 
 
 def _time_steps(torch, fn, steps, warmup):

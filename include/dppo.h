@@ -124,6 +124,10 @@ typedef struct dppo_opts {
                           and sets DPPO_STATUS_WAIT_LIMIT, in microseconds; 0 = about 2 s.  Waits normally take
                           microseconds; the limit only bounds the damage of a lost copy */
   int test_inject;     /* DPPO_INJECT_* bits, testing only; 0 in production                                          */
+  int fused_two_pass;  /* dppo_fused_lmhead_fwd_bwd only: 1 = every row takes the two-pass route (statistics GEMM, then a
+                          second GEMM over the same tiles that writes the finished bf16 gradient), which rounds dlogits once,
+                          so that dW carries one bf16 rounding instead of two (|error| <= 2^-8 |hidden|^T |dlogits|), at the
+                          price of computing every logits tile twice (about a third more time); 0 = single pass          */
 } dppo_opts;
 enum { DPPO_LM_HEAD_DV = 0, DPPO_LM_HEAD_VD = 1 };
 

@@ -29,13 +29,14 @@ class DppoOpts(ctypes.Structure):
     """dppo_opts of include/dppo.h (all-zero = defaults)."""
     _fields_ = [("loss_scale", c_float), ("dlogits_dtype", c_int), ("kernel", c_int), ("is_cap", c_float), ("eps_low", c_float),
                 ("lm_head_layout", c_int), ("gemm_cta_group", c_int), ("fused_rows_per_block", c_int), ("wait_limit_us", c_int),
-                ("test_inject", c_int)]
+                ("test_inject", c_int), ("fused_two_pass", c_int)]
 
 
 def _opts(loss_scale=0.0, dlogits_f32=False, kernel=KERNEL_AUTO, is_cap=0.0, eps_low=0.0, w_is_vd=False, cta_group=0,
-          rows_per_block=0, wait_limit_us=0, test_inject=0):
+          rows_per_block=0, wait_limit_us=0, test_inject=0, two_pass=False):
     return DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), float(is_cap), float(eps_low),
-                    1 if w_is_vd else 0, int(cta_group), int(rows_per_block), int(wait_limit_us), int(test_inject))
+                    1 if w_is_vd else 0, int(cta_group), int(rows_per_block), int(wait_limit_us), int(test_inject),
+                    1 if two_pass else 0)
 
 
 class DppoError(RuntimeError):
@@ -171,12 +172,12 @@ def dppo_fused_workspace_bytes(T, d, V, K=0):
 def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, delta=0.2,
                               loss_scale=0.0, want_stats=False, workspace=None, dHidden=None, dW=None, status=None, stream=None,
                               is_cap=0.0, eps_low=0.0, K=0, mu_topk_ids=None, mu_topk_p=None, given_divergence=None, w_is_vd=False,
-                              cta_group=0, rows_per_block=0, wait_limit_us=0, test_inject=0):
+                              cta_group=0, rows_per_block=0, wait_limit_us=0, test_inject=0, two_pass=False):
     """Calls ``dppo_fused_lmhead_fwd_bwd`` on CUDA tensors: hidden [T,d] bf16, W [d,V] bf16.  Returns
     dict(loss[1], divergence[T], mask[T], dHidden[T,d] fp32, dW[d,V] fp32, stats, status); nothing is synchronised.
     ``given_divergence``: as for ``dppo_loss_fwd_bwd`` (variant GIVEN_D).  ``w_is_vd``: W (and dW) are [V,d], the layout
     of a linear layer's weight, instead of [d,V].  ``cta_group``, ``rows_per_block``, ``wait_limit_us``, ``test_inject``: the
-    fields of dppo_opts of the same names (``rows_per_block`` = fused_rows_per_block)."""
+    fields of dppo_opts of the same names (``rows_per_block`` = fused_rows_per_block, ``two_pass`` = fused_two_pass)."""
     assert hidden.is_cuda and W.is_cuda and hidden.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
     assert hidden.is_contiguous() and W.is_contiguous() and hidden.shape[1] == W.shape[1 if w_is_vd else 0]
     T, d = hidden.shape
@@ -195,7 +196,7 @@ def dppo_fused_lmhead_fwd_bwd(hidden, W, sampled_ids, mu_logp, advantages, token
     if workspace is None:
         rows = min(T, rows_per_block) if rows_per_block > 0 else T
         workspace = torch.empty(dppo_fused_workspace_bytes(rows, d, V, K), dtype=torch.uint8, device=dev)
-    opts = _opts(loss_scale, False, 0, is_cap, eps_low, w_is_vd, cta_group, rows_per_block, wait_limit_us, test_inject)
+    opts = _opts(loss_scale, False, 0, is_cap, eps_low, w_is_vd, cta_group, rows_per_block, wait_limit_us, test_inject, two_pass)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     with torch.cuda.device(dev):
         rc = lib().dppo_fused_lmhead_fwd_bwd(_ptr(hidden), _ptr(W), T, d, V, _ptr(sampled_ids), _ptr(mu_logp),

@@ -311,6 +311,16 @@ __global__ void __launch_bounds__(256) fused_zero_rows_kernel(const int32_t* pos
   for (int64_t j = threadIdx.x; j < d / 4; j += blockDim.x) row[j] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
+// Two-pass mode: the rows of E from *n_grad up to the end of that block of 64 rows are read by the dW GEMM's last K block
+// (against zeros) and written by nobody else unless they belong to valid rows: zeros.
+__global__ void __launch_bounds__(256) fused_zero_e_tail_kernel(__nv_bfloat16* E, int64_t lde, const int32_t* n_grad, int64_t T) {
+  const int64_t r = (int64_t)*n_grad + blockIdx.x;
+  const int64_t end = ((int64_t)*n_grad + 63) / 64 * 64;
+  if (r >= end || r >= T) return;
+  uint4* row = reinterpret_cast<uint4*>(E + r * lde);
+  for (int64_t j = threadIdx.x; j < lde / 8; j += blockDim.x) row[j] = make_uint4(0, 0, 0, 0);
+}
+
 // Row i of the compact copies = row idx[i] of the sources for i < *n; after that zeros (zero_fill) or left alone.
 struct GatherArgs {
   const int32_t* idx;
@@ -346,6 +356,7 @@ struct ExpArgs {
   int32_t* rescue;          // [T] 1: the row goes through the two-pass kernels
   __nv_bfloat16* E;
   int64_t lde;
+  int force_two_pass;       // every valid row goes through the two-pass kernels (psum, z_a, cref2 are not read)
 };
 
 // Sums of exp(z - c) above this, or not finite, or not positive, send a row to the two-pass kernels: E and the row
@@ -366,7 +377,9 @@ __global__ void __launch_bounds__(256) fused_scalar_exp_kernel(RowParams p, ExpA
   float D = 0.f, r = 0.f, absdiff = 0.f, factor = 0.f;
   int M = 0;
   double g = 0.0;
-  if (valid) {
+  if (valid && x.force_two_pass) {
+    resc = 1;
+  } else if (valid) {
     double S_o = 0.0;                                   // over the entries other than the sampled token's
     for (int i = lane; i < x.tiles_n; i += 32) S_o += (double)x.psum[ts * x.tiles_n + i];
     S_o = warp_sum(S_o);
@@ -595,8 +608,11 @@ int fused_rows(const FusedCall& c, int64_t r0, int64_t Tb, bool first, bool last
     fused_gather_rows_kernel<<<(unsigned)Tb, 256, 0, st>>>(ga);
     DPPO_TRY(cudaGetLastError());
   }
+  const bool two_pass = c.o.fused_two_pass != 0;
   // 2. reference exponent of every packed row
-  if (c.wt)      // W^T is there: contiguous rows instead of strided columns (rows past the valid ones are zero: reference 0)
+  if (two_pass) {
+    fused_zero_e_tail_kernel<<<64, 256, 0, st>>>(E, L.lde, n_grad, Tb);
+  } else if (c.wt)      // W^T is there: contiguous rows instead of strided columns (rows past the valid ones are zero: reference 0)
     fused_topk_logits_kernel<<<row_warps, 256, 0, st>>>(hc, c.wt, Tb, d, V, I(L.ids_c), 1, F(L.cref2), kLog2e);
   else
     fused_ref_logit_kernel<<<row_warps, 256, 0, st>>>(hc, Wb, Tb, d, V, I(L.ids_c), n_valid, F(L.cref2));
@@ -606,7 +622,8 @@ int fused_rows(const FusedCall& c, int64_t r0, int64_t Tb, bool first, bool last
   gemm::Params g1 = {};
   g1.M = T; g1.N = (int)V; g1.K = (int)d; g1.psum = F(L.psum); g1.z_a = F(L.z_a); g1.ids = I(L.ids_c); g1.cref2 = F(L.cref2);
   g1.P = E; g1.ldp = L.lde; g1.status = c.status; g1.m_live = n_valid; g1.e_live = n_grad;
-  if (vd) DPPO_TRY((launch_gemm<gemm::EPI_EXP, false>(go, hc, d, Wb, d, g1, st)));     // B = W [V, d], K-major
+  if (two_pass) { /* every row is handled by step 5 */ }
+  else if (vd) DPPO_TRY((launch_gemm<gemm::EPI_EXP, false>(go, hc, d, Wb, d, g1, st)));     // B = W [V, d], K-major
   else DPPO_TRY((launch_gemm<gemm::EPI_EXP, true>(go, hc, d, Wb, V, g1, st)));         // B = W [d, V], MN-major
   // 4. per-row scalars
   float* z_topk = nullptr;
@@ -619,6 +636,7 @@ int fused_rows(const FusedCall& c, int64_t r0, int64_t Tb, bool first, bool last
     ExpArgs x = {};
     x.psum = F(L.psum); x.tiles_n = L.tiles_n; x.z_a = F(L.z_a); x.cref2 = F(L.cref2); x.pos = I(L.pos); x.n_grad = n_grad;
     x.z_topk = z_topk; x.row_factor = F(L.factor); x.rescue = I(L.rescue); x.E = E; x.lde = L.lde;
+    x.force_two_pass = two_pass ? 1 : 0;
     fused_scalar_exp_kernel<<<row_warps, 256, 0, st>>>(p, x);
     DPPO_TRY(cudaGetLastError());
   }
@@ -732,6 +750,7 @@ int dppo_fused_lmhead_fwd_bwd(const void* hidden, const void* W, int64_t T, int6
   if (((uintptr_t)dHidden % 16) || ((uintptr_t)dW % 16)) return DPPO_ERR_ALIGN;
   if (o.lm_head_layout != DPPO_LM_HEAD_DV && o.lm_head_layout != DPPO_LM_HEAD_VD) return DPPO_ERR_UNSUPPORTED;
   if (o.gemm_cta_group < 0 || o.gemm_cta_group > 2 || o.wait_limit_us < 0 || o.fused_rows_per_block < 0) return DPPO_ERR_UNSUPPORTED;
+  if (o.fused_two_pass != 0 && o.fused_two_pass != 1) return DPPO_ERR_UNSUPPORTED;
   const bool vd = (o.lm_head_layout == DPPO_LM_HEAD_VD);
   // row-block mode: the rows are finished block by block and the workspace is sized for one block
   const int64_t Tb_max = (o.fused_rows_per_block > 0 && (int64_t)o.fused_rows_per_block < T) ? (int64_t)o.fused_rows_per_block : T;
