@@ -65,7 +65,7 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
 }
 
 constexpr int kMaxStreamKSms = 160;                         // SMs the partial-sum buffer of the workspace is sized for
-constexpr size_t kStreamKBytes = (size_t)kMaxStreamKSms * 2 * gemm::BM * gemm::BN * sizeof(float);
+constexpr size_t kStreamKBytes = (size_t)kMaxStreamKSms * gemm::kMaxSegs * gemm::BM * gemm::BN * sizeof(float);
 
 template <int EPI, bool B_MN, int CG>
 cudaError_t launch_gemm_cg(const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
@@ -82,7 +82,7 @@ cudaError_t launch_gemm_cg(const void* A, int64_t lda, const void* B, int64_t ld
   const int64_t ntiles = (int64_t)((p.M + C::TILE_M - 1) / C::TILE_M) * ((p.N + gemm::BN - 1) / gemm::BN);
   const int slots = sms / CG;                               // CTA groups that can be resident at once
   const int groups = (int)(ntiles < slots ? ntiles : slots);
-  // stream-K needs its partial-sum buffer to hold two tiles per group
+  // the K split of the last wave needs its partial-sum buffer to hold kMaxSegs tiles per group
   if (EPI != gemm::EPI_STORE_F32 || p.c_transposed || p.accumulate || groups < 2 || groups * CG > kMaxStreamKSms) p.sk_part = nullptr;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(groups * CG));
@@ -526,7 +526,7 @@ FusedLayout fused_layout(int64_t T, int64_t d, int64_t V, int K) {
   L.rmap = take((size_t)T * 4);
   L.counts = take(4 * sizeof(int32_t));
   L.loss_ws = take(dppo_workspace_bytes(T, V, K, 0));
-  L.skpart = take(kStreamKBytes);                  // partial tiles of the dHidden GEMM (stream-K)
+  L.skpart = take(kStreamKBytes);                  // partial tiles of the dHidden GEMM (K split of its last wave)
   L.total = off;
   return L;
 }
@@ -669,8 +669,8 @@ int fused_rows(const FusedCall& c, int64_t r0, int64_t Tb, bool first, bool last
   }
   DPPO_TRY(launch_finalize(p, st, first, last));
   // 6. dHidden[idx[i], :] = factor[i] * (E[i, :] . W[d, V]^T) for the rows with a gradient; the other rows are zero.
-  //    Few output tiles, very long K: the K iterations of the tiles that do not fill a whole wave of CTA groups are
-  //    dealt out evenly to all groups (stream-K) and their partial tiles added up in a fixed order.
+  //    Few output tiles, very long K: the tiles that do not fill a whole wave of CTA groups are cut along K into
+  //    segments that do, and their partial tiles are added up in a fixed order.
   fused_zero_rows_kernel<<<(unsigned)Tb, 256, 0, st>>>(I(L.pos), n_grad, c.dHidden + r0 * d, d);
   DPPO_TRY(cudaGetLastError());
   gemm::Params g3 = {};

@@ -56,9 +56,9 @@ struct Params {
   float* C;
   int64_t ldc;
   float* sk_part;        // EPI_STORE_F32 (no transposed store, no accumulation): when the tiles do not fill whole waves of
-                         // CTA groups, the K iterations of the tiles of the last, partial wave are dealt out evenly to
-                         // all groups; each group leaves at most two partial tiles here ([2 * groups] slots of
-                         // TILE_M x BN floats), which gemm_streamk_fixup_kernel adds up in a fixed order.  null: whole
+                         // CTA groups, the tiles of the last, partial wave are cut along K into up to kMaxSegs segments
+                         // that are dealt to all groups; their partial tiles land here ([kMaxSegs * groups] slots of
+                         // TILE_M x BN floats) and gemm_streamk_fixup_kernel adds them up in a fixed order.  null: whole
                          // tiles only
   // Live extents, read from device memory at kernel start (null: the static M / K).  Rows of A at and beyond *m_live
   // get no output tile (at least one tile is always processed); K blocks at and beyond *k_live are not read (at least
@@ -189,28 +189,29 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// The list of work units of one CTA group.  First its whole tiles (tile = group, group + ngroups, ...).  With stream-K
-// (store epilogue with a partial-sum buffer) the whole tiles are those of the full waves only, and the K iterations of
-// the remaining tiles (fewer than there are groups) are dealt out evenly: group g takes the iterations
-// [g * ipg, (g + 1) * ipg) of the sequence (tile, k block), which touches at most two tiles; each such piece is a unit
-// whose accumulator goes to the partial-sum slot 2 * g + piece instead of C.
+// The list of work units of one CTA group.  First its whole tiles (tile = group, group + ngroups, ...).  With a
+// partial-sum buffer (store epilogue) the whole tiles are those of the full waves only, and the remaining tiles (fewer
+// than there are groups) are cut along K into `segs` equal segments: units (segment, tile), segment-major, dealt
+// round-robin to the groups.  All units in flight at a time then belong to one or two segments and walk K in step, so
+// that tiles of one row or column of the output still share their operand strips through L2; more segments fill the
+// last wave better.  A segment's accumulator goes to the partial-sum slot tile * segs + segment instead of C.
+constexpr int kMaxSegs = 8;
 struct Plan {
   int whole;            // whole-tile units of this group
-  int pieces;           // 0, 1 or 2 partial units after them
+  int sk_units;         // (segment, tile) units of this group after them
   int first_sk_tile;    // tile index of the first tile of the partial wave
-  int sk_tiles;         // tiles of the partial wave (0: no stream-K)
-  int ipg;              // K iterations per group in the partial wave
-  int lo, hi;           // this group's iterations of the partial wave
+  int sk_tiles;         // tiles of the partial wave (0: none is cut)
+  int segs, kseg;       // segments per tile, K blocks per segment
   int kblocks, group, ngroups;
-  __device__ __forceinline__ int units() const { return whole + pieces; }
+  __device__ __forceinline__ int units() const { return whole + sk_units; }
   // unit i -> tile, K blocks [kb0, kb1), partial-sum slot (-1: the result goes to C)
   __device__ __forceinline__ void unit(int i, int& tile, int& kb0, int& kb1, int& slot) const {
     if (i < whole) { tile = group + i * ngroups; kb0 = 0; kb1 = kblocks; slot = -1; return; }
-    const int pc = i - whole, t0 = lo / kblocks;
-    if (pc == 0) { tile = t0; kb0 = lo - t0 * kblocks; kb1 = (hi - t0 * kblocks < kblocks) ? hi - t0 * kblocks : kblocks; }
-    else { tile = t0 + 1; kb0 = 0; kb1 = hi - (t0 + 1) * kblocks; }
-    tile += first_sk_tile;
-    slot = 2 * group + pc;
+    const int j = group + (i - whole) * ngroups, seg = j / sk_tiles, r = j - seg * sk_tiles;
+    tile = first_sk_tile + r;
+    kb0 = seg * kseg;
+    kb1 = kb0 + kseg < kblocks ? kb0 + kseg : kblocks;
+    slot = r * segs + seg;
   }
 };
 template <int CG>
@@ -218,21 +219,29 @@ __device__ __forceinline__ Plan make_plan(bool allow_sk, int ntiles, int kblocks
   Plan pl;
   pl.kblocks = kblocks; pl.group = group; pl.ngroups = ngroups;
   const int full_waves = ntiles / ngroups, rem = ntiles - full_waves * ngroups;
-  // worth it when the partial wave would leave a tenth or more of the groups idle and K is long
-  const bool sk = allow_sk && rem > 0 && rem * 10 <= ngroups * 9 && kblocks >= 8 && (long long)rem * kblocks < (1ll << 30);
-  pl.sk_tiles = sk ? rem : 0;
   pl.first_sk_tile = full_waves * ngroups;
-  pl.pieces = 0; pl.ipg = 0; pl.lo = pl.hi = 0;
-  if (!sk) {
+  pl.sk_tiles = 0; pl.sk_units = 0; pl.segs = 1; pl.kseg = kblocks;
+  // time of the partial wave with s segments, in tile times: ceil(rem * s / ngroups) / s; the smallest s within 2 % of
+  // the best, and only if that saves 5 % of a tile time or more
+  int best = 1;
+  if (allow_sk && rem > 0) {
+    float tbest = 1.f;
+    for (int sgs = 2; sgs <= kMaxSegs && kblocks >= 8 * sgs; ++sgs) {
+      const float t = (float)((rem * sgs + ngroups - 1) / ngroups) / (float)sgs;
+      if (t < 0.98f * tbest) { tbest = t; best = sgs; }
+    }
+    if (tbest > 0.95f) best = 1;
+  }
+  if (best == 1) {
     pl.whole = group < ntiles ? (ntiles - group + ngroups - 1) / ngroups : 0;
     return pl;
   }
   pl.whole = full_waves;
-  const int total = rem * kblocks;
-  pl.ipg = (total + ngroups - 1) / ngroups;          // rem < ngroups, so ipg <= kblocks: a range touches at most two tiles
-  pl.lo = group * pl.ipg < total ? group * pl.ipg : total;
-  pl.hi = pl.lo + pl.ipg < total ? pl.lo + pl.ipg : total;
-  if (pl.lo < pl.hi) pl.pieces = (pl.lo / kblocks != (pl.hi - 1) / kblocks) ? 2 : 1;
+  pl.sk_tiles = rem;
+  pl.segs = best;
+  pl.kseg = (kblocks + best - 1) / best;               // kblocks >= 8 * segs: no segment is empty
+  const int total = rem * best;
+  pl.sk_units = group < total ? (total - group + ngroups - 1) / ngroups : 0;
   return pl;
 }
 
@@ -582,8 +591,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   }
 }
 
-// Second half of stream-K: adds up the partial tiles that gemm_tn_kernel<EPI_STORE_F32> left in p.sk_part, group after
-// group (a fixed order: the result does not depend on timing), applies the row factor and the row map and stores the
+// Second half of the K split: adds up the partial tiles that gemm_tn_kernel<EPI_STORE_F32> left in p.sk_part, group after
+// segment (a fixed order: the result does not depend on timing), applies the row factor and the row map and stores the
 // tile.  Launch with the same Params and the same number of CTA groups; grid = (ngroups - 1, TILE_M / 32), 256 threads.
 template <int CG>
 __global__ void __launch_bounds__(256) gemm_streamk_fixup_kernel(Params p, int ngroups) {
@@ -599,7 +608,6 @@ __global__ void __launch_bounds__(256) gemm_streamk_fixup_kernel(Params p, int n
   if (r >= pl.sk_tiles) return;
   const int tile = pl.first_sk_tile + r;
   const int tm = p.n_fastest ? tile / tiles_n : tile % tiles_m, nb = p.n_fastest ? tile % tiles_n : tile / tiles_m;
-  const int g0 = (r * kblocks) / pl.ipg, g1 = ((r + 1) * kblocks - 1) / pl.ipg;      // groups whose ranges meet this tile
   const int lrow = blockIdx.y * 32 + (threadIdx.x >> 3);                              // row of the tile: 32 rows per block,
   const int row = tm * C::TILE_M + lrow;                                              // 8 threads per row
   if (row >= m_lim) return;
@@ -607,9 +615,8 @@ __global__ void __launch_bounds__(256) gemm_streamk_fixup_kernel(Params p, int n
   float* out = p.C + (int64_t)(p.row_map ? p.row_map[row] : row) * p.ldc + nb * BN;
   for (int c4 = (threadIdx.x & 7); c4 < BN / 4; c4 += 8) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int g = g0; g <= g1; ++g) {
-      const int pc = ((g * pl.ipg) / kblocks == r) ? 0 : 1;       // the group's first piece lies in this tile, or its second
-      const float4 v = *reinterpret_cast<const float4*>(p.sk_part + ((int64_t)(2 * g + pc) * C::TILE_M + lrow) * BN + 4 * c4);
+    for (int sg = 0; sg < pl.segs; ++sg) {               // segment after segment: a fixed order
+      const float4 v = *reinterpret_cast<const float4*>(p.sk_part + ((int64_t)(r * pl.segs + sg) * C::TILE_M + lrow) * BN + 4 * c4);
       acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
     }
     acc.x *= sc; acc.y *= sc; acc.z *= sc; acc.w *= sc;

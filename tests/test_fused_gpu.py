@@ -449,7 +449,7 @@ def test_fused_full_size_in_row_blocks_with_a_bounded_workspace():
     T, d, V, R = 8192, 2048, 151936, 2048
     b = wl.lm_head_workload(DEV, seed=5)
     need = dppo.dppo_fused_workspace_bytes(R, d, V)
-    assert need < 0.8e9 and need == dppo.dppo_fused_workspace_bytes(min(T, R), d, V) and dppo.dppo_fused_workspace_bytes(T, d, V) > 2.4e9
+    assert need < 0.9e9 and need == dppo.dppo_fused_workspace_bytes(min(T, R), d, V) and dppo.dppo_fused_workspace_bytes(T, d, V) > 2.4e9
     ws = torch.full((need,), 0xFF, dtype=torch.uint8, device=DEV)
     W64 = b.lm_head.float().cpu().numpy().astype(np.float64)
     out = _check_all_valid_full_size(b, W64, ws, rows_per_block=R)
