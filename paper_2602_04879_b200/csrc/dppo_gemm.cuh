@@ -93,7 +93,8 @@ struct Params {
   int32_t* status;
   unsigned long long wait_ns;   // limit of every on-chip wait
   int inject;            // opts->test_inject
-  int accumulate;        // EPI_STORE_F32 (no K split, no row map): the product is added to what C holds
+  int accumulate;        // EPI_STORE_F32 (no K split, no row map): the product is added to what C holds (by reductions
+                         // performed in L2: the epilogue does not read C)
 };
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
@@ -182,6 +183,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
         "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Adds to global memory without reading it back (the addition is done by the L2 cache, the thread does not wait).
+// Used where every element of the output gets exactly one contribution per launch, so nothing depends on timing.
+__device__ __forceinline__ void red_add_f32x4(float* p, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void red_add_f32(float* p, float a) {
+  asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(a) : "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -421,25 +430,21 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
               float* ct = p.C + (int64_t)(n0 + c) * p.ldc + row;
               if (p.accumulate) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) ct[(int64_t)j * p.ldc] += __uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) red_add_f32(ct + (int64_t)j * p.ldc, __uint_as_float(r[j]));
               } else {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) ct[(int64_t)j * p.ldc] = __uint_as_float(r[j]);
               }
-            } else if (p.accumulate) {     // added to the rows finished by earlier calls (a later row block of the same dW)
+            } else if (p.accumulate) {
+              // added to what earlier launches left (a later row block of the same dW): one contribution per element
+              // and launch, launches in stream order, so the sum is the same every time
               if (n0 + c + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
-                float4 old[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) old[j] = *reinterpret_cast<const float4*>(dst + 4 * j);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  old[j].x += __uint_as_float(r[4 * j]); old[j].y += __uint_as_float(r[4 * j + 1]);
-                  old[j].z += __uint_as_float(r[4 * j + 2]); old[j].w += __uint_as_float(r[4 * j + 3]);
-                  *reinterpret_cast<float4*>(dst + 4 * j) = old[j];
-                }
+                for (int j = 0; j < 32; j += 4)
+                  red_add_f32x4(dst + j, __uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
               } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) dst[j] += __uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j) if (n0 + c + j < p.N) red_add_f32(dst + j, __uint_as_float(r[j]));
               }
             } else if (n0 + c + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
 #pragma unroll
