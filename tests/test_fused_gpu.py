@@ -278,6 +278,10 @@ def test_fused_tiny_shapes(T, d, V):
     assert torch.isfinite(out["dW"]).all() and torch.isfinite(out["dHidden"]).all()
     _check_fused(b, dppo.BINARY_TV, 0.2)
     _check_fused(b, dppo.BINARY_KL, 0.0)
+    # row blocks that leave a last block of one row (T = 65), blocks of one row, and the two-pass mode on the same shapes
+    _check_fused(b, dppo.BINARY_TV, 0.2, rows_per_block=64)
+    _check_fused(b, dppo.BINARY_KL, 0.0, rows_per_block=1 if T <= 7 else 16)
+    _check_fused(b, dppo.BINARY_TV, 0.2, two_pass=True, rows_per_block=64)
 
 
 @pytest.mark.parametrize("T,d,V,K", [(256, 128, 1024, 0), (300, 72, 1000, 6), (520, 136, 2056, 0)])
