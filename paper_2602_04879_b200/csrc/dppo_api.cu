@@ -15,7 +15,7 @@ inline size_t dtype_size(int dt) { return dt == DPPO_BF16 ? 2 : 4; }
 
 extern "C" {
 
-int dppo_version(void) { return 100; }
+int dppo_version(void) { return 200; }   // 0.2.0: dppo_opts grew (per-call switches), dppo_workspace_bytes takes the call's shape
 
 const char* dppo_error_string(int code) {
   switch (code) {
