@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         // per-thread partial: s = sum exp(z - ref); ref is the maximum of the thread's first entries
         // and moves up only when a chunk's sum shows that an entry exceeds it by > 44
         // the sampled token's entry is left out of the sums (the scalar warp adds it: 1 - pi(a) then comes from the
-        // sum over the other entries and keeps its relative accuracy when pi(a) is close to 1)
+        // sum over the other entries and keeps its relative accuracy when pi(a) is close to 1); see below how
         float ref = -INFINITY, nm = 0.f, s = 0.f;
         const RowGeom gm = row_geom<InT, SH>(p, t, row_bytes, C);
         constexpr uint32_t kChunkElems = kChunkBytes / sizeof(InT);
@@ -225,6 +225,16 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           const uint32_t sbase = slots_base + (uint32_t)pos.slot * kChunkBytes;
           const bool has_a = (c == a_chunk);                                       // warp-uniform
           if (ok) {
+            // The sampled token's entry is taken out of the sums by overwriting it with -inf in the slot, by the one
+            // thread that reads its vector (program order makes the store visible to that thread's own loads, no other
+            // thread reads that vector, and the gradient sweep reads the row from its own ring).  Selecting the entry in
+            // registers instead costs the straight-line path 2 - 3 % although it runs once per row.  The fence orders
+            // this generic-proxy write before the bulk copy that refills the slot later.
+            if (has_a && (a_loc / N) % kGroupThreads == gtid) {
+              if (sizeof(InT) == 2) asm volatile("st.shared.b16 [%0], %1;" ::"r"(sbase + a_loc * 2u), "h"((unsigned short)0xFF80) : "memory");
+              else asm volatile("st.shared.b32 [%0], %1;" ::"r"(sbase + a_loc * 4u), "r"(0xFF800000u) : "memory");
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
             // chunks that the bulk copy filled completely take the straight-line path
             const bool full_chunk = cbase + (uint32_t)kChunkBytes <= gm.xa;
             bool done = false;
@@ -240,13 +250,6 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
 #pragma unroll
                 for (int i = 0; i < N; ++i)
                   if ((uint32_t)i * (uint32_t)sizeof(InT) < gm.head) z[0][i] = -INFINITY;
-              }
-              if (has_a) {
-#pragma unroll
-                for (int k = 0; k < kVecPerThread; ++k)
-#pragma unroll
-                  for (int i = 0; i < N; ++i)
-                    if (((uint32_t)k * kGroupThreads + gtid) * N + i == a_loc) z[k][i] = -INFINITY;
               }
               if (ref == -INFINITY) {            // first chunk of the row: reference = maximum of the first entries
                 float vm = z[0][0];
@@ -295,11 +298,6 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
                       const uint32_t pos_b = cbase + off + (uint32_t)i * (uint32_t)sizeof(InT);
                       if (pos_b < gm.head || pos_b >= gm.xend) z[i] = -INFINITY;
                     }
-                  }
-                  if (has_a) {
-#pragma unroll
-                    for (int i = 0; i < N; ++i)
-                      if (off / (uint32_t)sizeof(InT) + i == a_loc) z[i] = -INFINITY;
                   }
                   float vm = z[0];
 #pragma unroll
