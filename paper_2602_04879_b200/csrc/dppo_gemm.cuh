@@ -9,8 +9,10 @@
 //   warps 2-5   epilogue: tcgen05.ld of the accumulator (one row per thread, 32 columns at a time) while the MMA warp
 //               already fills the other 256-column accumulator buffer
 // Tiles are walked M-fastest so that CTAs running at the same time share B strips through L2 (or N-fastest, on request,
-// to share A strips).  Epilogues: fp32 store with an optional row factor; exponentials against a per-row reference with
-// their row sums; per-tile softmax statistics with an online maximum; finished gradient rows.
+// to share A strips).  Epilogues: fp32 store with an optional row factor (or added to the output by L2 reductions);
+// exponentials against a per-row reference with their row sums; per-tile softmax statistics with an online maximum;
+// finished gradient rows.  With a partial-sum buffer the store variant cuts the tiles of its last, partial wave along K
+// (struct Plan) and a second kernel adds the segments up in a fixed order: no atomics, the same bits every time.
 // Every mbarrier wait is bounded; on expiry the CTA raises DPPO_STATUS_WAIT_LIMIT, skips the rest and frees its TMEM.
 //
 // CG = 2 runs the same roles on pairs of CTAs (a cluster of two SMs) with tcgen05.mma.cta_group::2: one work unit is a
