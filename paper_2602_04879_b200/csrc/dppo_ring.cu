@@ -189,9 +189,11 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
         // The sum stream runs at most one row and a few chunks ahead of the grad warps (at least one row, or
         // the grad warps could never get their coefficients).  Rows between their first and second read then
-        // occupy about #SMs x lead chunks of L2 (61 MB at V = 151936 bf16); a longer lead makes the second
-        // read miss L2, a shorter one leaves the sum warps idle.  Measured optimum on B200: C + 7.
-        const int lead = (C + 7 <= 26 || C + 2 > 26) ? ((C + 7 <= 26) ? C + 7 : C + 2) : 26;
+        // occupy about #SMs x lead chunks of L2 (71 MB at V = 151936 bf16); a longer lead makes the second
+        // read miss L2, a shorter one leaves the sum warps idle, and the chunks beyond the row are also the time
+        // the scalar warp has for a row (its stage is longest for the Top-K variants: with C + 7 they ran 3 - 8 %
+        // slower than the Binary ones, from C + 11 on all variants run alike).  Measured on B200: C + 11 .. C + 15.
+        const int lead = (C + 11 <= 30) ? C + 11 : ((C + 2 > 30) ? C + 2 : 30);
         produce_stream<InT, SH>(p, slots_base, smem, full_base, empty_base, 0, ns_sum, row_bytes, C, policy, wc,
                                 &misc->grad_chunks, (unsigned int)lead);
       } else {
