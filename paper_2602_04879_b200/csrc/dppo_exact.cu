@@ -316,14 +316,16 @@ constexpr int kXChunk = 16384;                       // bytes per tensor per slo
 constexpr int kXSlots = 6;
 constexpr int kXConsumers = 512;
 constexpr int kXWarps = kXConsumers / 32;
-constexpr int kXThreads = kXConsumers + 32;          // + producer warp
+constexpr int kXThreads = kXConsumers + 64;          // + producer warp + merger warp (one-sweep mode)
 constexpr int kXVec = kXChunk / 16 / kXConsumers;    // 16-byte vectors per thread per chunk and tensor
 constexpr int kXMiscBytes = 2048;
 static_assert(kXVec * kXConsumers * 16 == kXChunk, "chunk geometry");
 
 struct XMisc {
   unsigned long long full[kXSlots], empty[kXSlots];
-  unsigned long long red[2];             // all consumer warps have posted their partials (sweep 1 / sweep 2)
+  unsigned long long red[2];             // all consumer warps have posted their partials (two sweeps: sweep 1 / sweep 2;
+                                         // one sweep: partials buffer 0 / 1)
+  unsigned long long red_free[2];        // one sweep: the merger warp has read partials buffer 0 / 1
   Acc3 pi[2][kXWarps], mu[2][kXWarps];   // per-warp partials of a row, two rows deep: without a second sweep a warp may post
                                           // the next row's partials while another still reads this row's
   double tv[kXWarps];
@@ -354,20 +356,25 @@ __device__ __forceinline__ void to_pairs(const float* z, float2* z2) {
   for (int i = 0; i < N / 2; ++i) z2[i] = make_float2(z[2 * i], z[2 * i + 1]);
 }
 
-template <typename InT>
+// ONE: no TV output: one sweep per row pair, rows finished by the merger warp (launched with kXThreads threads);
+// otherwise two sweeps and no merger warp (launched with kXThreads - 32 threads).
+template <typename InT, bool ONE>
 __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int N = XVecOf<InT>::N;
   XMisc* misc = reinterpret_cast<XMisc*>(smem + (size_t)kXSlots * 2 * kXChunk);
   const uint32_t slots_base = smem_u32(smem);
   const uint32_t full_base = smem_u32(&misc->full[0]), empty_base = smem_u32(&misc->empty[0]), red_base = smem_u32(&misc->red[0]);
+  const uint32_t free_base = smem_u32(&misc->red_free[0]);
   const WaitCtl wc{&misc->abort_flag, p.wait_ns};
-  const int passes = p.tv ? 2 : 1;          // without a TV output the rows are read once
+  constexpr int passes = ONE ? 1 : 2;       // without a TV output the rows are read once
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     for (int i = 0; i < kXSlots; ++i) { mbar_init(full_base + 8u * i, 1); mbar_init(empty_base + 8u * i, kXWarps); }
     mbar_init(red_base, kXWarps);
     mbar_init(red_base + 8u, kXWarps);
+    mbar_init(free_base, 1);
+    mbar_init(free_base + 8u, 1);
     misc->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -404,6 +411,39 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
             bulk_load(dst + kXChunk, zm + off, bytes, bar, policy);
           }
         }
+      }
+    }
+  } else if (warp == kXWarps + 1) {
+    // ------------------------------------------------------------------ merger (one-sweep mode): finishes the rows
+    // whose partials the consumer warps have posted, so that those never wait for one another
+    if (passes == 1) {
+      uint32_t nrow = 0;
+      for (int64_t t = blockIdx.x; t < p.T; t += gridDim.x) {
+        if (p.token_mask && p.token_mask[t] == 0) continue;
+        const uint32_t pb = nrow & 1u, use = nrow >> 1;
+        if (!mbar_wait_warp(red_base + 8u * pb, use & 1u, wc)) break;
+        Acc3 xp{-INFINITY, 0.f, 0.f}, xq{-INFINITY, 0.f, 0.f};
+        if (lane < kXWarps) { xp = misc->pi[pb][lane]; xq = misc->mu[pb][lane]; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          Acc3 x{__shfl_xor_sync(0xffffffffu, xp.m, o), __shfl_xor_sync(0xffffffffu, xp.s, o), __shfl_xor_sync(0xffffffffu, xp.a, o)};
+          Acc3 y{__shfl_xor_sync(0xffffffffu, xq.m, o), __shfl_xor_sync(0xffffffffu, xq.s, o), __shfl_xor_sync(0xffffffffu, xq.a, o)};
+          xp.merge(x);
+          xq.merge(y);
+        }
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(free_base + 8u * pb);               // the partials are in registers: the buffer may be reused
+          const double lse_p = (double)xp.m + log((double)xp.s), lse_q = (double)xq.m + log((double)xq.s);
+          if (isfinite(lse_p) && isfinite(lse_q)) {
+            p.entropy[t] = (float)(lse_p - (double)xp.a / (double)xp.s);
+            p.kl[t] = kl_out((double)xq.a / (double)xq.s - lse_q + lse_p);
+          } else {
+            p.entropy[t] = 0.f; p.kl[t] = 0.f;
+            atomicOr(p.status, DPPO_STATUS_NONFINITE_ROW);
+          }
+        }
+        ++nrow;
       }
     }
   } else {
@@ -458,6 +498,20 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
         amu.merge(y);
       }
       const uint32_t pb = nrow & 1u;
+      if (passes == 1) {
+        // One sweep: the warp posts its partials and goes on with the next row; the merger warp finishes the row.
+        // Buffer pb was last used two rows ago: wait until the merger has read it.
+        bool okw = true;
+        if (lane == 0) {
+          const uint32_t use = nrow >> 1;
+          if (use > 0) okw = mbar_wait(free_base + 8u * pb, (use - 1u) & 1u, wc);
+          if (okw) { misc->pi[pb][warp] = api; misc->mu[pb][warp] = amu; mbar_arrive(red_base + 8u * pb); }
+        }
+        ok = __shfl_sync(0xffffffffu, (int)okw, 0) != 0;
+        if (!ok) break;
+        ++nrow;
+        continue;
+      }
       if (lane == 0) { misc->pi[pb][warp] = api; misc->mu[pb][warp] = amu; mbar_arrive(red_base); }
       ok = mbar_wait_warp(red_base, nrow & 1u, wc);
       if (!ok) break;
@@ -482,7 +536,6 @@ __global__ void __launch_bounds__(kXThreads, 1) dppo_exact_ring_kernel(ExactPara
           atomicOr(p.status, DPPO_STATUS_NONFINITE_ROW);
         }
       }
-      if (passes == 1) { ++nrow; continue; }
       // ---- sweep 2 (a non-finite row still drains its chunks: the producer does not know)
       const float cp = -(float)lse_p * kLog2e, cq = -(float)lse_q * kLog2e;
       float acc = 0.f;
@@ -573,12 +626,17 @@ extern "C" int dppo_exact_divergence(const void* logits, const void* mu_logits, 
   // aligned rows whose byte length is a multiple of 16 go through the shared-memory ring
   if (vec_ok && (V * (int64_t)esz) % 16 == 0 && V * (int64_t)esz < ((int64_t)1 << 31)) {
     const int smem = kXSlots * 2 * kXChunk + kXMiscBytes;
-    cudaError_t e = (dtype == DPPO_BF16)
-        ? cudaFuncSetAttribute(dppo_exact_ring_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
-        : cudaFuncSetAttribute(dppo_exact_ring_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(dppo_exact_ring_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(dppo_exact_ring_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(dppo_exact_ring_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(dppo_exact_ring_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return DPPO_ERR_CUDA;
-    if (dtype == DPPO_BF16) dppo_exact_ring_kernel<__nv_bfloat16><<<grid, kXThreads, smem, st>>>(p);
-    else dppo_exact_ring_kernel<float><<<grid, kXThreads, smem, st>>>(p);
+    const bool one = (tv == nullptr);
+    const int threads = one ? kXThreads : kXThreads - 32;
+    if (dtype == DPPO_BF16 && one) dppo_exact_ring_kernel<__nv_bfloat16, true><<<grid, threads, smem, st>>>(p);
+    else if (dtype == DPPO_BF16) dppo_exact_ring_kernel<__nv_bfloat16, false><<<grid, threads, smem, st>>>(p);
+    else if (one) dppo_exact_ring_kernel<float, true><<<grid, threads, smem, st>>>(p);
+    else dppo_exact_ring_kernel<float, false><<<grid, threads, smem, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? DPPO_OK : DPPO_ERR_CUDA;
   }
   if (dtype == DPPO_BF16) dppo_exact_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(p, vec_ok);
