@@ -561,3 +561,25 @@ def test_full_size_ragged_topk_kl_k64_whole_batch():
     assert rows_checked == 8 * len(lengths) and blocked > 0
     assert abs(sub_gpu - sub_ora) <= 1e-3 * abs(sub_ora)
     assert np.isfinite(total_gpu)
+
+
+def test_host_buffer_entry_with_more_chunks_than_loss_slots():
+    """One row per chunk and more chunks than the entry point keeps chunk losses on the device for (4096): the losses are
+    collected in between and the total still matches the device entry point; one status word serves all chunks."""
+    T, V = 4300, 520
+    logits, a, mu_logp, _, _ = wl.logits_rows(0, T, V, torch.float32, 41, DEV, sigma=2.0, zipf=1.1, sigma_mu=0.3, K=0)
+    adv = torch.where(torch.arange(T, device=DEV) % 3 == 0, -0.7, 1.0).to(torch.float32)
+    tok = (torch.arange(T, device=DEV) % 11 != 5).to(torch.uint8)
+    a = a.clone()
+    a[4200] = V + 9                                   # a bad id in a late chunk: its status bit must reach the caller
+    b = wl.Batch(logits, a, mu_logp, adv, tok, None, None)
+    dev = _run(b, dppo.BINARY_KL, 0, 0.01, dppo.KERNEL_AUTO)
+    pin = lambda x: x.cpu().pin_memory()
+    out = dppo.dppo_loss_fwd_bwd_host(pin(logits), pin(a), pin(mu_logp), pin(adv), pin(tok), dppo.BINARY_KL, 0, 0.01,
+                                      rows_per_chunk=1, want_dlogits=True, device=DEV)
+    assert out["status"] == dppo.binding.STATUS_BAD_SAMPLED_ID == int(dev["status"].item())
+    assert torch.equal(out["mask"], dev["mask"].cpu())
+    assert torch.allclose(out["divergence"], dev["divergence"].cpu(), atol=1e-7, rtol=0)
+    assert abs(out["loss"] - float(dev["loss"].item())) <= 1e-5 * abs(out["loss"]) + 1e-12
+    a_, b_ = out["dlogits"], dev["dlogits"].cpu()
+    assert torch.all((a_ - b_).abs() <= 1e-5 * b_.abs() + 1e-12)
