@@ -319,6 +319,10 @@ const char* dppo_error_string(int code);
 /* Library version: major * 10000 + minor * 100 + patch. */
 int dppo_version(void);
 
+/* sizeof(dppo_opts) as this library was built: lets a binding written in another language check that its copy of the
+ * struct has not drifted. */
+size_t dppo_opts_size(void);
+
 #ifdef __cplusplus
 }
 #endif

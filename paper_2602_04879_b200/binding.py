@@ -53,6 +53,10 @@ def lib():
             raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2602_04879_b200.build` (there is no fallback path)")
         L = ctypes.CDLL(_LIB_PATH)
         L.dppo_version.restype = c_int
+        L.dppo_opts_size.restype = c_size_t
+        if int(L.dppo_opts_size()) != ctypes.sizeof(DppoOpts):
+            raise RuntimeError(f"{_LIB_PATH}: dppo_opts is {int(L.dppo_opts_size())} bytes in the library, {ctypes.sizeof(DppoOpts)} in this binding "
+                               "(rebuild the library: `python -m paper_2602_04879_b200.build`)")
         L.dppo_error_string.restype = c_char_p
         L.dppo_error_string.argtypes = [c_int]
         L.dppo_workspace_bytes.restype = c_size_t

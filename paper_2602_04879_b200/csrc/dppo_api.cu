@@ -17,6 +17,8 @@ extern "C" {
 
 int dppo_version(void) { return 200; }   // 0.2.0: dppo_opts grew (per-call switches), dppo_workspace_bytes takes the call's shape
 
+size_t dppo_opts_size(void) { return sizeof(dppo_opts); }
+
 const char* dppo_error_string(int code) {
   switch (code) {
     case DPPO_OK: return "ok";

@@ -36,6 +36,21 @@ def test_every_declared_symbol_is_exported(binding):
     assert binding.version() >= 100
 
 
+def test_options_struct_and_workspace_sizes(binding):
+    """The binding's copy of dppo_opts has the library's size and field order (the header's struct, field by field), and
+    the fused variant's workspace in row-block mode depends on the block, not on T."""
+    B = binding
+    assert int(B.lib().dppo_opts_size()) == ctypes.sizeof(B.DppoOpts)
+    hdr = open(os.path.join(ROOT, "include", "dppo.h")).read()
+    body = re.sub(r"/\*.*?\*/", "", hdr[hdr.index("typedef struct dppo_opts {"):hdr.index("} dppo_opts;")], flags=re.S)
+    fields = re.findall(r"\b(?:float|int)\s+([a-z_]+)\s*;", body)
+    assert fields == [f[0] for f in B.DppoOpts._fields_]
+    d, V = 2048, 151936
+    whole, block = B.dppo_fused_workspace_bytes(8192, d, V), B.dppo_fused_workspace_bytes(2048, d, V)
+    assert whole > 2.5e9 and block < 0.9e9 and B.dppo_fused_workspace_bytes(2048, d, V, 20) - block > 2 * d * V - 4096
+    assert B.dppo_fused_workspace_bytes(-1, d, V) == 0
+
+
 def test_error_strings(binding):
     seen = set()
     for code in range(0, -13, -1):
