@@ -64,15 +64,36 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of the fp32 output C [rows, cols] (leading dimension ld elements) for the store epilogue: boxes of 32
+// columns (128 bytes, the swizzle span) x 32 rows.
+bool make_map_c(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+  EncodeFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+  cuuint32_t box[2] = {32u, 32u};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 constexpr int kMaxStreamKSms = 160;                         // SMs the partial-sum buffer of the workspace is sized for
 constexpr size_t kStreamKBytes = (size_t)kMaxStreamKSms * gemm::kMaxSegs * gemm::BM * gemm::BN * sizeof(float);
 
 template <int EPI, bool B_MN, int CG>
 cudaError_t launch_gemm_cg(const void* A, int64_t lda, const void* B, int64_t ldb, gemm::Params p, cudaStream_t st) {
   using C = gemm::Cfg<CG>;
-  CUtensorMap ma, mb;
+  CUtensorMap ma, mb, mc;
   if (!make_map(&ma, A, p.M, p.K, lda, gemm::BM)) return cudaErrorInvalidValue;
   if (!(B_MN ? make_map(&mb, B, p.K, p.N, ldb, gemm::BK) : make_map(&mb, B, p.N, p.K, ldb, C::B_COLS))) return cudaErrorInvalidValue;
+  // plain outputs (every row of every tile goes to its own place in C) are stored through shared memory by bulk tensor
+  // copies when the layout allows a tensor map (16-byte aligned base and row pitch)
+  p.tma_store = 0;
+  mc = ma;
+  if (EPI == gemm::EPI_STORE_F32 && !p.row_map && !p.c_transposed && !p.m_live && !p.sk_part && p.ldc % 4 == 0 &&
+      ((uintptr_t)p.C % 16) == 0 && make_map_c(&mc, p.C, p.M, p.N, p.ldc))
+    p.tma_store = 1;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -94,7 +115,7 @@ cudaError_t launch_gemm_cg(const void* A, int64_t lda, const void* B, int64_t ld
   attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (CG > 1) ? 1 : 0;
-  e = cudaLaunchKernelEx(&cfg, kernel, ma, mb, p);
+  e = cudaLaunchKernelEx(&cfg, kernel, ma, mb, mc, p);
   if (e != cudaSuccess || !p.sk_part) return e;
   // the tiles of the partial wave: their partial sums are added up in a fixed order
   gemm::gemm_streamk_fixup_kernel<CG><<<dim3((unsigned)(groups - 1), (unsigned)(C::TILE_M / 32)), 256, 0, st>>>(p, groups);

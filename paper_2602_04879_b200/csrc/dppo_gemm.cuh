@@ -9,7 +9,8 @@
 //   warps 2-5   epilogue: tcgen05.ld of the accumulator (one row per thread, 32 columns at a time) while the MMA warp
 //               already fills the other 256-column accumulator buffer
 // Tiles are walked M-fastest so that CTAs running at the same time share B strips through L2 (or N-fastest, on request,
-// to share A strips).  Epilogues: fp32 store with an optional row factor (or added to the output by L2 reductions);
+// to share A strips).  Epilogues: fp32 store with an optional row factor (or added to the output by L2 reductions; plain
+// outputs go through shared memory and bulk tensor stores / reduce-adds);
 // exponentials against a per-row reference with their row sums; per-tile softmax statistics with an online maximum;
 // finished gradient rows.  With a partial-sum buffer the store variant cuts the tiles of its last, partial wave along K
 // (struct Plan) and a second kernel adds the segments up in a fixed order: no atomics, the same bits every time.
@@ -47,7 +48,9 @@ template <int CG> struct Cfg {
   static constexpr int A_STAGE_BYTES = BM * BK * 2, B_STAGE_BYTES = B_COLS * BK * 2;
   static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
   static constexpr int STAGES = (CG == 1) ? 4 : 6;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  // store epilogue through shared memory: two buffers of 32 rows x 32 fp32 columns per epilogue warp
+  static constexpr int OUT_BYTES = 4 * 2 * 32 * 32 * 4;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 enum { EPI_STORE_F32 = 0, EPI_STATS = 1, EPI_GRAD = 2, EPI_EXP = 3 };
@@ -97,6 +100,9 @@ struct Params {
   int inject;            // opts->test_inject
   int accumulate;        // EPI_STORE_F32 (no K split, no row map): the product is added to what C holds (by reductions
                          // performed in L2: the epilogue does not read C)
+  int tma_store;         // EPI_STORE_F32 (no row map, not transposed): map_c describes C (fp32, boxes of 32 x 32, 128-byte
+                         // swizzle) and the epilogue stores (or adds) its blocks through shared memory with bulk tensor
+                         // copies: whole 128-byte lines per row instead of 16 bytes per thread and instruction
 };
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
@@ -194,6 +200,19 @@ __device__ __forceinline__ void red_add_f32x4(float* p, float a, float b, float 
 __device__ __forceinline__ void red_add_f32(float* p, float a) {
   asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(a) : "memory");
 }
+// Bulk tensor store / reduction of one 32 x 32 fp32 block from shared memory (128-byte swizzled) into C.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(src) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// at most N of this thread's bulk groups may still be reading shared memory
+template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -260,13 +279,15 @@ __device__ __forceinline__ Plan make_plan(bool allow_sk, int ntiles, int kblocks
 // then loaded as boxes of 64 columns x 64 k-rows.  CG = 2: launched as clusters of two CTAs (see the top of the file).
 template <int EPI, bool B_MN, int CG>
 __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a,
-                                                             const __grid_constant__ CUtensorMap map_b, Params p) {
+                                                             const __grid_constant__ CUtensorMap map_b,
+                                                             const __grid_constant__ CUtensorMap map_c, Params p) {
   using C = Cfg<CG>;
   constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, A_STAGE_BYTES = C::A_STAGE_BYTES;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment for the 128-byte swizzle atoms (the same offset in both CTAs of a pair)
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + STAGES * STAGE_BYTES);
+  unsigned char* out_stage = smem + STAGES * STAGE_BYTES;      // 1024-byte aligned: whole swizzle atoms
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + STAGES * STAGE_BYTES + C::OUT_BYTES);
   const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
   const uint32_t tfull0 = smem_u32(bars + 2 * STAGES), tempty0 = smem_u32(bars + 2 * STAGES + 2);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
@@ -391,7 +412,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
   } else {
     // ------------------------------------------------------------------ epilogue warps (TMEM lane quarter = warp % 4)
     const int q = warp & 3;
-    uint32_t it = 0;
+    uint32_t it = 0, out_it = 0;                 // out_it: blocks this warp has handed to bulk tensor copies
     for (int u = 0; u < pl.units(); ++u, ++it) {
       int tile, kb0, kb1, slot;
       pl.unit(u, tile, kb0, kb1, slot);
@@ -415,6 +436,40 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
           tmem_ld32(taddr + c, r);
 #pragma unroll
           for (int j = 0; j < 32; j += 4) *reinterpret_cast<uint4*>(dst + c + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+        }
+      } else if (EPI == EPI_STORE_F32 && p.tma_store) {
+        // Through shared memory: the thread writes its row's 32 columns into the warp's 32 x 32 block (16-byte pieces
+        // placed by the 128-byte swizzle, so that the 32 rows of a warp do not collide on the banks), one lane hands the
+        // block to a bulk tensor copy, which stores it, or adds it to C, 128 contiguous bytes per row; rows and columns
+        // beyond C are clipped by the tensor map.  Two blocks per warp in turn.
+        const float sc = (row_ok && p.row_scale) ? p.row_scale[row] : 1.f;
+        const uint32_t wbuf = smem_u32(out_stage) + (uint32_t)q * (2u * 4096u);
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          if (n0 + c < p.N && m0 + q * 32 < m_lim) {            // warp-uniform: the block meets C
+            const uint32_t buf = wbuf + (uint32_t)(out_it & 1u) * 4096u;
+            if (lane == 0 && out_it >= 2) bulk_wait_read<1>();  // the copy that read this buffer two blocks ago is done with it
+            __syncwarp();
+            if (p.row_scale) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * sc);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint32_t addr = buf + (uint32_t)lane * 128u + (uint32_t)((j ^ (lane & 7)) * 16);
+              asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+              if (p.accumulate) tma_reduce_add_2d(&map_c, buf, n0 + c, m0 + q * 32);
+              else tma_store_2d(&map_c, buf, n0 + c, m0 + q * 32);
+              bulk_commit();
+            }
+            ++out_it;
+          }
         }
       } else if (EPI == EPI_STORE_F32) {
 #pragma unroll 1
@@ -577,6 +632,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tn_kernel(const __grid_consta
         else mbar_arrive(tempty0 + 8 * b);
       }
     }
+    // bulk tensor copies of this warp that are still under way read its shared-memory blocks: they finish first
+    if (EPI == EPI_STORE_F32 && lane == 0 && out_it > 0) bulk_wait_all<0>();
   }
 
   __syncwarp();
