@@ -153,6 +153,19 @@ def test_qwen_topk_tv_k20(qwen_rows):
     assert torch.all(bin_["divergence"] <= out["divergence"] + 1e-6)
 
 
+@pytest.mark.parametrize("V,n_resp,resp_len", [(32000, 15, 40), (128256, 10, 31), (262144, 5, 31), (1 << 20, 3, 13)])
+def test_other_vocabulary_sizes(V, n_resp, resp_len):
+    """Vocabularies of other model families and a one-million-entry one (32 and 128 chunks of 16 KB per row: the first read then
+    leads the second by one row and two chunks instead of the usual margin), bf16, rows on a ragged last wave: Top-K KL and
+    Binary-TV with a threshold that blocks part of the rows, every output against the oracle."""
+    b = wl.qwen_vocab_rows(DEV, seed=11, n_resp=n_resp, resp_len=resp_len, V=V, K=20, group=n_resp, sigma_mu=0.2)
+    out = _run(b, dppo.TOPK_KL, 20, 1e9, dppo.KERNEL_AUTO)
+    _full_check(b, dppo.TOPK_KL, 20, _stress_delta(out["divergence"]), dppo.KERNEL_AUTO, expect_blocked=lambda k, n: 0.05 * n < k < 0.5 * n)
+    bb = wl.Batch(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, None, None)
+    out = _run(bb, dppo.BINARY_TV, 0, 1.0, dppo.KERNEL_AUTO)
+    _full_check(bb, dppo.BINARY_TV, 0, _stress_delta(out["divergence"]), dppo.KERNEL_AUTO, expect_blocked=lambda k, n: 0.05 * n < k < 0.5 * n)
+
+
 # ------------------------------------------------------------------------------------- config 4
 
 def test_ragged_topk_kl_k64():
