@@ -4,9 +4,9 @@
 //
 //   sum stream    producer warp S copies the chunks of row n+k from global memory (first touch: HBM,
 //                 L2 evict-last hint); 8 sum warps add up exp(z - ref) against a per-thread reference
-//                 (moved up only if a chunk would overflow) and hand per-warp partials to the scalar warp
-//   scalar warp   log-sum-exp, ratio, divergence, mask, loss term of the row; posts the gradient
-//                 coefficients
+//                 (moved up only if a chunk would overflow) and hand per-warp partials to a scalar warp
+//   scalar warps  (two, taking the rows in turn) log-sum-exp, ratio, divergence, mask, loss term of the
+//                 row; post the gradient coefficients
 //   grad stream   producer warp G copies the chunks of row n a second time (they were read a few
 //                 microseconds earlier by the sum stream and normally still sit in L2; evict-first
 //                 hint); 8 grad warps write the gradient with 128-bit streaming stores
@@ -29,7 +29,17 @@ constexpr int kChunkBytes = 16384;
 constexpr int kGroupThreads = 256;              // threads of the sum group and of the grad group
 constexpr int kGroupWarps = kGroupThreads / 32;
 constexpr int kVecPerThread = kChunkBytes / 16 / kGroupThreads;   // 16-byte vectors per thread per chunk
-constexpr int kRingThreads = 2 * kGroupThreads + 96;              // + scalar warp + two producer warps
+constexpr int kScalarWarps = 2;     // they take the CTA's valid rows in turn (three would put the CTA at 21 warps, which the
+                                    // register file holds only with spills: measured slower)
+constexpr int kHand = 2;            // hand-off buffers sum -> scalar -> grad: valid row n uses buffer n % kHand (4 measured the same)
+constexpr int kRingThreads = 2 * kGroupThreads + 32 * kScalarWarps + 64;   // + scalar warps + two producer warps
+static_assert(kHand >= kScalarWarps, "a buffer per scalar warp at least");
+// buffer of valid row n, parity of the barrier phase of that use, and whether the buffer has been used before
+struct Hand { uint32_t b, par; bool again; };
+__device__ __forceinline__ Hand hand_of(uint32_t n) {
+  const uint32_t u = n / (uint32_t)kHand;
+  return Hand{n - u * (uint32_t)kHand, u & 1u, n >= (uint32_t)kHand};
+}
 constexpr int kMiscBytes = 1024;                // barriers + hand-off buffers
 constexpr int kMaxSlots = 14;                   // both rings together
 static_assert(kVecPerThread * kGroupThreads * 16 == kChunkBytes, "chunk geometry");
@@ -37,12 +47,12 @@ static_assert(kVecPerThread * kGroupThreads * 16 == kChunkBytes, "chunk geometry
 struct RingMisc {
   unsigned long long full[kMaxSlots];    // chunk landed            (producer -> consumers of that ring)
   unsigned long long empty[kMaxSlots];   // chunk consumed          (consumers -> producer)
-  unsigned long long part_full[2];       // partials of a row ready (sum -> scalar)
-  unsigned long long part_empty[2];
-  unsigned long long coef_full[2];       // coefficients of a row ready (scalar -> grad)
-  unsigned long long coef_empty[2];
-  float2 part[2][kGroupWarps];           // (reference, sum of exp) per sum warp
-  RowCoef coef[2];
+  unsigned long long part_full[kHand];       // partials of a row ready (sum -> scalar)
+  unsigned long long part_empty[kHand];
+  unsigned long long coef_full[kHand];       // coefficients of a row ready (scalar -> grad)
+  unsigned long long coef_empty[kHand];
+  float2 part[kHand][kGroupWarps];           // (reference, sum of exp) per sum warp
+  RowCoef coef[kHand];
   int abort_flag;
   unsigned int grad_chunks;              // chunks the grad warps have finished (written by one lane)
 };
@@ -163,7 +173,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
       mbar_init(full_base + 8u * i, 1);
       mbar_init(empty_base + 8u * i, kGroupWarps);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kHand; ++i) {
       mbar_init(part_full + 8u * i, kGroupWarps);
       mbar_init(part_empty + 8u * i, 1);
       mbar_init(coef_full + 8u * i, 1);
@@ -180,12 +190,12 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
   const int C = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);      // chunks per row (shifted rows: of most rows)
   const int64_t t0 = blockIdx.x, G = gridDim.x;
 
-  if (warp >= 2 * kGroupWarps + 1) {
+  if (warp >= 2 * kGroupWarps + kScalarWarps) {
     // ------------------------------------------------------------------ producers (one lane each)
     // (test injection: the producers issue nothing, so that every consumer wait of the CTA runs out)
     if (lane == 0 && !(p.inject & DPPO_INJECT_NO_COPIES)) {
       uint64_t policy;
-      if (warp == 2 * kGroupWarps + 1) {
+      if (warp == 2 * kGroupWarps + kScalarWarps) {
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
         // The sum stream runs at most one row and a few chunks ahead of the grad warps (at least one row, or
         // the grad warps could never get their coefficients).  Rows between their first and second read then
@@ -329,9 +339,10 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           merge_ms(ref, s, m2, s2);
         }
         if (lane == 0) {
-          const uint32_t b = vrow & 1u;
+          const Hand h = hand_of(vrow);
+          const uint32_t b = h.b;
           bool ok = true;
-          if (vrow >= 2) ok = mbar_wait(part_empty + 8u * b, ((vrow >> 1) & 1u) ^ 1u, wc);
+          if (h.again) ok = mbar_wait(part_empty + 8u * b, h.par ^ 1u, wc);
           if (ok) {
             misc->part[b][warp] = make_float2(ref, s);
             mbar_arrive(part_full + 8u * b);
@@ -369,8 +380,9 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           }
         }
       } else {
-        const uint32_t b = vrow & 1u;
-        const bool have = mbar_wait_warp(coef_full + 8u * b, (vrow >> 1) & 1u, wc);
+        const Hand h = hand_of(vrow);
+        const uint32_t b = h.b;
+        const bool have = mbar_wait_warp(coef_full + 8u * b, h.par, wc);
         RowCoef coef = misc->coef[b];
         __syncwarp();
         if (lane == 0 && have) mbar_arrive(coef_empty + 8u * b);
@@ -444,7 +456,11 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
       meta = meta_next;
     }
   } else {
-    // ------------------------------------------------------------------ scalar warp
+    // ------------------------------------------------------------------ scalar warps
+    // The scalar warps take the CTA's valid rows in turn, so that a row's scalar stage (a dependent global load, fp64
+    // exponentials and logarithms, for the Top-K variants a gather of K logits) may take several row times: with short
+    // rows (a vocabulary of 32 000 is four chunks) one warp cannot keep up.  Rows without a sweep go to warp 0.
+    const uint32_t sw = (uint32_t)(warp - 2 * kGroupWarps);
     const double scale = p.hdr->scale;
     const bool topk = (p.variant == DPPO_TOPK_TV || p.variant == DPPO_TOPK_KL) && p.K > 0;
     uint32_t vrow = 0;
@@ -452,13 +468,19 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
     for (int64_t t = t0; t < p.T; t += G) {
       const int meta_next = load_meta(p, t + G);
       if (__shfl_sync(0xffffffffu, (int)wc.aborted(), 0)) break;
+      if (kScalarWarps > 1 && ((meta >= 0) ? (vrow % (uint32_t)kScalarWarps) : 0u) != sw) {      // another warp's row
+        if (meta >= 0) ++vrow;
+        meta = meta_next;
+        continue;
+      }
       int flags = (meta == -2) ? DPPO_STATUS_BAD_SAMPLED_ID : 0;
       float D = 0.f, r = 0.f, absdiff = 0.f;
       int M = 0;
       double g = 0.0;
       if (meta >= 0) {
         const int a = meta;
-        const uint32_t b = vrow & 1u;
+        const Hand h = hand_of(vrow);
+        const uint32_t b = h.b;
         const InT* zrow = reinterpret_cast<const InT*>(p.logits) + t * p.ld_in;
         const float z_a = to_f32<InT>(zrow[a]);                       // in flight while we wait for the partials
         // Top-K variants: this lane's list entries (positions lane, lane + 32, ...) and their logits are fetched now
@@ -479,7 +501,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
           for (int i = 0; i < kPre; ++i)
             if (id_pre[i] >= 0 && (int64_t)id_pre[i] < p.V) zk_pre[i] = to_f32<InT>(zrow[id_pre[i]]);
         }
-        const bool have = mbar_wait_warp(part_full + 8u * b, (vrow >> 1) & 1u, wc);
+        const bool have = mbar_wait_warp(part_full + 8u * b, h.par, wc);
         float2 pr = make_float2(-INFINITY, 0.f);
         if (lane < kGroupWarps) pr = misc->part[b][lane];
         __syncwarp();
@@ -518,7 +540,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) dppo_row_ring_kernel(RowParam
         }
         if (lane == 0) {
           bool ok = have;
-          if (ok && vrow >= 2) ok = mbar_wait(coef_empty + 8u * b, ((vrow >> 1) & 1u) ^ 1u, wc);
+          if (ok && h.again) ok = mbar_wait(coef_empty + 8u * b, h.par ^ 1u, wc);
           if (ok) {
             misc->coef[b] = coef;
             mbar_arrive(coef_full + 8u * b);
