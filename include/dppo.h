@@ -128,6 +128,11 @@ typedef struct dppo_opts {
                           second GEMM over the same tiles that writes the finished bf16 gradient), which rounds dlogits once,
                           so that dW carries one bf16 rounding instead of two (|error| <= 2^-8 |hidden|^T |dlogits|), at the
                           price of computing every logits tile twice (about a third more time); 0 = single pass          */
+  int row_cluster;     /* ring kernel of dppo_loss_fwd_bwd: SMs that share a row (each streams every n-th 16 KB chunk of it
+                          and the per-row sums are exchanged through distributed shared memory).  0 = automatic: 1 for rows
+                          of up to 27 chunks (V <= 221 184 bf16), 2 up to 64 chunks, then 4, so that the rows in flight
+                          between their first and second read still fit L2; 1, 2, 4 = forced.  Results do not depend on it
+                          beyond the order of the fp32 additions in the row sums */
 } dppo_opts;
 enum { DPPO_LM_HEAD_DV = 0, DPPO_LM_HEAD_VD = 1 };
 

@@ -29,14 +29,14 @@ class DppoOpts(ctypes.Structure):
     """dppo_opts of include/dppo.h (all-zero = defaults)."""
     _fields_ = [("loss_scale", c_float), ("dlogits_dtype", c_int), ("kernel", c_int), ("is_cap", c_float), ("eps_low", c_float),
                 ("lm_head_layout", c_int), ("gemm_cta_group", c_int), ("fused_rows_per_block", c_int), ("wait_limit_us", c_int),
-                ("test_inject", c_int), ("fused_two_pass", c_int)]
+                ("test_inject", c_int), ("fused_two_pass", c_int), ("row_cluster", c_int)]
 
 
 def _opts(loss_scale=0.0, dlogits_f32=False, kernel=KERNEL_AUTO, is_cap=0.0, eps_low=0.0, w_is_vd=False, cta_group=0,
-          rows_per_block=0, wait_limit_us=0, test_inject=0, two_pass=False):
+          rows_per_block=0, wait_limit_us=0, test_inject=0, two_pass=False, row_cluster=0):
     return DppoOpts(float(loss_scale), DLOGITS_F32 if dlogits_f32 else DLOGITS_SAME, int(kernel), float(is_cap), float(eps_low),
                     1 if w_is_vd else 0, int(cta_group), int(rows_per_block), int(wait_limit_us), int(test_inject),
-                    1 if two_pass else 0)
+                    1 if two_pass else 0, int(row_cluster))
 
 
 class DppoError(RuntimeError):
@@ -129,7 +129,7 @@ def _divergence_buffer(T, dev, variant, given):
 def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None, variant=BINARY_TV, K=0, delta=0.2,
                       mu_topk_ids=None, mu_topk_p=None, loss_scale=0.0, dlogits_f32=False, kernel=KERNEL_AUTO,
                       dlogits=None, want_stats=False, workspace=None, status=None, stream=None, is_cap=0.0, eps_low=0.0,
-                      given_divergence=None, wait_limit_us=0, test_inject=0):
+                      given_divergence=None, wait_limit_us=0, test_inject=0, row_cluster=0):
     """Calls ``dppo_loss_fwd_bwd`` on CUDA tensors.  Output tensors are allocated with torch unless
     given.  Returns dict(loss[1], divergence[T], mask[T], dlogits[T,V], stats[8] or None, status[1]);
     nothing is synchronised.  ``given_divergence`` [T] fp32: the per-token divergence for variant GIVEN_D (copied into
@@ -155,7 +155,8 @@ def dppo_loss_fwd_bwd(logits, sampled_ids, mu_logp, advantages, token_mask=None,
                         ("mu_topk_ids", mu_topk_ids, torch.int32), ("mu_topk_p", mu_topk_p, torch.float32)):
         if t is not None:
             assert t.is_cuda and t.dtype == dt and t.is_contiguous(), name
-    opts = _opts(loss_scale, dlogits_f32, kernel, is_cap, eps_low, wait_limit_us=wait_limit_us, test_inject=test_inject)
+    opts = _opts(loss_scale, dlogits_f32, kernel, is_cap, eps_low, wait_limit_us=wait_limit_us, test_inject=test_inject,
+                 row_cluster=row_cluster)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     with torch.cuda.device(dev):
         rc = lib().dppo_loss_fwd_bwd(_ptr(logits), T, V, logits.stride(0) if T > 0 else V, _dtype_code(logits),

@@ -60,6 +60,7 @@ int dppo_loss_fwd_bwd(const void* logits, int64_t T, int64_t V, int64_t logits_r
   if (o.dlogits_dtype != DPPO_DLOGITS_SAME && o.dlogits_dtype != DPPO_DLOGITS_F32) return DPPO_ERR_DTYPE;
   if (variant < DPPO_BINARY_TV || variant > DPPO_GIVEN_D) return DPPO_ERR_VARIANT;
   if (o.kernel < DPPO_KERNEL_AUTO || o.kernel > DPPO_KERNEL_RING || o.wait_limit_us < 0) return DPPO_ERR_UNSUPPORTED;
+  if (o.row_cluster != 0 && o.row_cluster != 1 && o.row_cluster != 2 && o.row_cluster != 4) return DPPO_ERR_UNSUPPORTED;
   if (!loss || !status) return DPPO_ERR_NULL;
   if (T > 0 && (!logits || !sampled_ids || !mu_logp || !advantages || !divergence || !mask || !dlogits)) return DPPO_ERR_NULL;
   const bool topk = (variant == DPPO_TOPK_TV || variant == DPPO_TOPK_KL);
@@ -83,7 +84,7 @@ int dppo_loss_fwd_bwd(const void* logits, int64_t T, int64_t V, int64_t logits_r
   p.sampled_ids = sampled_ids; p.mu_logp = mu_logp; p.topk_ids = mu_topk_ids; p.topk_p = mu_topk_p;
   p.adv = advantages; p.token_mask = token_mask;
   p.variant = variant; p.K = K; p.delta = delta; p.loss_scale = o.loss_scale; p.is_cap = o.is_cap; p.eps_low = o.eps_low;
-  p.wait_ns = dppo::wait_limit_ns(o.wait_limit_us); p.inject = o.test_inject;
+  p.wait_ns = dppo::wait_limit_ns(o.wait_limit_us); p.inject = o.test_inject; p.row_cluster = o.row_cluster;
   p.dlogits = dlogits; p.ld_out = dlogits_row_stride;
   p.divergence = divergence; p.mask = mask; p.loss = loss; p.stats = stats; p.status = status;
   char* ws = reinterpret_cast<char*>(workspace);

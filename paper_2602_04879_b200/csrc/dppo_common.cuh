@@ -43,6 +43,7 @@ struct RowParams {
   float eps_low;             // lower clip range of DPPO_PPO_CLIP (<= 0: delta)
   unsigned long long wait_ns;  // limit of every on-chip wait
   int inject;                // opts->test_inject
+  int row_cluster;           // opts->row_cluster (ring kernel: 0 = automatic)
   void* dlogits;
   int64_t ld_out;
   float* divergence;

@@ -14,11 +14,12 @@ DEV = "cuda:0"
 KERNELS = {"ring": dppo.KERNEL_RING, "generic": dppo.KERNEL_GENERIC}
 
 
-def _run(batch, variant, K, delta, kernel, dlogits_f32=False, loss_scale=0.0, want_stats=True, dlogits=None, is_cap=0.0, eps_low=0.0):
+def _run(batch, variant, K, delta, kernel, dlogits_f32=False, loss_scale=0.0, want_stats=True, dlogits=None, is_cap=0.0, eps_low=0.0,
+         row_cluster=0):
     out = dppo.dppo_loss_fwd_bwd(batch.logits, batch.sampled_ids, batch.mu_logp, batch.advantages, batch.token_mask,
                                  variant, K, delta, batch.mu_topk_ids, batch.mu_topk_p, loss_scale=loss_scale,
                                  dlogits_f32=dlogits_f32, kernel=kernel, want_stats=want_stats, dlogits=dlogits,
-                                 is_cap=is_cap, eps_low=eps_low)
+                                 is_cap=is_cap, eps_low=eps_low, row_cluster=row_cluster)
     torch.cuda.synchronize()
     return out
 
@@ -36,8 +37,9 @@ def _stress_delta(D):
     return float(np.float32(0.5 * (d[i] + d[i + 1])))
 
 
-def _full_check(batch, variant, K, delta, kernel, dlogits_f32=False, loss_scale=0.0, expect_blocked=None, is_cap=0.0, eps_low=0.0):
-    out = _run(batch, variant, K, delta, kernel, dlogits_f32, loss_scale, is_cap=is_cap, eps_low=eps_low)
+def _full_check(batch, variant, K, delta, kernel, dlogits_f32=False, loss_scale=0.0, expect_blocked=None, is_cap=0.0, eps_low=0.0,
+                row_cluster=0):
+    out = _run(batch, variant, K, delta, kernel, dlogits_f32, loss_scale, is_cap=is_cap, eps_low=eps_low, row_cluster=row_cluster)
     assert int(out["status"].item()) == 0
     h = P.host_inputs(batch)
     ora = P.run_oracle(h, variant, K, delta, None if loss_scale == 0.0 else loss_scale, is_cap=is_cap if is_cap > 0 else None,
@@ -164,6 +166,37 @@ def test_other_vocabulary_sizes(V, n_resp, resp_len):
     bb = wl.Batch(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, None, None)
     out = _run(bb, dppo.BINARY_TV, 0, 1.0, dppo.KERNEL_AUTO)
     _full_check(bb, dppo.BINARY_TV, 0, _stress_delta(out["divergence"]), dppo.KERNEL_AUTO, expect_blocked=lambda k, n: 0.05 * n < k < 0.5 * n)
+
+
+@pytest.mark.parametrize("row_cluster", [2, 4])
+def test_rows_shared_by_the_sms_of_a_cluster(row_cluster):
+    """``opts.row_cluster`` forced on shapes the automatic choice would give one SM per row: 2 or 4 SMs stream alternate
+    chunks of a row and exchange their partial sums.  Rows of 19 chunks with a ragged tail (the chunks do not divide evenly),
+    invalid rows (zero fill split among the SMs), shifted rows, rows of a single chunk (SMs without any chunk of the row),
+    fewer rows than clusters; every output against the oracle, and twice the same bits."""
+    b = wl.qwen_vocab_rows(DEV, seed=13, n_resp=5, resp_len=31, K=20, group=5, sigma_mu=0.2)
+    b.token_mask = (torch.arange(b.T, device=DEV) % 11 != 3).to(torch.uint8)
+    b.logits[3] = float("nan")                                  # an invalid row's content must not matter
+    out = _run(b, dppo.TOPK_KL, 20, 1e9, dppo.KERNEL_RING, row_cluster=row_cluster)
+    o1, _, _ = _full_check(b, dppo.TOPK_KL, 20, _stress_delta(out["divergence"][b.token_mask != 0]), dppo.KERNEL_RING, row_cluster=row_cluster,
+                           expect_blocked=lambda k, n: 0.05 * n < k < 0.5 * n)
+    o2 = _run(b, dppo.TOPK_KL, 20, _stress_delta(out["divergence"][b.token_mask != 0]), dppo.KERNEL_RING, row_cluster=row_cluster)
+    assert torch.equal(o1["dlogits"], o2["dlogits"]) and torch.equal(o1["loss"], o2["loss"]) and torch.equal(o1["divergence"], o2["divergence"])
+    _full_check(b, dppo.BINARY_KL, 0, 0.001, dppo.KERNEL_RING, row_cluster=row_cluster)
+    # one SM per row gives the same mask and divergence up to the order of the additions in the row sums
+    ref = _run(b, dppo.BINARY_KL, 0, 0.001, dppo.KERNEL_RING, row_cluster=1)
+    got = _run(b, dppo.BINARY_KL, 0, 0.001, dppo.KERNEL_RING, row_cluster=row_cluster)
+    assert torch.allclose(ref["divergence"], got["divergence"], atol=2e-6, rtol=1e-5)
+    # shifted rows (a vocabulary that is not a multiple of 8), several chunks, Top-K, invalid rows
+    T, V = 150, 40003
+    logits, a, mu_logp, ids, ps = wl.logits_rows(0, T, V, torch.bfloat16, 23, DEV, sigma=2.0, zipf=1.1, sigma_mu=0.5, K=5)
+    adv = torch.where(torch.arange(T, device=DEV) % 3 == 0, -1.0, 0.7).to(torch.float32)
+    tok = (torch.arange(T, device=DEV) % 7 != 2).to(torch.uint8)
+    bs = wl.Batch(logits, a, mu_logp, adv, tok, ids, ps)
+    _full_check(bs, dppo.TOPK_TV, 5, 0.01, dppo.KERNEL_RING, row_cluster=row_cluster)
+    # rows of one chunk, fp32, and fewer rows than clusters
+    _full_check(wl.tiny_binary_tv(DEV, seed=0), dppo.BINARY_TV, 0, 0.2, dppo.KERNEL_RING, row_cluster=row_cluster)
+    _full_check(wl.tiny_binary_tv(DEV, seed=2, T=3, V=4096, resp_len=1), dppo.BINARY_TV, 0, 0.01, dppo.KERNEL_RING, row_cluster=row_cluster)
 
 
 # ------------------------------------------------------------------------------------- config 4

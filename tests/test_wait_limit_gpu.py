@@ -29,16 +29,18 @@ def _small():
     return wl.tiny_binary_tv(DEV, seed=3, T=48, V=4096)
 
 
-def test_row_kernel_gives_up_and_the_next_call_is_fine():
+@pytest.mark.parametrize("row_cluster", [1, 2])
+def test_row_kernel_gives_up_and_the_next_call_is_fine(row_cluster):
+    """One SM per row, and pairs of SMs sharing the rows (they leave through their cluster barrier)."""
     b = _small()
     t0 = time.perf_counter()
-    out = dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.BINARY_TV, 0, 0.2,
+    out = dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.BINARY_TV, 0, 0.2, row_cluster=row_cluster,
                                  kernel=dppo.KERNEL_RING, wait_limit_us=LIMIT_US, test_inject=binding.INJECT_NO_COPIES)
     torch.cuda.synchronize()
     assert time.perf_counter() - t0 < 5.0                                   # a few waits of 20 ms, not the default 2 s each
     assert int(out["status"].item()) & binding.STATUS_WAIT_LIMIT
     # the same call without the injection, with the same short limit: waits take microseconds, so it never runs out
-    out = dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.BINARY_TV, 0, 0.2,
+    out = dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, dppo.BINARY_TV, 0, 0.2, row_cluster=row_cluster,
                                  kernel=dppo.KERNEL_RING, wait_limit_us=LIMIT_US)
     torch.cuda.synchronize()
     assert int(out["status"].item()) == 0
