@@ -296,13 +296,13 @@ def bench_other_configs(dppo, wl, dev, steps=100, warmup=10, n_resp=16):
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the row kernel.  Counted by ncu on the reduced
-# case of the same kernel (T = 2048 rows, 1.2 GB on the device; mean of three launches: 701.4 MB read + 564.4 MB written
+# case of the same kernel (T = 2048 rows, 1.2 GB on the device; mean of three launches: 696.1 MB read + 563.9 MB written
 # for 622.3 + 622.3 MB algorithmic; summary under profiles/) and scaled to the T = 16384 rows of a benchmark launch: the
 # traffic of this kernel is proportional to the rows it streams.  The reduced case flatters the writes a little (about
 # 58 MB of the last rows are still dirty in L2 when the kernel ends).  Tied to the hash of the kernel sources: once they
 # change the figure no longer applies and None is reported.
-TRAFFIC_BYTES_PER_LAUNCH = int(round((701.42e6 + 564.41e6) * (T_ROWS / 2048)))
-TRAFFIC_KERNEL_SHA = "418aa71419e7eb64"
+TRAFFIC_BYTES_PER_LAUNCH = int(round((696.08e6 + 563.85e6) * (T_ROWS / 2048)))
+TRAFFIC_KERNEL_SHA = "1d339af8d1e71244"
 
 
 def measured_traffic():
