@@ -130,7 +130,7 @@ typedef struct dppo_opts {
                           price of computing every logits tile twice (about a third more time); 0 = single pass          */
   int row_cluster;     /* ring kernel of dppo_loss_fwd_bwd: SMs that share a row (each streams every n-th 16 KB chunk of it
                           and the per-row sums are exchanged through distributed shared memory).  0 = automatic: 1 for rows
-                          of up to 27 chunks (V <= 221 184 bf16), 2 up to 64 chunks, then 4, so that the rows in flight
+                          of up to 20 chunks (V <= 163 840 bf16), 2 up to 64 chunks, then 4, so that the rows in flight
                           between their first and second read still fit L2; 1, 2, 4 = forced.  Results do not depend on it
                           beyond the order of the fp32 additions in the row sums */
 } dppo_opts;

@@ -642,14 +642,15 @@ static int ring_mode(const RowParams& p, int in_dtype, int out_dtype) {
 
 bool ring_layout_ok(const RowParams& p, int in_dtype, int out_dtype) { return ring_mode(p, in_dtype, out_dtype) != 0; }
 
-// CTAs that share a row.  One CTA per row needs a lead of one row plus a margin (11 chunks, 4 at the least) within the 30
-// chunks per CTA that L2 holds between the two reads: rows of up to 27 chunks.  Beyond that two CTAs share a row, and four
-// for rows of more than 64 chunks (a device of 148 SMs runs 33 clusters of four at a time, so four cost a tenth of the
-// SMs).  Measured on B200, bf16, fraction of the HBM copy peak with 1 / 2 / 4 CTAs per row: V = 151 936 (19 chunks)
-// 0.87 / 0.80 / -; 201 088 (25) 0.79 - 0.83 / 0.80 / -; 262 144 (32) 0.74 / 0.81 / 0.77; 2^20 (128) 0.66 / 0.66 / 0.69.
+// CTAs that share a row.  One CTA per row needs a lead of one row plus a margin (11 chunks) within the 30 chunks per CTA
+// that L2 holds between the two reads (a higher cap was measured slower): rows of up to 19 chunks have it in full, and
+// from 21 chunks on two CTAs per row are faster, four for rows of more than 64 chunks (a device of 148 SMs runs only 33
+// clusters of four at a time).  Measured on B200, bf16, fraction of the HBM copy peak with 1 / 2 CTAs per row: 19 chunks
+// (V = 155 648) 0.87 / 0.82; 22 chunks 0.80 / 0.84; 24 chunks 0.79 / 0.82; 27 chunks 0.79 / 0.82; 32 chunks 0.74 / 0.81
+// (four: 0.77); 128 chunks (V = 2^20) 0.66 / 0.66 (four: 0.69).
 static int ring_cluster(int64_t row_bytes) {
   const int64_t C = (row_bytes + kChunkBytes - 1) / kChunkBytes;
-  return C <= 27 ? 1 : (C <= 64 ? 2 : kMaxCluster);
+  return C <= 20 ? 1 : (C <= 64 ? 2 : kMaxCluster);
 }
 
 template <typename InT, typename OutT, bool SH, int CL>
