@@ -302,7 +302,7 @@ def bench_other_configs(dppo, wl, dev, steps=100, warmup=10, n_resp=16):
 # 58 MB of the last rows are still dirty in L2 when the kernel ends).  Tied to the hash of the kernel sources: once they
 # change the figure no longer applies and None is reported.
 TRAFFIC_BYTES_PER_LAUNCH = int(round((696.08e6 + 563.85e6) * (T_ROWS / 2048)))
-TRAFFIC_KERNEL_SHA = "f58768310a6a5709"
+TRAFFIC_KERNEL_SHA = "587001d6fe5cd0f6"
 
 
 def measured_traffic():

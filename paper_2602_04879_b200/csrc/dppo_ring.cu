@@ -685,8 +685,10 @@ static cudaError_t launch_ring_c(const RowParams& p, cudaStream_t st) {
   if (nc <= 0) {
     cfg.gridDim = dim3((unsigned)(sms / CL * CL), 1, 1);
     e = cudaOccupancyMaxActiveClusters(&nc, kernel, &cfg);
-    if (e != cudaSuccess) return e;
-    if (nc <= 0) return cudaErrorInvalidConfiguration;
+    if (e != cudaSuccess || nc <= 0) {      // no room for such clusters on this device: one CTA per row
+      (void)cudaGetLastError();
+      return launch_ring_c<InT, OutT, SH, 1>(p, st);
+    }
     if (nc > sms / CL) nc = sms / CL;
     if (dev >= 0 && dev < 64) max_clusters[dev] = nc;
   }
