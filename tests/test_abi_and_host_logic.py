@@ -122,6 +122,8 @@ def test_misuse_is_rejected_before_launch(binding):
         assert _call(B, dl=0x10000 - 2 * row, opts=o) == -9     # ends inside the logits
         assert _call(B, logits=0x10000, ld=128, dl=0x10000 + row, ld_out=128, opts=o) == -9   # interleaved rows of one allocation
     assert _call(B, opts=B.DppoOpts(0.0, 0, 0, 0.0, 0.0, 0, 0, 0, -5)) == -11      # negative wait limit
+    for bad in (-1, 3, 8):                                                          # SMs per row: 0 (automatic), 1, 2 or 4
+        assert _call(B, opts=B.DppoOpts(row_cluster=bad)) == -11
     # forcing the bulk-copy kernel on a layout it cannot take
     assert _call(B, V=63, ld=63, ld_out=64, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0.0, 0.0)) == -7     # rows shifted differently
     assert _call(B, logits=0x10002, opts=B.DppoOpts(0.0, 0, B.KERNEL_RING, 0.0, 0.0)) == -7
