@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the other streaming configurations and the exact-divergence monitor (extra objects at N=1)")
     ap.add_argument("--variants-only", action="store_true", help="run only those extra measurements (profiling aid)")
+    ap.add_argument("--vocab-sweep", action="store_true",
+                    help="run only the streaming kernel over other vocabulary sizes, with 1 and 2 SMs per row where rows are long (profiling aid)")
     return ap.parse_args()
 
 
@@ -155,6 +157,34 @@ def _time_steps(torch, fn, steps, warmup):
     e1.record()
     torch.cuda.synchronize()
     return e0.elapsed_time(e1) / steps
+
+
+def bench_vocab_sweep(dppo, wl, dev, steps=100, warmup=10):
+    """The streaming kernel at the vocabulary sizes of other model families (bf16, about 2.5 GB of logits each, Binary-TV
+    and Top-K TV with K = 20): ms per launch and fraction of the measured HBM copy peak (bytes = logits read + dlogits
+    written), with the automatic number of SMs per row and, for rows of 19 chunks of 16 KB and more, with 1 and 2 forced."""
+    import torch
+    peak, peak_src = measured_peaks()
+    out = []
+    for V in (32000, 32768, 50257, 65536, 128256, 151936, 155648, 180224, 201088, 221184, 262144):
+        T = max(148, (2_500_000_000 // (V * 2)) // 148 * 148) // 4 * 4
+        b = wl.qwen_vocab_rows(dev, seed=3, n_resp=4, resp_len=T // 4, V=V, K=20, group=4)
+        dl = torch.empty_like(b.logits)
+        ws = torch.empty(dppo.dppo_workspace_bytes(T), dtype=torch.uint8, device=dev)
+        st = torch.zeros(1, dtype=torch.int32, device=dev)
+        chunks = -(-V * 2 // 16384)
+        for cl in ((0,) if chunks < 19 else (0, 1, 2)):
+            row = {"V": V, "rows": T, "chunks_per_row": chunks, "row_cluster": cl}
+            for name, var, K in (("binary_tv", dppo.BINARY_TV, 0), ("topk_tv_k20", dppo.TOPK_TV, 20)):
+                fn = lambda: dppo.dppo_loss_fwd_bwd(b.logits, b.sampled_ids, b.mu_logp, b.advantages, None, var, K, DELTA, dlogits=dl, workspace=ws,
+                                                    status=st, mu_topk_ids=b.mu_topk_ids if K else None, mu_topk_p=b.mu_topk_p if K else None,
+                                                    row_cluster=cl)
+                ms = _time_steps(torch, fn, steps, warmup)
+                row[name] = {"ms": round(ms, 4), "frac_of_hbm_peak": round(T * V * 4 / (ms * 1e-3) / 1e9 / peak, 3)}
+            assert int(st.item()) == 0
+            out.append(row)
+        del b, dl
+    return {"peak_gbs": peak, "peak_source": "of " + peak_src, "cases": out}
 
 
 def bench_other_configs(dppo, wl, dev, steps=100, warmup=10, n_resp=16):
@@ -530,6 +560,10 @@ def run_ours(args):
     variant = dppo.BINARY_TV if args.variant == "binary_tv" else dppo.BINARY_KL
     if args.fused_only:
         print(json.dumps({"fused_lm_head": bench_fused(dppo, wl, dev, steps=max(1, min(args.steps, 40)), warmup=max(1, min(args.warmup, 10)), T=args.fused_rows)}))
+        return
+
+    if args.vocab_sweep:
+        print(json.dumps({"vocab_sweep": bench_vocab_sweep(dppo, wl, dev, steps=max(1, min(args.steps, 100)), warmup=max(1, min(args.warmup, 10)))}))
         return
 
     if args.variants_only:
